@@ -1,0 +1,150 @@
+"""ctypes front end of the CPU oracle (test infrastructure, not the product).
+
+Compiles ``oracle_a48.cpp`` with g++ on first use and exposes its entry points
+on numpy arrays.  Only tests, the smoke check and the benchmark's CPU-baseline
+leg may import this module; the CUDA library never does.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "oracle_a48.cpp")
+_LIB = os.path.join(_HERE, "liboracle_a48.so")
+_lib = None
+
+_i64 = ctypes.c_int64
+_f64 = ctypes.c_double
+
+
+class BlockParams(ctypes.Structure):
+    _fields_ = [
+        ("hidden", _i64), ("n_heads", _i64), ("head_dim", _i64), ("ffn", _i64),
+        ("B", _i64), ("T", _i64), ("pos0", _i64), ("ctx_cap", _i64),
+        ("k_o", _i64), ("k_down", _i64),
+        ("norm_eps", _f64), ("quant_eps", _f64), ("rope_base", _f64),
+    ]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle shared library (g++ only); returns its path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-ffp-contract=off", _SRC, "-o", _LIB]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a, ty):
+    return a.ctypes.data_as(ctypes.POINTER(ty)) if a is not None else None
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+def ternarise(W, eps=1e-5):
+    """Eq. 2.  Returns (codes int8 [N,K], alpha float64)."""
+    W = _f32(W)
+    N, K = W.shape
+    t = np.empty((N, K), np.int8)
+    alpha = _f64(0.0)
+    rc = _load().oracle_a48_ternarise(_p(W, ctypes.c_float), _i64(N), _i64(K), _f64(eps), _p(t, ctypes.c_int8),
+                                      ctypes.byref(alpha))
+    assert rc == 0, rc
+    return t, alpha.value
+
+
+def quant_int4(X, eps=1e-5, nthreads=1):
+    """Eq. 7.  Returns (codes int8 [M,K] in [-8,7], scale float64 [M] = beta/sqrt7)."""
+    X = _f32(X)
+    M, K = X.shape
+    q = np.empty((M, K), np.int8)
+    d = np.empty(M, np.float64)
+    rc = _load().oracle_a48_quant_int4(_p(X, ctypes.c_float), _i64(M), _i64(K), _f64(eps), _p(q, ctypes.c_int8),
+                                       _p(d, _f64), ctypes.c_int(nthreads))
+    assert rc == 0, rc
+    return q, d
+
+
+def topk_quant_int8(X, k, eps=1e-5, nthreads=1):
+    """Eq. 1 and 3.  Returns (codes int8 [M,K], scale float64 [M] = gamma/127, mask uint8 [M,K])."""
+    X = _f32(X)
+    M, K = X.shape
+    c = np.empty((M, K), np.int8)
+    d = np.empty(M, np.float64)
+    mask = np.empty((M, K), np.uint8)
+    rc = _load().oracle_a48_topk_quant_int8(_p(X, ctypes.c_float), _i64(M), _i64(K), _i64(k), _f64(eps),
+                                            _p(c, ctypes.c_int8), _p(d, _f64), _p(mask, ctypes.c_uint8),
+                                            ctypes.c_int(nthreads))
+    assert rc == 0, rc
+    return c, d, mask
+
+
+def quant_fp4(X, nthreads=1):
+    """Eq. 8-9 (E2M1).  Returns (grid codes int8 in {0,±1,±2,±3,±4,±6,±8,±12}, scale float64 [M] = |x|max/12)."""
+    X = _f32(X)
+    M, K = X.shape
+    g = np.empty((M, K), np.int8)
+    d = np.empty(M, np.float64)
+    rc = _load().oracle_a48_quant_fp4(_p(X, ctypes.c_float), _i64(M), _i64(K), _p(g, ctypes.c_int8), _p(d, _f64),
+                                      ctypes.c_int(nthreads))
+    assert rc == 0, rc
+    return g, d
+
+
+def linear(codes, scale, t, alpha, nthreads=1, want_acc=True, want_y=True):
+    """Eq. 1 / Eq. 6.  Returns (acc int64 [M,N] or None, y float64 [M,N] or None)."""
+    codes = np.ascontiguousarray(codes, dtype=np.int8)
+    t = np.ascontiguousarray(t, dtype=np.int8)
+    scale = np.ascontiguousarray(scale, dtype=np.float64)
+    M, K = codes.shape
+    N, K2 = t.shape
+    assert K == K2
+    acc = np.empty((M, N), np.int64) if want_acc else None
+    y = np.empty((M, N), np.float64) if want_y else None
+    rc = _load().oracle_a48_linear(_p(codes, ctypes.c_int8), _p(scale, _f64), _i64(M), _p(t, ctypes.c_int8),
+                                   _f64(alpha), _i64(N), _i64(K), _p(acc, _i64), _p(y, _f64),
+                                   ctypes.c_int(nthreads))
+    assert rc == 0, rc
+    return acc, y
+
+
+def block_forward(X, weights, g1, g2, *, n_heads, B, T, pos0=0, ctx_cap=0, kcache=None, vcache=None,
+                  k_o, k_down, norm_eps=1e-5, quant_eps=1e-5, rope_base=10000.0, nthreads=1):
+    """One transformer block.  ``weights`` = dict with fp32 latents q,k,v,o [H,H], gate,up [F,H], down [H,F].
+
+    Returns (out float64 [B*T,H], k_new, v_new float64 [B,n_heads,T,head_dim]).
+    """
+    X = _f32(X)
+    M, H = X.shape
+    assert M == B * T
+    F = weights["gate"].shape[0]
+    w = {n: _f32(weights[n]) for n in ("q", "k", "v", "o", "gate", "up", "down")}
+    g1 = _f32(g1)
+    g2 = _f32(g2)
+    hd = H // n_heads
+    p = BlockParams(H, n_heads, hd, F, B, T, pos0, ctx_cap, k_o, k_down, norm_eps, quant_eps, rope_base)
+    out = np.empty((M, H), np.float64)
+    k_new = np.empty((B, n_heads, T, hd), np.float64)
+    v_new = np.empty((B, n_heads, T, hd), np.float64)
+    kc = _f32(kcache) if kcache is not None else None
+    vc = _f32(vcache) if vcache is not None else None
+    cf = ctypes.c_float
+    rc = _load().oracle_a48_block_forward(ctypes.byref(p), _p(X, cf), _p(w["q"], cf), _p(w["k"], cf), _p(w["v"], cf),
+                                          _p(w["o"], cf), _p(w["gate"], cf), _p(w["up"], cf), _p(w["down"], cf),
+                                          _p(g1, cf), _p(g2, cf), _p(kc, cf), _p(vc, cf), _p(out, _f64),
+                                          _p(k_new, _f64), _p(v_new, _f64), ctypes.c_int(nthreads))
+    assert rc == 0, rc
+    return out, k_new, v_new

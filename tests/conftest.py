@@ -1,0 +1,32 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+
+
+def golden(name):
+    """Parse a tests/golden/*.txt fixture: '#' lines are citations, the rest 'key value...' rows."""
+    rows = {}
+    with open(os.path.join(ROOT, "tests", "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            parts = line.split()
+            rows[parts[0]] = [float(v) for v in parts[1:]]
+    return rows
+
+
+@pytest.fixture(scope="session")
+def oracle():
+    from oracle import oracle_a48
+    oracle_a48.build()
+    return oracle_a48
