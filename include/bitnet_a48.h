@@ -1,0 +1,198 @@
+/*
+ * bitnet_a48.h — C ABI of the B200 (sm_100a) BitLinear forward of BitNet a4.8
+ * (arXiv 2411.04965).
+ *
+ * Conventions shared by every call
+ *   - Pointers named *_dev are DEVICE memory owned by the caller and must be
+ *     16-byte aligned (BITNET_A48_ERR_ALIGNMENT otherwise).  Pointers named
+ *     *_host are host memory.  The only library-owned memory sits behind the
+ *     opaque weight / block handles and is released by the matching *_free.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work on it and return without synchronising unless the
+ *     comment of the call says otherwise.
+ *   - Matrices are row-major.  Activations are X[M,K] (M tokens, K features);
+ *     weights are W[N,K] (N output features), because the paper writes
+ *     Y = Q_a(X) · Q_w(W)^T (Eq. 1, Eq. 6).
+ *   - No call aborts or throws: every failure is a status code, and arguments
+ *     are validated on the host before anything is launched.  Inputs must be
+ *     finite; on NaN/Inf the codes are unspecified but no fault occurs.
+ *   - There is no CPU fallback: without a CUDA device every compute call
+ *     returns BITNET_A48_ERR_CUDA.
+ */
+#ifndef BITNET_A48_H
+#define BITNET_A48_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BITNET_A48_OK = 0,
+    BITNET_A48_ERR_INVALID_ARG = 1, /* null pointer, k out of range, bad enum */
+    BITNET_A48_ERR_SHAPE = 2,       /* non-positive or unsupported extent */
+    BITNET_A48_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
+    BITNET_A48_ERR_UNSUPPORTED = 4, /* requested kernel cannot run this shape / layout missing */
+    BITNET_A48_ERR_CUDA = 5,        /* a CUDA runtime call failed */
+    BITNET_A48_ERR_TIMEOUT = 6,     /* a bounded in-kernel wait gave up (see bitnet_a48_kernel_status) */
+    BITNET_A48_ERR_NOMEM = 7,       /* workspace too small or allocation failed */
+    BITNET_A48_ERR_LIMIT = 8        /* size beyond a documented fixed maximum */
+} bitnet_a48_status;
+
+/* Which activation quantiser produced the codes given to bitnet_a48_linear. */
+typedef enum {
+    BITNET_A48_ACT_INT4 = 0,      /* Eq. 7: codes in [-8,7], scale = beta/sqrt(7) */
+    BITNET_A48_ACT_TOPK_INT8 = 1, /* Eq. 1+3: codes in [-127,127], zero where masked, scale = gamma/127 */
+    BITNET_A48_ACT_FP4 = 2        /* Eq. 8-9: grid codes in {0,±1,±2,±3,±4,±6,±8,±12}, scale = |x|max/12 */
+} bitnet_a48_act;
+
+/* Packed layouts a weight handle can carry (bit mask for pack_ternary). */
+#define BITNET_A48_LAYOUT_GEMM 1u   /* tile-major, for the tcgen05 prefill kernel */
+#define BITNET_A48_LAYOUT_DECODE 2u /* fragment-major, for the weight-streaming decode kernel */
+#define BITNET_A48_LAYOUT_SPARSE 4u /* channel-major, for the zero-skipping batch-1 decode kernel */
+#define BITNET_A48_LAYOUT_ALL 7u
+
+/* Kernel selection for bitnet_a48_linear_ex (tests and benchmarks force one). */
+typedef enum {
+    BITNET_A48_ALGO_AUTO = 0,
+    BITNET_A48_ALGO_SIMPLE = 1,       /* tiled dp4a kernel, any shape; the in-tree cross-check */
+    BITNET_A48_ALGO_GEMM_TCGEN05 = 2, /* prefill: tcgen05 kind::i8, int32 accumulators in TMEM */
+    BITNET_A48_ALGO_DECODE = 3,       /* M <= 64: streams every weight byte once */
+    BITNET_A48_ALGO_DECODE_SPARSE = 4 /* M == 1: fetches only channels whose code is non-zero */
+} bitnet_a48_algo;
+
+typedef struct bitnet_a48_weight bitnet_a48_weight; /* packed ternary matrix + alpha + N, K */
+typedef struct bitnet_a48_block bitnet_a48_block;   /* one transformer block: 7 weights, 2 gains, dims */
+
+const char* bitnet_a48_status_string(bitnet_a48_status s);
+
+/* ---------------------------------------------------------------------------
+ * Weight quantiser, Eq. 2:  Q_w(W) = alpha·RoundClip(W/(alpha+eps), -1, 1),
+ * alpha = mean|W| over the whole matrix; RoundClip is Eq. 4 with round-half-to-
+ * even.  Reads W_dev (fp32 [N,K]), stores the codes at 2 bits per weight in the
+ * layouts named by layout_flags (a canonical row-major layout is always kept)
+ * and alpha (computed in float64, kept as fp32) in device memory.
+ * Allocates the handle's device buffers (cudaMalloc; may synchronise), then
+ * enqueues the packing kernels on `stream`.  *out is owned by the caller and
+ * released with bitnet_a48_weight_free.  K < 2^24 and N*K < 2^40.
+ */
+bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, float eps, unsigned layout_flags,
+                                          bitnet_a48_weight** out, void* stream);
+
+/* Expands the canonical packed layout back to one int8 code per weight
+ * (codes_dev [N,K], values in {-1,0,1}) and copies alpha to *alpha_host.
+ * Either output may be NULL.  Synchronises `stream`. */
+bitnet_a48_status bitnet_a48_weight_unpack(const bitnet_a48_weight* w, int8_t* codes_dev, float* alpha_host,
+                                           void* stream);
+/* Expands one of the optional layouts (a single BITNET_A48_LAYOUT_* bit) to
+ * int8 codes, for checking that every layout holds the same matrix. */
+bitnet_a48_status bitnet_a48_weight_unpack_layout(const bitnet_a48_weight* w, unsigned layout, int8_t* codes_dev,
+                                                  void* stream);
+bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int* K, unsigned* layout_flags);
+/* Bytes of packed weight data a kernel reads for this matrix (N*K/4 rounded up per row). */
+size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w);
+void bitnet_a48_weight_free(bitnet_a48_weight* w);
+
+/* ---------------------------------------------------------------------------
+ * Activation quantiser for the inputs of attention and FFN, Eq. 7:
+ *   per token m: beta = mean_k|x|;  codes = RoundClip(sqrt7/(beta+eps)·x, -8, 7);
+ *   scale[m] = beta/sqrt7.
+ * X_dev fp32 [M,K] -> codes_dev int8 [M,K] (one code per byte), scale_dev fp32 [M].
+ * The mean and the multiply are evaluated in float64.  K <= 2^20.
+ */
+bitnet_a48_status bitnet_a48_quant_int4(const float* X_dev, int M, int K, float eps, int8_t* codes_dev,
+                                        float* scale_dev, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Sparsify-then-quantise for the intermediate states, Eq. 1 and 3:
+ *   per token m: gamma = max_k|x|; q = RoundClip(127/(gamma+eps)·x, -128, 127);
+ *   mask = the k largest |x| (ties: lowest index first; -0 ties +0);
+ *   codes = q·mask; scale[m] = gamma/127.
+ * mask_bits_dev is NULL or uint32 [M, ceil(K/32)], bit (j%32) of word j/32 = mask of feature j.
+ * 1 <= k <= K <= 2^20.
+ */
+bitnet_a48_status bitnet_a48_topk_quant_int8(const float* X_dev, int M, int K, int k, float eps,
+                                             int8_t* codes_dev, float* scale_dev, uint32_t* mask_bits_dev,
+                                             void* stream);
+
+/* FP4 (E2M1) MinMax quantiser, Eq. 8-9: per token, 2^b = 12/|x|max, step =
+ * 2^(max(floor(log2|x·2^b|),1)-1), code = step·round(x·2^b/step) (an integer in
+ * {0,±1,±2,±3,±4,±6,±8,±12}), scale[m] = |x|max/12.  Same shapes as quant_int4. */
+bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t* codes_dev, float* scale_dev,
+                                       void* stream);
+
+/* ---------------------------------------------------------------------------
+ * BitLinear contraction and rescale, Eq. 1 / Eq. 6:
+ *   acc[m,n] = sum_k codes[m,k]·t[n,k]   (exact, int32)
+ *   Y[m,n]   = fp32(acc[m,n]) · (scale[m] · alpha)
+ * codes_dev int8 [M,K], scale_dev fp32 [M], Y_dev fp32 [M,N]; acc_dev is NULL or
+ * int32 [M,N] (the raw accumulators, for parity checks).  `kind` tells which
+ * quantiser made the codes (it selects the zero-skipping decode path for
+ * top-K inputs at M == 1; the result does not depend on it).
+ * workspace_dev: at least bitnet_a48_linear_workspace_bytes(w, M) bytes, or NULL
+ * when that is 0.  Nothing is allocated and nothing synchronises.
+ */
+bitnet_a48_status bitnet_a48_linear(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
+                                    int M, bitnet_a48_act kind, float* Y_dev, int32_t* acc_dev,
+                                    void* workspace_dev, size_t workspace_bytes, void* stream);
+/* Same, with the kernel chosen by the caller.  BITNET_A48_ERR_UNSUPPORTED when
+ * that kernel cannot run the shape or the handle lacks its layout. */
+bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
+                                       int M, bitnet_a48_act kind, bitnet_a48_algo algo, float* Y_dev,
+                                       int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
+
+/* One BitLinear end to end from HOST buffers (Eq. 6 with kind INT4, Eq. 1 with
+ * kind TOPK_INT8 and top-k count k): copies X_host fp32 [M,K] to the device,
+ * quantises, contracts, rescales and copies Y back to Y_host fp32 [M,N].
+ * X_host / Y_host should be page-locked for full copy speed.  workspace_dev
+ * must hold bitnet_a48_bitlinear_host_workspace_bytes(w, M) bytes.
+ * Synchronises `stream` before returning. */
+bitnet_a48_status bitnet_a48_bitlinear_host(const bitnet_a48_weight* w, const float* X_host, int M,
+                                            bitnet_a48_act kind, int k, float eps, float* Y_host,
+                                            void* workspace_dev, size_t workspace_bytes, void* stream);
+size_t bitnet_a48_bitlinear_host_workspace_bytes(const bitnet_a48_weight* w, int M);
+
+/* ---------------------------------------------------------------------------
+ * Transformer block in the BitNet b1.58 layout with every projection a
+ * BitLinear (Section 2.1): INT4 inputs for q,k,v and gate,up (Eq. 6-7), top-K +
+ * INT8 inputs for the attention output and FFN down projections (Eq. 1, 3),
+ * ReLU²GLU (Eq. 5).  Readings where the paper is silent: pre-RMSNorm with
+ * gains, RoPE on (i, i+head_dim/2) pairs, causal softmax attention in fp32,
+ * fp32 KV cache laid out [B][n_heads][ctx_cap][head_dim], no biases.
+ */
+typedef struct {
+    int hidden, n_heads, ffn;
+    int k_o, k_down;   /* top-k counts for the o_proj and down_proj inputs */
+    int ctx_cap;       /* positions each KV-cache row can hold */
+    float norm_eps, quant_eps, rope_base;
+} bitnet_a48_block_config;
+
+/* weights: q, k, v, o [hidden,hidden], gate, up [ffn,hidden], down [hidden,ffn] in this order.
+ * The block borrows the weight handles and the gain vectors (fp32 [hidden], device);
+ * they must outlive it. */
+bitnet_a48_status bitnet_a48_block_create(const bitnet_a48_block_config* cfg, const bitnet_a48_weight* const weights[7],
+                                          const float* gain_attn_dev, const float* gain_ffn_dev, bitnet_a48_block** out);
+void bitnet_a48_block_free(bitnet_a48_block* blk);
+size_t bitnet_a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
+/* X_dev fp32 [B*T, hidden] -> Y_dev fp32 [B*T, hidden].  Tokens of batch b sit at
+ * positions pos0..pos0+T-1; their keys/values are written into the caches at
+ * those positions and attention reads positions 0..own position.  The caches
+ * may be NULL only when pos0 == 0 and T is the whole sequence (keys/values then
+ * live in the workspace).  All kernels run on `stream`; nothing synchronises. */
+bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const float* X_dev, int B, int T, int pos0,
+                                           float* kcache_dev, float* vcache_dev, float* Y_dev, void* workspace_dev,
+                                           size_t workspace_bytes, void* stream);
+
+/* Reads the device-side status words that kernels with bounded waits set when
+ * a wait gives up (0 = no kernel has reported anything) and clears them.
+ * Synchronises the device.  words_host receives 4 values: [0] error code,
+ * [1] barrier id, [2] block index, [3] iteration. */
+bitnet_a48_status bitnet_a48_kernel_status(unsigned int words_host[4]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITNET_A48_H */

@@ -1,0 +1,404 @@
+// Transformer block around the BitLinear calls (Section 2.1, Eq. 5): RMSNorm
+// (fused into the INT4 quantiser), RoPE, causal softmax attention, ReLU²GLU and
+// the residual adds.  Everything here is fp32 glue; the contractions go through
+// the same quantiser and linear launchers the public entry points use.
+#include "internal.h"
+
+namespace {
+
+size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+struct BlockWs {
+    size_t codes, scale, q, k, v, att, hres, tmp, gate, up, rope, kc, vc, lin, total;
+};
+
+BlockWs block_ws(const bitnet_a48_block* blk, int B, int T) {
+    const size_t M = (size_t)B * T, H = blk->cfg.hidden, F = blk->cfg.ffn;
+    const size_t hd = H / blk->cfg.n_heads;
+    BlockWs w;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o += up256(bytes); return r; };
+    w.codes = take(M * (H > F ? H : F));
+    w.scale = take(M * 4);
+    w.q = take(M * H * 4);
+    w.k = take(M * H * 4);
+    w.v = take(M * H * 4);
+    w.att = take(M * H * 4);
+    w.hres = take(M * H * 4);
+    w.tmp = take(M * H * 4);
+    w.gate = take(M * F * 4);
+    w.up = take(M * F * 4);
+    w.rope = take((size_t)T * (hd / 2) * 8);
+    w.kc = take(M * H * 4);
+    w.vc = take(M * H * 4);
+    size_t lin = 0;
+    for (int i = 0; i < 7; ++i) {
+        size_t b = a48_decode_workspace_bytes(blk->w[i], (int)M);
+        lin = b > lin ? b : lin;
+    }
+    w.lin = take(lin);
+    w.total = o;
+    return w;
+}
+
+// cos/sin of position * base^(-2i/head_dim), evaluated in float64, stored as fp32.
+__global__ void rope_table_kernel(int pos0, int T, int half, double base, float2* __restrict__ table) {
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= T * half) return;
+    int t = idx / half, i = idx % half;
+    double ang = (double)(pos0 + t) * pow(base, -(double)i / (double)half);
+    double s, c;
+    sincos(ang, &s, &c);
+    table[idx] = make_float2((float)c, (float)s);
+}
+
+// Rotates q in place on (i, i+hd/2) pairs, rotates k, and stores rotated k and v
+// into the cache rows [b][h][pos0+t][:].
+__global__ void rope_cache_kernel(float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                                  const float2* __restrict__ table, int B, int T, int nh, int hd, int pos0, int cap,
+                                  float* __restrict__ kcache, float* __restrict__ vcache) {
+    const int half = hd / 2;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t total = (size_t)B * T * nh * half;
+    if (idx >= total) return;
+    int i = (int)(idx % half);
+    int h = (int)((idx / half) % nh);
+    size_t m = idx / ((size_t)half * nh);
+    int t = (int)(m % T), b = (int)(m / T);
+    float2 cs = table[t * half + i];
+    size_t src = m * (size_t)nh * hd + (size_t)h * hd + i;
+    float ql = q[src], qh = q[src + half];
+    q[src] = ql * cs.x - qh * cs.y;
+    q[src + half] = qh * cs.x + ql * cs.y;
+    float kl = k[src], kh = k[src + half];
+    size_t dst = (((size_t)b * nh + h) * cap + (pos0 + t)) * hd + i;
+    kcache[dst] = kl * cs.x - kh * cs.y;
+    kcache[dst + half] = kh * cs.x + kl * cs.y;
+    vcache[dst] = v[src];
+    vcache[dst + half] = v[src + half];
+}
+
+// Causal softmax(q k^T / sqrt(hd)) v for query tiles of 64, keys streamed in tiles
+// of 64 through shared memory, fp32 throughout, online softmax.
+// grid: (ceil(T/64), nh, B); block: 256 threads as 16 (query groups) x 16.
+template <int HDP>
+__global__ void __launch_bounds__(256) attn_tile_kernel(const float* __restrict__ q, const float* __restrict__ kcache,
+                                                        const float* __restrict__ vcache, int T, int nh, int hd,
+                                                        int pos0, int cap, float scale, float* __restrict__ out) {
+    constexpr int BQ = 64, BK = 64, LD = HDP + 4, LDS_ = BK + 1, CPT = HDP / 16;
+    extern __shared__ float smem[];
+    float* Qs = smem;               // [BQ][LD]
+    float* Ks = Qs + BQ * LD;       // [BK][LD]
+    float* Vs = Ks + BK * LD;       // [BK][LD]
+    float* Ss = Vs + BK * LD;       // [BQ][LDS_]
+    float* row_m = Ss + BQ * LDS_;  // [BQ]
+    float* row_l = row_m + BQ;
+    float* row_c = row_l + BQ;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
+    const size_t H = (size_t)nh * hd;
+    const float* kbase = kcache + ((size_t)b * nh + h) * cap * hd;
+    const float* vbase = vcache + ((size_t)b * nh + h) * cap * hd;
+
+    for (int i = tid; i < BQ * (HDP / 4); i += 256) {
+        int r = i / (HDP / 4), c4 = i % (HDP / 4);
+        float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (q0 + r < T && c4 * 4 < hd)
+            val = *reinterpret_cast<const float4*>(q + ((size_t)b * T + q0 + r) * H + (size_t)h * hd + c4 * 4);
+        *reinterpret_cast<float4*>(Qs + r * LD + c4 * 4) = val;
+    }
+    if (tid < BQ) {
+        row_m[tid] = -INFINITY;
+        row_l[tid] = 0.f;
+    }
+    float o[4][CPT];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) o[i][c] = 0.f;
+
+    const int q_last = min(q0 + BQ, T) - 1;
+    const int n_keys = pos0 + q_last + 1;  // causal: keys up to the last query's own position
+    for (int k0 = 0; k0 < n_keys; k0 += BK) {
+        __syncthreads();
+        for (int i = tid; i < BK * (HDP / 4); i += 256) {
+            int r = i / (HDP / 4), c4 = i % (HDP / 4);
+            float4 kv = make_float4(0.f, 0.f, 0.f, 0.f), vv = kv;
+            if (k0 + r < n_keys && c4 * 4 < hd) {
+                kv = *reinterpret_cast<const float4*>(kbase + (size_t)(k0 + r) * hd + c4 * 4);
+                vv = *reinterpret_cast<const float4*>(vbase + (size_t)(k0 + r) * hd + c4 * 4);
+            }
+            *reinterpret_cast<float4*>(Ks + r * LD + c4 * 4) = kv;
+            *reinterpret_cast<float4*>(Vs + r * LD + c4 * 4) = vv;
+        }
+        __syncthreads();
+        // S sub-tile: queries 4ty..4ty+3, keys tx, tx+16, tx+32, tx+48
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+#pragma unroll 4
+        for (int d = 0; d < HDP; d += 4) {
+            float4 qa[4], ka[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) qa[i] = *reinterpret_cast<const float4*>(Qs + (4 * ty + i) * LD + d);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ka[j] = *reinterpret_cast<const float4*>(Ks + (tx + 16 * j) * LD + d);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    s[i][j] += qa[i].x * ka[j].x + qa[i].y * ka[j].y + qa[i].z * ka[j].z + qa[i].w * ka[j].w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int qpos = pos0 + q0 + 4 * ty + i, kpos = k0 + tx + 16 * j;
+                Ss[(4 * ty + i) * LDS_ + tx + 16 * j] = (kpos <= qpos && kpos < n_keys) ? s[i][j] * scale : -INFINITY;
+            }
+        __syncthreads();
+        {  // online softmax: 4 threads per query row, 16 keys each
+            int r = tid >> 2, part = tid & 3;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) mx = fmaxf(mx, Ss[r * LDS_ + part * 16 + j]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            float m_old = row_m[r], m_new = fmaxf(m_old, mx);
+            float sum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                float sv = Ss[r * LDS_ + part * 16 + j];
+                float p = (sv == -INFINITY) ? 0.f : expf(sv - m_new);
+                Ss[r * LDS_ + part * 16 + j] = p;
+                sum += p;
+            }
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            float corr = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
+            __syncwarp();
+            if (part == 0) {
+                row_m[r] = m_new;
+                row_l[r] = row_l[r] * corr + sum;
+                row_c[r] = corr;
+            }
+        }
+        __syncthreads();
+        // O = O*corr + P V : queries 4ty..4ty+3, columns tx*CPT..tx*CPT+CPT-1
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float c = row_c[4 * ty + i];
+#pragma unroll
+            for (int cc = 0; cc < CPT; ++cc) o[i][cc] *= c;
+        }
+#pragma unroll 4
+        for (int kk = 0; kk < BK; ++kk) {
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = Ss[(4 * ty + i) * LDS_ + kk];
+            float vreg[CPT];
+#pragma unroll
+            for (int c4 = 0; c4 < CPT / 4; ++c4) {
+                float4 t4 = *reinterpret_cast<const float4*>(Vs + kk * LD + tx * CPT + c4 * 4);
+                vreg[c4 * 4 + 0] = t4.x; vreg[c4 * 4 + 1] = t4.y; vreg[c4 * 4 + 2] = t4.z; vreg[c4 * 4 + 3] = t4.w;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int cc = 0; cc < CPT; ++cc) o[i][cc] += p[i] * vreg[cc];
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int r = 4 * ty + i;
+        if (q0 + r >= T) continue;
+        float inv = 1.f / row_l[r];
+#pragma unroll
+        for (int cc = 0; cc < CPT; ++cc) {
+            int col = tx * CPT + cc;
+            if (col < hd) out[((size_t)b * T + q0 + r) * H + (size_t)h * hd + col] = o[i][cc] * inv;
+        }
+    }
+}
+
+// Few queries per sequence (decode): one block per (query, head, batch); the 8
+// warps stride over the keys, each lane holding hd/32 (rounded up) columns.
+template <int CPL>
+__global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__ q, const float* __restrict__ kcache,
+                                                       const float* __restrict__ vcache, int T, int nh, int hd,
+                                                       int pos0, int cap, float scale, float* __restrict__ out) {
+    __shared__ float sm_m[8], sm_l[8];
+    __shared__ float sm_o[8][32 * CPL];
+    const int t = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t H = (size_t)nh * hd;
+    const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
+    const float* kbase = kcache + ((size_t)b * nh + h) * cap * hd;
+    const float* vbase = vcache + ((size_t)b * nh + h) * cap * hd;
+    float qreg[CPL], o[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) {
+        int col = lane + 32 * c;
+        qreg[c] = col < hd ? qr[col] * scale : 0.f;
+        o[c] = 0.f;
+    }
+    float m = -INFINITY, l = 0.f;
+    const int n_keys = pos0 + t + 1;
+    for (int j = warp; j < n_keys; j += 8) {
+        float dot = 0.f;
+        float vv[CPL];
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+            int col = lane + 32 * c;
+            float kv = col < hd ? kbase[(size_t)j * hd + col] : 0.f;
+            vv[c] = col < hd ? vbase[(size_t)j * hd + col] : 0.f;
+            dot += qreg[c] * kv;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+        float m_new = fmaxf(m, dot);
+        float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+        float p = expf(dot - m_new);
+        l = l * corr + p;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) o[c] = o[c] * corr + p * vv[c];
+        m = m_new;
+    }
+    if (lane == 0) {
+        sm_m[warp] = m;
+        sm_l[warp] = l;
+    }
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) sm_o[warp][lane + 32 * c] = o[c];
+    __syncthreads();
+    if (warp == 0) {
+        float mm = -INFINITY;
+        for (int w = 0; w < 8; ++w) mm = fmaxf(mm, sm_m[w]);
+        float ll = 0.f;
+        float acc[CPL];
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) acc[c] = 0.f;
+        for (int w = 0; w < 8; ++w) {
+            if (sm_m[w] == -INFINITY) continue;
+            float f = expf(sm_m[w] - mm);
+            ll += sm_l[w] * f;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][lane + 32 * c] * f;
+        }
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+            int col = lane + 32 * c;
+            if (col < hd) out[((size_t)b * T + t) * H + (size_t)h * hd + col] = acc[c] / ll;
+        }
+    }
+}
+
+__global__ void add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ y, size_t n4) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 x = reinterpret_cast<const float4*>(a)[i], z = reinterpret_cast<const float4*>(b)[i];
+    reinterpret_cast<float4*>(y)[i] = make_float4(x.x + z.x, x.y + z.y, x.z + z.z, x.w + z.w);
+}
+
+// Eq. 5: up ⊙ ReLU²(gate), written over gate.
+__global__ void relu2glu_kernel(float* __restrict__ gate, const float* __restrict__ up, size_t n4) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 g = reinterpret_cast<float4*>(gate)[i], u = reinterpret_cast<const float4*>(up)[i];
+    auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
+    reinterpret_cast<float4*>(gate)[i] = make_float4(f(g.x, u.x), f(g.y, u.y), f(g.z, u.z), f(g.w, u.w));
+}
+
+template <int HDP>
+bitnet_a48_status launch_attn_tile(const float* q, const float* kc, const float* vc, int B, int T, int nh, int hd,
+                                   int pos0, int cap, float* out, cudaStream_t st) {
+    constexpr int LD = HDP + 4;
+    size_t smem = (size_t)(3 * 64 * LD + 64 * 65 + 3 * 64) * sizeof(float);
+    A48_CUDA_TRY(cudaFuncSetAttribute(attn_tile_kernel<HDP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((T + 63) / 64, nh, B);
+    attn_tile_kernel<HDP><<<grid, 256, smem, st>>>(q, kc, vc, T, nh, hd, pos0, cap, 1.f / sqrtf((float)hd), out);
+    return BITNET_A48_OK;
+}
+
+}  // namespace
+
+size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T) { return block_ws(blk, B, T).total; }
+
+bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X, int B, int T, int pos0,
+                                    float* kcache, float* vcache, float* Y, void* ws, size_t ws_bytes,
+                                    cudaStream_t st) {
+    const bitnet_a48_block_config& c = blk->cfg;
+    const int H = c.hidden, F = c.ffn, nh = c.n_heads, hd = H / nh, M = B * T;
+    if (hd % 4 != 0 || hd > 256 || H % 4 != 0 || F % 4 != 0) return BITNET_A48_ERR_SHAPE;
+    if (B > 65535 || nh > 65535) return BITNET_A48_ERR_SHAPE;
+    BlockWs o = block_ws(blk, B, T);
+    char* base = static_cast<char*>(ws);
+    int8_t* codes = reinterpret_cast<int8_t*>(base + o.codes);
+    float* scale = reinterpret_cast<float*>(base + o.scale);
+    float* q = reinterpret_cast<float*>(base + o.q);
+    float* k = reinterpret_cast<float*>(base + o.k);
+    float* v = reinterpret_cast<float*>(base + o.v);
+    float* att = reinterpret_cast<float*>(base + o.att);
+    float* hres = reinterpret_cast<float*>(base + o.hres);
+    float* tmp = reinterpret_cast<float*>(base + o.tmp);
+    float* gate = reinterpret_cast<float*>(base + o.gate);
+    float* up = reinterpret_cast<float*>(base + o.up);
+    float2* rope = reinterpret_cast<float2*>(base + o.rope);
+    void* lin = base + o.lin;
+    const size_t lin_bytes = ws_bytes - o.lin;
+    int cap = c.ctx_cap;
+    if (!kcache) {  // keys/values of this call only: keep them in the workspace
+        kcache = reinterpret_cast<float*>(base + o.kc);
+        vcache = reinterpret_cast<float*>(base + o.vc);
+        cap = T;
+    }
+    bitnet_a48_status s;
+#define A48_TRY(e) do { s = (e); if (s != BITNET_A48_OK) return s; } while (0)
+    auto linear = [&](int wi, bitnet_a48_act kind, float* out) {
+        return bitnet_a48_linear_ex(blk->w[wi], codes, scale, M, kind, BITNET_A48_ALGO_AUTO, out, nullptr, lin,
+                                    lin_bytes, st);
+    };
+    // attention sub-layer
+    A48_TRY(a48_launch_quant_int4(X, M, H, c.quant_eps, codes, scale, blk->g_attn, c.norm_eps, st));
+    A48_TRY(linear(0, BITNET_A48_ACT_INT4, q));
+    A48_TRY(linear(1, BITNET_A48_ACT_INT4, k));
+    A48_TRY(linear(2, BITNET_A48_ACT_INT4, v));
+    {
+        int n = T * (hd / 2);
+        rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
+        size_t total = (size_t)M * nh * (hd / 2);
+        rope_cache_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(q, k, v, rope, B, T, nh, hd, pos0, cap,
+                                                                          kcache, vcache);
+    }
+    if (T <= 8) {
+        dim3 grid(T, nh, B);
+        const float sc = 1.f / sqrtf((float)hd);
+        if (hd <= 64) attn_row_kernel<2><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
+        else if (hd <= 128) attn_row_kernel<4><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
+        else attn_row_kernel<8><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
+    } else if (hd <= 64) {
+        A48_TRY(launch_attn_tile<64>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+    } else if (hd <= 128) {
+        A48_TRY(launch_attn_tile<128>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+    } else {
+        A48_TRY(launch_attn_tile<256>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+    }
+    A48_TRY(a48_launch_topk_quant_int8(att, M, H, c.k_o, c.quant_eps, codes, scale, nullptr, st));
+    A48_TRY(linear(3, BITNET_A48_ACT_TOPK_INT8, tmp));
+    const size_t nH4 = (size_t)M * H / 4, nF4 = (size_t)M * F / 4;
+    add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
+    // feed-forward sub-layer
+    A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+    A48_TRY(linear(4, BITNET_A48_ACT_INT4, gate));
+    A48_TRY(linear(5, BITNET_A48_ACT_INT4, up));
+    relu2glu_kernel<<<(unsigned)((nF4 + 255) / 256), 256, 0, st>>>(gate, up, nF4);
+    A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
+    A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));
+    add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(hres, tmp, Y, nH4);
+#undef A48_TRY
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}

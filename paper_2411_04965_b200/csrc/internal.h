@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of libbitnet_a48.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bitnet_a48.h"
+
+#define A48_CUDA_TRY(expr)                                  \
+    do {                                                    \
+        cudaError_t err__ = (expr);                         \
+        if (err__ != cudaSuccess) return BITNET_A48_ERR_CUDA; \
+    } while (0)
+
+static inline bool a48_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline int a48_round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// 2-bit encoding of a ternary code t in every layout: e = t + 1 (0 -> -1, 1 -> 0, 2 -> +1).
+//
+// Canonical layout ("l0"): row-major [N][K4] bytes with K4 = ceil(K/4); byte j of
+// row n holds k = 4j..4j+3, the lowest two bits first; positions beyond K hold
+// code 0.
+struct bitnet_a48_weight {
+    int N, K;
+    int K4;          // bytes per canonical row
+    int Np, Kp;      // N rounded up to 256, K rounded up to 128 (tiled layouts)
+    unsigned flags;  // BITNET_A48_LAYOUT_* present
+    float* alpha_dev;      // fp32 alpha
+    double* alpha64_dev;   // float64 alpha (packing only)
+    double* partial_dev;   // per-block partial sums of |W|
+    uint8_t* l0;           // canonical layout, N*K4 bytes
+    uint8_t* gemm;         // tile-major layout, Np*Kp/4 bytes (or NULL)
+    uint8_t* decode;       // fragment-major layout (or NULL)
+    uint8_t* sparse;       // channel-major layout (or NULL)
+    size_t decode_bytes, sparse_bytes;
+};
+
+struct bitnet_a48_block {
+    bitnet_a48_block_config cfg;
+    const bitnet_a48_weight* w[7];  // q k v o gate up down
+    const float* g_attn;
+    const float* g_ffn;
+};
+
+// ---- pack.cu
+bitnet_a48_status a48_launch_pack(bitnet_a48_weight* w, const float* W_dev, float eps, cudaStream_t st);
+bitnet_a48_status a48_launch_unpack_l0(const bitnet_a48_weight* w, int8_t* codes_dev, cudaStream_t st);
+bitnet_a48_status a48_launch_unpack_layout(const bitnet_a48_weight* w, unsigned layout, int8_t* codes_dev,
+                                           cudaStream_t st);
+
+// ---- quant.cu
+// gain == nullptr: plain quantiser.  gain != nullptr: x is first RMS-normalised
+// (eps norm_eps) and multiplied by gain, rounded to fp32, then quantised.
+bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps, int8_t* codes, float* scale,
+                                        const float* gain, float norm_eps, cudaStream_t st);
+bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
+                                             float* scale, uint32_t* mask_bits, cudaStream_t st);
+bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st);
+
+// ---- linear_simple.cu
+bitnet_a48_status a48_launch_linear_simple(const bitnet_a48_weight* w, const int8_t* codes, const float* scale,
+                                           int M, float* Y, int32_t* acc, cudaStream_t st);
+
+// ---- gemm_tcgen05.cu
+bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M);
+bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
+                                          float* Y, int32_t* acc, cudaStream_t st);
+bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]);
+
+// ---- decode.cu
+bool a48_decode_supported(const bitnet_a48_weight* w, int M);
+bool a48_decode_sparse_supported(const bitnet_a48_weight* w, int M);
+size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M);
+bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
+                                    float* Y, int32_t* acc, void* ws, size_t ws_bytes, cudaStream_t st);
+bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int8_t* codes, const float* scale,
+                                           int M, float* Y, int32_t* acc, void* ws, size_t ws_bytes,
+                                           cudaStream_t st);
+
+// ---- block.cu
+size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
+bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X, int B, int T, int pos0,
+                                    float* kcache, float* vcache, float* Y, void* ws, size_t ws_bytes,
+                                    cudaStream_t st);

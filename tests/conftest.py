@@ -30,3 +30,20 @@ def oracle():
     from oracle import oracle_a48
     oracle_a48.build()
     return oracle_a48
+
+
+@pytest.fixture(scope="session")
+def a48():
+    """The ctypes binding over the CUDA library, built in-tree on first use."""
+    from paper_2411_04965_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="session")
+def cuda_dev():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("a test marked gpu ran without a CUDA device")
+    return torch.device("cuda:0")

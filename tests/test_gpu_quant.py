@@ -1,0 +1,101 @@
+"""CUDA quantisers and weight packer against the CPU oracle (bit-exact codes, masks and scales to fp32)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from parity import assert_codes_match, unpack_mask_bits
+from paper_2411_04965_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-5
+# K values: 256 (one warp per row), 1536/3200/4096 (wider groups), 8640/11008 (12 vectors per thread,
+# ragged tail), 250 and 13004 (generic path: unaligned / beyond the register-resident limit)
+SHAPES = [(32, 256), (37, 768), (19, 1536), (13, 3200), (21, 4096), (9, 8640), (11, 11008), (7, 250), (3, 13004),
+          (300, 512)]
+
+
+def _inputs(kind, M, K, seed):
+    if kind == "gauss":
+        return synth.gaussian_outlier_activations(M, K, seed)
+    return synth.student_t3(M, K, seed)
+
+
+@pytest.mark.parametrize("M,K", SHAPES)
+def test_quant_int4_matches_oracle(a48, oracle, cuda_dev, M, K):
+    x = _inputs("gauss", M, K, seed=M + K)
+    x[M // 2] = 0.0  # an all-zero token
+    codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+    q_ref, d_ref = oracle.quant_int4(x.numpy(), EPS, nthreads=4)
+    beta = d_ref * math.sqrt(7.0)
+    n_bad = assert_codes_match(codes.cpu().numpy(), q_ref, x.numpy(), math.sqrt(7.0) / (beta + EPS), "int4")
+    assert n_bad == 0 or n_bad < 1e-6 * M * K
+    assert np.array_equal(scale.cpu().numpy(), d_ref.astype(np.float32))
+    assert codes.min() >= -8 and codes.max() <= 7
+
+
+@pytest.mark.parametrize("M,K", SHAPES)
+@pytest.mark.parametrize("kfrac", [0.5, 0.0, 1.0])
+def test_topk_quant_int8_matches_oracle(a48, oracle, cuda_dev, M, K, kfrac):
+    k = max(1, min(K, int(round(kfrac * K))))
+    x = _inputs("t3", M, K, seed=2 * M + K)
+    x[0] = 0.0  # all-zero token: the first k indices win the tie
+    if M > 2:
+        x[1] = torch.round(x[1])  # many equal magnitudes, ties straddle the k-th place
+        x[2] = torch.relu(x[2]) ** 2  # ReLU²-like: about half exact zeros
+    codes, scale, bits = a48.topk_quant_int8(x.to(cuda_dev), k, EPS, want_mask=True)
+    c_ref, d_ref, m_ref = oracle.topk_quant_int8(x.numpy(), k, EPS, nthreads=4)
+    mask = unpack_mask_bits(bits.cpu().numpy(), K)
+    assert np.array_equal(mask, m_ref), "top-k mask differs"
+    assert (mask.sum(1) == k).all()
+    gamma = d_ref * 127.0
+    assert_codes_match(codes.cpu().numpy(), c_ref, x.numpy(), 127.0 / (gamma + EPS), "int8")
+    assert np.array_equal(scale.cpu().numpy(), d_ref.astype(np.float32))
+    assert np.array_equal(codes.cpu().numpy() != 0, (c_ref != 0))
+
+
+def test_topk_without_mask_output(a48, oracle, cuda_dev):
+    x = synth.student_t3(5, 1024, seed=3)
+    codes, scale, bits = a48.topk_quant_int8(x.to(cuda_dev), 512, EPS)
+    assert bits is None
+    c_ref, _, _ = oracle.topk_quant_int8(x.numpy(), 512, EPS)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+
+
+@pytest.mark.parametrize("M,K", [(16, 512), (5, 250), (3, 4096)])
+def test_quant_fp4_matches_oracle(a48, oracle, cuda_dev, M, K):
+    x = synth.student_t3(M, K, seed=M * K)
+    x[0] = 0.0
+    codes, scale = a48.quant_fp4(x.to(cuda_dev))
+    g_ref, d_ref = oracle.quant_fp4(x.numpy())
+    assert np.array_equal(codes.cpu().numpy(), g_ref)
+    assert np.array_equal(scale.cpu().numpy(), d_ref.astype(np.float32))
+
+
+@pytest.mark.parametrize("N,K", [(256, 256), (768, 256), (100, 250), (130, 384), (1536, 4096), (257, 129)])
+def test_pack_ternary_matches_oracle_in_every_layout(a48, oracle, cuda_dev, N, K):
+    W = synth.latent_weights(N, K, seed=N + K)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_ALL)
+    codes, alpha = a48.weight_unpack(w)
+    t_ref, a_ref = oracle.ternarise(W.numpy(), EPS)
+    assert np.array_equal(codes.cpu().numpy(), t_ref)
+    assert alpha == np.float32(a_ref)
+    for layout in (a48.LAYOUT_GEMM, a48.LAYOUT_DECODE, a48.LAYOUT_SPARSE):
+        again = a48.weight_unpack_layout(w, layout)
+        assert np.array_equal(again.cpu().numpy(), t_ref), f"layout {layout} holds a different matrix"
+    assert w.packed_bytes == N * ((K + 3) // 4)
+    w.free()
+
+
+def test_pack_ternary_ties_and_ternary_latents(a48, oracle, cuda_dev):
+    W = torch.tensor([[0.5, -0.5, 1.5, 1.5]] * 4, dtype=torch.float32)
+    w = a48.pack_ternary(W.to(cuda_dev), 0.0, 0)
+    codes, alpha = a48.weight_unpack(w)
+    assert codes.cpu().tolist() == [[0, 0, 1, 1]] * 4 and alpha == 1.0
+    W = synth.ternary_latents(96, 160, seed=1)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, 0)
+    codes, alpha = a48.weight_unpack(w)
+    t_ref, a_ref = oracle.ternarise(W.numpy(), EPS)
+    assert np.array_equal(codes.cpu().numpy(), t_ref) and alpha == np.float32(a_ref)
