@@ -1,0 +1,490 @@
+#!/usr/bin/env python
+"""Benchmark of the BitNet a4.8 BitLinear forward on B200.
+
+One step = the seven BitLinears of one 7B-shape transformer layer over 16384
+tokens (prefill of 4096 tokens x batch 4): the per-token quantisers (INT4 for
+the q/k/v and gate/up inputs, top-K 50 % + INT8 for the o and down inputs)
+followed by the packed-ternary contractions and their rescale.  The headline
+value is dense-equivalent TOPS (2*M*N*K summed over the seven projections,
+divided by the step time, quantisers included).  The same JSON line also
+carries the batch-1 decode figure (GB/s of packed weight bytes streamed over
+every matrix of the 32-layer model), block tokens/s, the roofline of the
+dominant kernel, the end-to-end figure with host buffers, and the CPU oracle
+timed on a bounded sample.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+For N > 1 launch with torch.distributed.run; every rank runs an independent
+replica (tokens shard with no exchange), so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+# 7B shape (model-configuration table of the paper): hidden 4096, GLU 11008, 32 heads, 32 layers
+H, F, NH, LAYERS = 4096, 11008, 32, 32
+M_PREFILL = 16384  # 4096 tokens x batch 4
+EPS = 1e-5
+PROJ = (("q", H, H, "int4"), ("k", H, H, "int4"), ("v", H, H, "int4"), ("o", H, H, "topk"),
+        ("gate", F, H, "int4"), ("up", F, H, "int4"), ("down", H, F, "topk"))
+STEP_OPS = sum(2 * M_PREFILL * n * k for _, n, k, _ in PROJ)
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), filled in from profiles/; None until a capture exists for this kernel.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.uuid = None
+        try:
+            self.uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+        except Exception:
+            pass
+        self.proc, self.out = None, None
+
+    def start(self):
+        try:
+            self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd += ["-i", self.uuid]
+            self.proc = subprocess.Popen(cmd, stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.flush()
+        self.out.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.out.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.out.name)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = sorted(s for s, p in zip(sm, power) if p >= 0.5 * max(power)) or sorted(sm)
+        return {"sm_mhz": busy[len(busy) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------------- reference arm (CPU oracle)
+def oracle_layer_sample(oracle, n_tokens, nthreads, seed=4):
+    """The seven BitLinears of one 7B-shape layer on n_tokens tokens with the CPU oracle; returns seconds."""
+    from paper_2411_04965_b200 import synth
+    xh = synth.gaussian_outlier_activations(n_tokens, H, seed).numpy()
+    sh = synth.student_t3(n_tokens, H, seed + 1).numpy()
+    sf = synth.student_t3(n_tokens, F, seed + 2).numpy()
+    codes = {}
+    rng_w = {}
+    for i, (name, n, k, _) in enumerate(PROJ):  # weight ternarisation is set-up, not part of the step
+        t, alpha = oracle.ternarise(synth.ternary_latents(n, k, seed=100 + i).numpy(), EPS)
+        rng_w[name] = (t, alpha)
+    t0 = time.perf_counter()
+    q4, d4 = oracle.quant_int4(xh, EPS, nthreads=nthreads)
+    for name in ("q", "k", "v"):
+        oracle.linear(q4, d4, *rng_w[name], nthreads=nthreads, want_acc=False)
+    c8, d8, _ = oracle.topk_quant_int8(sh, H // 2, EPS, nthreads=nthreads)
+    oracle.linear(c8, d8, *rng_w["o"], nthreads=nthreads, want_acc=False)
+    q4, d4 = oracle.quant_int4(xh, EPS, nthreads=nthreads)
+    for name in ("gate", "up"):
+        oracle.linear(q4, d4, *rng_w[name], nthreads=nthreads, want_acc=False)
+    c8, d8, _ = oracle.topk_quant_int8(sf, F // 2, EPS, nthreads=nthreads)
+    oracle.linear(c8, d8, *rng_w["down"], nthreads=nthreads, want_acc=False)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import oracle_a48 as oracle
+    oracle.build()
+    cores = len(os.sched_getaffinity(0))
+    n_tok = 16
+    for _ in range(min(args.warmup, 1)):
+        oracle_layer_sample(oracle, 4, cores)
+    times = [oracle_layer_sample(oracle, n_tok, cores) for _ in range(args.steps)]
+    t = sum(times) / len(times)
+    tops = STEP_OPS * (n_tok / M_PREFILL) / t / 1e12
+    sample = f"{n_tok} of {M_PREFILL} tokens through the 7 BitLinears of one layer per step"
+    line = {
+        "impl": "reference", "metric": "bitlinear_prefill_tops_7b", "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64 accumulators, float64 scales", "data": "synthetic",
+        "config": {"workload": "7B-shape layer, 7 BitLinears, prefill 4096 tokens x batch 4 (bounded sample)",
+                   "sample": sample},
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- our arm
+class Layer:
+    """Packed weights of one 7B-shape layer plus resident activation buffers."""
+
+    def __init__(self, a48, dev, seed, layouts):
+        from paper_2411_04965_b200 import synth
+        self.w = {}
+        for i, (name, n, k, _) in enumerate(PROJ):
+            lat = synth.ternary_latents(n, k, seed=seed * 16 + i, device=dev)
+            self.w[name] = a48.pack_ternary(lat, EPS, layouts)
+            del lat
+        torch.cuda.synchronize()
+
+
+def run_ours(args):
+    from paper_2411_04965_b200 import binding as a48
+    from paper_2411_04965_b200 import build as a48_build
+    from paper_2411_04965_b200 import synth
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the BitLinear path has no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        a48_build.build()
+    if world > 1:
+        dist.barrier()
+    a48.lib()
+    peaks = load_peaks()
+    M = M_PREFILL
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- resident inputs: larger than L2 (268 MB + 268 MB + 721 MB of fp32 activations per step)
+    layer = Layer(a48, dev, seed=4 + rank, layouts=a48.LAYOUT_ALL)
+    x_h = synth.gaussian_outlier_activations(M, H, seed=40 + rank, device=dev)
+    s_h = synth.student_t3(M, H, seed=41 + rank, device=dev)
+    s_f = synth.student_t3(M, F, seed=42 + rank, device=dev)
+    codes_h = torch.empty(M, H, dtype=torch.int8, device=dev)
+    codes_f = torch.empty(M, F, dtype=torch.int8, device=dev)
+    scale = torch.empty(M, dtype=torch.float32, device=dev)
+    y_h = torch.empty(M, H, dtype=torch.float32, device=dev)
+    y_f = torch.empty(M, F, dtype=torch.float32, device=dev)
+    gemm_events = []
+
+    def gemm(name, codes, kind, out, record):
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        a48.linear(layer.w[name], codes, scale, kind, a48.ALGO_AUTO, Y=out)
+        if record:
+            e1.record(stream)
+            gemm_events.append((name, e0, e1))
+
+    def step(record=False):
+        a48.quant_int4(x_h, EPS, codes_h, scale)
+        for name in ("q", "k", "v"):
+            gemm(name, codes_h, a48.ACT_INT4, y_h, record)
+        a48.topk_quant_int8(s_h, H // 2, EPS, codes_h, scale)
+        gemm("o", codes_h, a48.ACT_TOPK_INT8, y_h, record)
+        a48.quant_int4(x_h, EPS, codes_h, scale)
+        for name in ("gate", "up"):
+            gemm(name, codes_h, a48.ACT_INT4, y_f, record)
+        a48.topk_quant_int8(s_f, F // 2, EPS, codes_f, scale)
+        gemm("down", codes_f, a48.ACT_TOPK_INT8, y_h, record)
+        return 11  # kernel launches of this library per step
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(dev)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    launches = 0
+    for _ in range(args.steps):
+        launches += step(record=True)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = ms_total / args.steps
+    tops = STEP_OPS * world / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = sum(a.elapsed_time(b) for _, a, b in gemm_events)
+    gemm_ops = sum(2 * M * n * k for name, _, _ in gemm_events for pn, n, k, _ in PROJ if pn == name)
+    achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    int8_peak = 2.0 * peaks["bf16_tflops_sustained"]  # nominal int8:bf16 ratio of 2 on the sustained bf16 figure
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
+                "frac": achieved / int8_peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "kernel": "BitLinear contraction (prefill)", "launches": len(gemm_events),
+                "avg_launch_ms": gemm_ms / len(gemm_events),
+                "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']} peaks"}
+
+    # ---- end to end with host buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.skip_e2e:
+        xh_host = x_h.cpu().pin_memory()
+        sh_host = s_h.cpu().pin_memory()
+        sf_host = s_f.cpu().pin_memory()
+        yh_host = torch.empty(M, H, dtype=torch.float32).pin_memory()
+        yf_host = torch.empty(M, F, dtype=torch.float32).pin_memory()
+        ws_bytes = max(a48.bitlinear_host_workspace_bytes(layer.w[n], M) for n, *_ in PROJ)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
+        def step_host():
+            for name in ("q", "k", "v"):
+                a48.bitlinear_host(layer.w[name], xh_host, yh_host, a48.ACT_INT4, 0, EPS, ws)
+            a48.bitlinear_host(layer.w["o"], sh_host, yh_host, a48.ACT_TOPK_INT8, H // 2, EPS, ws)
+            for name in ("gate", "up"):
+                a48.bitlinear_host(layer.w[name], xh_host, yf_host, a48.ACT_INT4, 0, EPS, ws)
+            a48.bitlinear_host(layer.w["down"], sf_host, yh_host, a48.ACT_TOPK_INT8, F // 2, EPS, ws)
+
+        step_host()
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            step_host()
+        barrier()
+        dt = max_over_ranks((time.perf_counter() - t0) * 1e3) / n_e2e
+        h2d = 6 * M * H * 4 + M * F * 4
+        d2h = 5 * M * H * 4 + 2 * M * F * 4
+        e2e = {"value": STEP_OPS * world / (dt * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": dt, "steps": n_e2e}
+        del xh_host, sh_host, sf_host, yh_host, yf_host, ws
+
+    # ---- batch-1 decode over every matrix of the model (distinct buffers >> L2)
+    decode = None
+    if not args.skip_decode:
+        decode = bench_decode(a48, synth, dev, stream, peaks, rank)
+
+    # ---- block forward tokens/s
+    block = None
+    if not args.skip_block:
+        block = bench_block(a48, synth, dev, stream, layer)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        from oracle import oracle_a48 as oracle
+        oracle.build()
+        cores = len(os.sched_getaffinity(0))
+        n_tok = 32
+        t = oracle_layer_sample(oracle, n_tok, cores)
+        cpu_baseline = {"value": STEP_OPS * (n_tok / M) / t / 1e12, "unit": "TOPS", "cores": cores, "kind": "oracle",
+                        "sample": f"{n_tok} of {M} tokens through the 7 BitLinears of one 7B-shape layer, {t:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": "bitlinear_prefill_tops_7b", "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x int2 -> int32 (scales fp64/fp32)", "data": "synthetic",
+            "config": {"workload": "7B-shape layer (hidden 4096, GLU 11008): 7 BitLinears incl. quantisers, "
+                                   "prefill 4096 tokens x batch 4 = 16384 tokens",
+                       "l2": "inputs larger than L2 (1.26 GB of fp32 activations + 1.3 GB of outputs per step)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e,
+            "cpu_baseline": cpu_baseline, "decode": decode, "block": block,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def bench_decode(a48, synth, dev, stream, peaks, rank):
+    """Batch-1 BitLinear over all 7 x 32 matrices of the 7B shape, captured once in a CUDA graph."""
+    weights = []
+    for layer_i in range(LAYERS):
+        for i, (name, n, k, kind) in enumerate(PROJ):
+            lat = synth.ternary_latents(n, k, seed=1000 + layer_i * 8 + i + 7000 * rank, device=dev)
+            weights.append((a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE | a48.LAYOUT_SPARSE), n, k, kind))
+            del lat
+    x_h = synth.gaussian_outlier_activations(1, H, seed=50, device=dev)
+    s_h = synth.student_t3(1, H, seed=51, device=dev)
+    s_f = synth.student_t3(1, F, seed=52, device=dev)
+    c4, d4 = a48.quant_int4(x_h, EPS)
+    c8h, d8h, _ = a48.topk_quant_int8(s_h, H // 2, EPS)
+    c8f, d8f, _ = a48.topk_quant_int8(s_f, F // 2, EPS)
+    y = torch.empty(1, F, dtype=torch.float32, device=dev)
+    ws_need = max(a48.linear_workspace_bytes(w, 1) for w, *_ in weights)
+    ws = torch.empty(max(ws_need, 16), dtype=torch.uint8, device=dev)
+    packed_bytes = sum(w.packed_bytes for w, *_ in weights)
+    nz = {"int4": float((c4 != 0).float().mean()), "topk_h": float((c8h != 0).float().mean()),
+          "topk_f": float((c8f != 0).float().mean())}
+    needed_bytes = 0
+    for w, n, k, kind in weights:
+        frac = nz["int4"] if kind == "int4" else (nz["topk_h"] if k == H else nz["topk_f"])
+        needed_bytes += w.packed_bytes * frac
+
+    def chain():
+        for w, n, k, kind in weights:
+            if kind == "int4":
+                a48.linear(w, c4, d4, a48.ACT_INT4, Y=y[:, :n], workspace=ws)
+            elif k == H:
+                a48.linear(w, c8h, d8h, a48.ACT_TOPK_INT8, Y=y[:, :n], workspace=ws)
+            else:
+                a48.linear(w, c8f, d8f, a48.ACT_TOPK_INT8, Y=y[:, :n], workspace=ws)
+
+    for _ in range(2):
+        chain()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        chain()
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            chain()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    e0.record(stream)
+    for _ in range(reps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    gbs_dense = packed_bytes / (ms * 1e-3) / 1e9
+    out = {"metric": "decode_weight_stream_gbs_7b_batch1", "value": gbs_dense, "unit": "GB/s",
+           "ms_per_token_all_bitlinears": ms, "packed_weight_bytes": packed_bytes, "matrices": len(weights),
+           "hbm_peak_gbs": peaks["hbm_gbs"], "frac_of_hbm_peak": gbs_dense / peaks["hbm_gbs"],
+           "algorithmic_gbs": needed_bytes / (ms * 1e-3) / 1e9, "nonzero_code_fraction": nz,
+           "tokens_per_s": 1e3 / ms, "note": "CUDA-graph chain over 224 distinct matrices (1.6 GB >> L2); "
+           "value counts every packed byte, algorithmic_gbs only channels with a non-zero code"}
+    for w, *_ in weights:
+        w.free()
+    return out
+
+
+def bench_block(a48, synth, dev, stream, layer):
+    """Block forward tokens/s at the 7B shape: prefill 4096 x 4 and batch-1 decode at context 2048."""
+    g1 = synth.norm_gains(H, 60, device=dev)
+    g2 = synth.norm_gains(H, 61, device=dev)
+    out = {}
+    blk = a48.Block(layer.w, g1, g2, n_heads=NH, k_o=H // 2, k_down=F // 2, ctx_cap=4096)
+    # prefill
+    B, T = 4, 4096
+    x = synth.gaussian_outlier_activations(B * T, H, seed=62, device=dev)
+    ws = torch.empty(blk.workspace_bytes(B, T), dtype=torch.uint8, device=dev)
+    y = torch.empty_like(x)
+    kc = torch.zeros(B, NH, 4096, H // NH, dtype=torch.float32, device=dev)
+    vc = torch.zeros_like(kc)
+    blk.forward(x, B, T, 0, kc, vc, Y=y, workspace=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 2
+    e0.record(stream)
+    for _ in range(reps):
+        blk.forward(x, B, T, 0, kc, vc, Y=y, workspace=ws)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    out["prefill"] = {"tokens_per_s": B * T / (ms * 1e-3), "ms": ms, "B": B, "T": T}
+    # decode: one token per sequence against a 2048-token context
+    for Bd in (1, 8):
+        xd = synth.gaussian_outlier_activations(Bd, H, seed=63, device=dev)
+        kcd = synth.kv_cache(Bd, NH, 4096, H // NH, seed=64, device=dev)
+        vcd = synth.kv_cache(Bd, NH, 4096, H // NH, seed=65, device=dev)
+        yd = torch.empty_like(xd)
+        wsd = torch.empty(blk.workspace_bytes(Bd, 1), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd)
+        torch.cuda.synchronize()
+        reps = 20
+        e0.record(stream)
+        for _ in range(reps):
+            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        out[f"decode_b{Bd}"] = {"tokens_per_s": Bd / (ms * 1e-3), "ms": ms, "context": 2048}
+    blk.free()
+    out["note"] = "one 7B-shape block (fp32 attention glue included); tokens/s per block, not per model"
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-decode", action="store_true")
+    ap.add_argument("--skip-block", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
