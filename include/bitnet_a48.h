@@ -53,6 +53,9 @@ typedef enum {
 #define BITNET_A48_LAYOUT_DECODE 2u /* fragment-major, for the weight-streaming decode kernel */
 #define BITNET_A48_LAYOUT_SPARSE 4u /* channel-major, for the zero-skipping batch-1 decode kernel */
 #define BITNET_A48_LAYOUT_ALL 7u
+/* One int8 code per weight (4x the packed size); only the shared-memory-operand
+ * variant of the tensor-core kernel reads it.  Not part of LAYOUT_ALL. */
+#define BITNET_A48_LAYOUT_I8 8u
 
 /* Kernel selection for bitnet_a48_linear_ex (tests and benchmarks force one). */
 typedef enum {
@@ -60,7 +63,8 @@ typedef enum {
     BITNET_A48_ALGO_SIMPLE = 1,       /* tiled dp4a kernel, any shape; the in-tree cross-check */
     BITNET_A48_ALGO_GEMM_TCGEN05 = 2, /* prefill: tcgen05 kind::i8, int32 accumulators in TMEM */
     BITNET_A48_ALGO_DECODE = 3,       /* M <= 64: streams every weight byte once */
-    BITNET_A48_ALGO_DECODE_SPARSE = 4 /* M == 1: fetches only channels whose code is non-zero */
+    BITNET_A48_ALGO_DECODE_SPARSE = 4, /* M == 1: fetches only channels whose code is non-zero */
+    BITNET_A48_ALGO_GEMM_TCGEN05_I8 = 5 /* comparison variant: int8 weight copy staged through shared memory */
 } bitnet_a48_algo;
 
 typedef struct bitnet_a48_weight bitnet_a48_weight; /* packed ternary matrix + alpha + N, K */

@@ -25,6 +25,7 @@ void free_weight_buffers(bitnet_a48_weight* w) {
     cudaFree(w->gemm);
     cudaFree(w->decode);
     cudaFree(w->sparse);
+    cudaFree(w->i8);
 }
 
 bitnet_a48_status check_act_args(const void* X, int M, int K, const void* codes, const void* scale) {
@@ -56,7 +57,7 @@ const char* bitnet_a48_status_string(bitnet_a48_status s) {
 
 bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, float eps, unsigned layout_flags,
                                           bitnet_a48_weight** out, void* stream) {
-    if (!W_dev || !out || (layout_flags & ~BITNET_A48_LAYOUT_ALL) || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
+    if (!W_dev || !out || (layout_flags & ~(BITNET_A48_LAYOUT_ALL | BITNET_A48_LAYOUT_I8)) || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
     if (N <= 0 || K <= 0 || K >= (1 << 24) || (size_t)N * (size_t)K >= ((size_t)1 << 40)) return BITNET_A48_ERR_SHAPE;
     if (!a48_aligned16(W_dev)) return BITNET_A48_ERR_ALIGNMENT;
     if (!have_device()) return BITNET_A48_ERR_CUDA;
@@ -76,6 +77,7 @@ bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, floa
     if (ok && (layout_flags & BITNET_A48_LAYOUT_GEMM)) ok = cudaMalloc(&w->gemm, (size_t)w->Np * w->Kp / 4) == cudaSuccess;
     if (ok && (layout_flags & BITNET_A48_LAYOUT_DECODE)) ok = cudaMalloc(&w->decode, w->decode_bytes) == cudaSuccess;
     if (ok && (layout_flags & BITNET_A48_LAYOUT_SPARSE)) ok = cudaMalloc(&w->sparse, w->sparse_bytes) == cudaSuccess;
+    if (ok && (layout_flags & BITNET_A48_LAYOUT_I8)) ok = cudaMalloc(&w->i8, (size_t)w->Np * w->Kp) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         free_weight_buffers(w);
@@ -165,7 +167,7 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
                                        int M, bitnet_a48_act kind, bitnet_a48_algo algo, float* Y_dev,
                                        int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
     if (!w || !codes_dev || !scale_dev || !Y_dev) return BITNET_A48_ERR_INVALID_ARG;
-    if ((int)kind < 0 || (int)kind > 2 || (int)algo < 0 || (int)algo > 4) return BITNET_A48_ERR_INVALID_ARG;
+    if ((int)kind < 0 || (int)kind > 2 || (int)algo < 0 || (int)algo > 5) return BITNET_A48_ERR_INVALID_ARG;
     if (M <= 0) return BITNET_A48_ERR_SHAPE;
     if (!a48_aligned16(codes_dev) || !a48_aligned16(scale_dev) || !a48_aligned16(Y_dev) || !a48_aligned16(acc_dev) ||
         !a48_aligned16(workspace_dev))
@@ -177,7 +179,7 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
             algo = BITNET_A48_ALGO_DECODE_SPARSE;
         else if (a48_decode_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE;
-        else if (a48_gemm_tcgen05_supported(w, M))
+        else if (a48_gemm_tcgen05_supported(w, M, false))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05;
         else
             algo = BITNET_A48_ALGO_SIMPLE;
@@ -186,8 +188,11 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
         case BITNET_A48_ALGO_SIMPLE:
             return a48_launch_linear_simple(w, codes_dev, scale_dev, M, Y_dev, acc_dev, st);
         case BITNET_A48_ALGO_GEMM_TCGEN05:
-            if (!a48_gemm_tcgen05_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
-            return a48_launch_gemm_tcgen05(w, codes_dev, scale_dev, M, Y_dev, acc_dev, st);
+            if (!a48_gemm_tcgen05_supported(w, M, false)) return BITNET_A48_ERR_UNSUPPORTED;
+            return a48_launch_gemm_tcgen05(w, codes_dev, scale_dev, M, Y_dev, acc_dev, false, st);
+        case BITNET_A48_ALGO_GEMM_TCGEN05_I8:
+            if (!a48_gemm_tcgen05_supported(w, M, true)) return BITNET_A48_ERR_UNSUPPORTED;
+            return a48_launch_gemm_tcgen05(w, codes_dev, scale_dev, M, Y_dev, acc_dev, true, st);
         case BITNET_A48_ALGO_DECODE:
             if (!a48_decode_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
             return a48_launch_decode(w, codes_dev, scale_dev, M, Y_dev, acc_dev, workspace_dev, workspace_bytes, st);

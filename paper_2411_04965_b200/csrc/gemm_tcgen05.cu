@@ -1,9 +1,475 @@
-// placeholder until the tcgen05 kernel lands
+// Prefill BitLinear contraction (Eq. 1 / Eq. 6) on the 5th-generation tensor cores:
+// tcgen05.mma kind::i8 (s8 x s8 -> s32) with the accumulators in tensor memory.
+//
+// Orientation.  The MMA computes D[128 x 256] = A[128 x K] * B[K x 256] with
+//   A = a tile of 128 weight rows (output features n), expanded to int8 codes,
+//   B = a tile of 256 tokens of activation codes (row-major [M,K] is exactly the
+//       K-major operand layout the MMA wants),
+// so the accumulator holds Y^T: TMEM lane = output feature, TMEM column = token.
+// The epilogue thread that owns lane n writes Y[m, n] for consecutive m, which
+// makes every warp store a contiguous 128-byte run of one output row.
+//
+// Two variants share the pipeline:
+//   TS (default): the 2-bit weights are read straight from global memory (L2
+//       resident) by four expander warps, widened to int8 in registers with a
+//       byte-permute lookup, and written into tensor memory with tcgen05.st; the
+//       MMA takes A from tensor memory.  The weights never occupy shared memory,
+//       whose bandwidth is left to the activation operand.
+//   SS: both operands come from shared memory via TMA; A is a pre-expanded int8
+//       copy of the weights (BITNET_A48_LAYOUT_I8).  Comparison / bring-up variant.
+//
+// Warp roles (one persistent CTA per SM): warp 0 TMA producer, warp 1 MMA issuer
+// and TMEM owner, warps 2-5 weight expanders (TS only), warps 6-9 epilogue.
+// Every mbarrier wait is bounded; a wait that gives up records a status word and
+// the CTA drains and exits without touching tensor memory again.
+#include <cuda.h>
+
 #include "internal.h"
-bool a48_gemm_tcgen05_supported(const bitnet_a48_weight*, int) { return false; }
-bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight*, const int8_t*, const float*, int, float*, int32_t*,
-                                          cudaStream_t) { return BITNET_A48_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
+constexpr int TILE_M = 256;  // tokens per tile       (MMA N)
+constexpr int BK = 128;      // channels per pipeline stage = one 128-byte swizzle row of int8
+constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
+constexpr int A_STAGES = 8;  // tensor-memory stages of the expanded weight operand (32 columns each)
+constexpr int A_COLS = BK / 4;
+constexpr int ACC_COLS = TILE_M;
+constexpr int TMEM_COLS = 512;
+constexpr int B_TILE_BYTES = TILE_M * BK;
+constexpr int A_TILE_BYTES = TILE_N * BK;
+constexpr int NUM_THREADS = 320;
+constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
+
+template <bool TS>
+struct Cfg {
+    static constexpr int STAGES = TS ? 6 : 4;
+    static constexpr int STAGE_BYTES = B_TILE_BYTES + (TS ? 0 : A_TILE_BYTES);
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 1024 /*barriers*/;
+};
+
+__device__ unsigned int g_status[4];
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting or the wait ran out of
+// time; in the latter case the first such event is recorded in g_status.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id,
+                                       uint32_t iter) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = clock64();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitClocks) {
+                *abort_flag = 1;
+                if (atomicCAS(&g_status[0], 0u, (unsigned)BITNET_A48_ERR_TIMEOUT) == 0u) {
+                    g_status[1] = id;
+                    g_status[2] = blockIdx.x;
+                    g_status[3] = iter;
+                }
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile whose rows are 128
+// bytes, laid down by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);        // start address, bits [0,14)
+    d |= (uint64_t)(1024u >> 4) << 32;              // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                         // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                         // layout type: 128-byte swizzle
+    return d;
+}
+
+// kind::i8 instruction descriptor: s8 x s8 -> s32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(0u), "r"(sel));
+    return d;
+}
+
+// One packed word (16 fields e = t+1) -> four words of int8 codes, in the field
+// order of the tile-major layout: output q takes the fields at bits s_q + 4j,
+// s_q = {0, 2, 16, 18}.  Two fields share a nibble, so after masking every
+// nibble is a selector 0..2 into the byte table {-1, 0, +1}.
+__device__ __forceinline__ void expand_word(uint32_t p, uint32_t* out) {
+    constexpr uint32_t kTable = 0x000100ffu;
+    const uint32_t q = p & 0x33333333u, r = (p >> 2) & 0x33333333u;
+    out[0] = prmt(kTable, q);
+    out[1] = prmt(kTable, r);
+    out[2] = prmt(kTable, q >> 16);
+    out[3] = prmt(kTable, r >> 16);
+}
+
+struct GemmParams {
+    const uint8_t* wt;    // tile-major packed weights (TS)
+    const float* scale;   // [M]
+    const float* alpha;   // device scalar
+    float* Y;             // [M, N]
+    int32_t* acc;         // [M, N] or nullptr
+    int M, N, K;
+    int kblocks, n_tiles, m_tiles;
+};
+
+template <bool TS>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+    gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
+                        const GemmParams p) {
+    using C = Cfg<TS>;
+    constexpr int STAGES = C::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* ctrl = smem + STAGES * C::STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] aempty[A] acc_full acc_empty
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 512);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 516);
+
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
+    const uint32_t bar_afull = bar_empty + 8 * STAGES, bar_aempty = bar_afull + 8 * A_STAGES;
+    const uint32_t bar_acc_full = bar_aempty + 8 * A_STAGES, bar_acc_empty = bar_acc_full + 8;
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < A_STAGES; ++s) {
+            mbar_init(bar_afull + 8 * s, 128);
+            mbar_init(bar_aempty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 128);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_acc = tmem_base;
+    const uint32_t tmem_a = tmem_base + ACC_COLS;
+    const int total_tiles = p.n_tiles * p.m_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
+                    const uint32_t dst = smem_base + s * C::STAGE_BYTES;
+                    mbar_expect_tx(bar_full + 8 * s, C::STAGE_BYTES);
+                    tma_load_2d(dst, &tm_act, kb * BK, m0, bar_full + 8 * s);
+                    if (!TS) tma_load_2d(dst + B_TILE_BYTES, &tm_w, kb * BK, n0, bar_full + 8 * s);
+                }
+            }
+            if (!ok) {
+                // aborting: let the copies already issued land before the CTA exits
+                for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
+                    const uint32_t j = it - back, s = j % STAGES, ph = (j / STAGES) & 1;
+                    const unsigned long long t0 = clock64();
+                    while (!mbar_try(bar_full + 8 * s, ph) && clock64() - t0 < kWaitClocks) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_i8(TILE_N, TILE_M);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+                if (!(ok = mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag, 2, tcount))) break;
+                tc_fence_after();
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
+                    if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_flag, 3, it))) break;
+                    if (TS && !(ok = mbar_wait(bar_afull + 8 * sa, pha, abort_flag, 4, it))) break;
+                    tc_fence_after();
+                    const uint32_t b_addr = smem_base + s * C::STAGE_BYTES;
+                    const uint64_t b_desc = smem_desc_sw128(b_addr);
+                    const uint64_t a_desc = smem_desc_sw128(b_addr + B_TILE_BYTES);
+#pragma unroll
+                    for (int j = 0; j < BK / UMMA_K; ++j) {
+                        const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
+                        // advancing 32 channels = 32 bytes inside the swizzle row = +2 in the address field
+                        if (TS) mma_ts(tmem_acc, tmem_a + sa * A_COLS + j * (UMMA_K / 4), b_desc + 2 * j, idesc, accum);
+                        else mma_ss(tmem_acc, a_desc + 2 * j, b_desc + 2 * j, idesc, accum);
+                    }
+                    tc_commit(bar_empty + 8 * s);
+                    if (TS) tc_commit(bar_aempty + 8 * sa);
+                }
+                if (ok) tc_commit(bar_acc_full);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------- weight expanders (TS)
+        if (TS) {
+            const int quad = warp & 3;            // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+            const int row = quad * 32 + lane;     // weight row inside the tile = TMEM lane
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int nt = tile % p.n_tiles;
+                const uint8_t* tile_base = p.wt + (size_t)nt * p.kblocks * 4096;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
+                    const uint4* src = reinterpret_cast<const uint4*>(tile_base + (size_t)kb * 4096);
+                    const uint4 lo = __ldg(src + row), hi = __ldg(src + 128 + row);
+                    uint32_t v[32];
+                    expand_word(lo.x, v + 0);
+                    expand_word(lo.y, v + 4);
+                    expand_word(lo.z, v + 8);
+                    expand_word(lo.w, v + 12);
+                    expand_word(hi.x, v + 16);
+                    expand_word(hi.y, v + 20);
+                    expand_word(hi.z, v + 24);
+                    expand_word(hi.w, v + 28);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1, abort_flag, 5, it));
+                    if (!ok) break;
+                    tc_fence_after();
+                    tmem_st32(tmem_a + ((uint32_t)(quad * 32) << 16) + sa * A_COLS, v);
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    tc_fence_before();
+                    mbar_arrive(bar_afull + 8 * sa);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------- epilogue
+        const int quad = warp & 3;
+        const float alpha = *p.alpha;
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+            const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, tcount & 1, abort_flag, 6, tcount));
+            if (!ok) break;
+            tc_fence_after();
+            const int n = n0 + quad * 32 + lane;
+            const bool n_ok = n < p.N;
+#pragma unroll 1
+            for (int c0 = 0; c0 < TILE_M; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + c0, r);
+                // lane j fetches the rescale factor of token m0+c0+j (Eq. 2/3/7 prefactors); shared by shuffle
+                const int mj = m0 + c0 + lane;
+                const float sv = mj < p.M ? __ldg(p.scale + mj) * alpha : 0.f;
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float sc = __shfl_sync(0xffffffffu, sv, j);
+                    const int m = m0 + c0 + j;
+                    if (n_ok && m < p.M) {
+                        const size_t o = (size_t)m * p.N + n;
+                        p.Y[o] = (float)(int)r[j] * sc;
+                        if (p.acc) p.acc[o] = (int)r[j];
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar_acc_empty);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// int8 matrix [rows, cols] row-major (row pitch = pitch bytes), box = 128 bytes x box_rows, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    }
+    return n;
+}
+
+template <bool TS>
+bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
+                         int32_t* acc, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        A48_CUDA_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<TS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          Cfg<TS>::SMEM_BYTES));
+        attr_set = true;
+    }
+    CUtensorMap tm_act, tm_w;
+    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TILE_M)) return BITNET_A48_ERR_CUDA;
+    if (TS) {
+        tm_w = tm_act;  // unused
+    } else if (!make_map(&tm_w, w->i8, (uint64_t)w->Np, (uint64_t)w->Kp, (uint64_t)w->Kp, TILE_N)) {
+        return BITNET_A48_ERR_CUDA;
+    }
+    GemmParams p;
+    p.wt = w->gemm;
+    p.scale = scale;
+    p.alpha = w->alpha_dev;
+    p.Y = Y;
+    p.acc = acc;
+    p.M = M;
+    p.N = w->N;
+    p.K = w->K;
+    p.kblocks = w->Kp / BK;
+    p.n_tiles = (w->N + TILE_N - 1) / TILE_N;
+    p.m_tiles = (M + TILE_M - 1) / TILE_M;
+    const int total = p.n_tiles * p.m_tiles;
+    const int grid = total < sm_count() ? total : sm_count();
+    gemm_tcgen05_kernel<TS><<<grid, NUM_THREADS, Cfg<TS>::SMEM_BYTES, st>>>(tm_act, tm_w, p);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+}  // namespace
+
+bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss) {
+    if (w->K % 16 != 0 || M < 1) return false;  // TMA needs a 16-byte row pitch
+    return ss ? w->i8 != nullptr : w->gemm != nullptr;
+}
+
+bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
+                                          float* Y, int32_t* acc, bool ss, cudaStream_t st) {
+    return ss ? launch<false>(w, codes, scale, M, Y, acc, st) : launch<true>(w, codes, scale, M, Y, acc, st);
+}
+
 bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]) {
-    for (int i = 0; i < 4; ++i) words_host[i] = 0;
+    A48_CUDA_TRY(cudaDeviceSynchronize());
+    A48_CUDA_TRY(cudaMemcpyFromSymbol(words_host, g_status, sizeof(unsigned int) * 4));
+    const unsigned int zero[4] = {0, 0, 0, 0};
+    A48_CUDA_TRY(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
     return BITNET_A48_OK;
 }

@@ -32,6 +32,7 @@ struct bitnet_a48_weight {
     uint8_t* gemm;         // tile-major layout, Np*Kp/4 bytes (or NULL)
     uint8_t* decode;       // fragment-major layout (or NULL)
     uint8_t* sparse;       // channel-major layout (or NULL)
+    int8_t* i8;            // int8 codes [Np][Kp], zero padded (or NULL)
     size_t decode_bytes, sparse_bytes;
 };
 
@@ -62,9 +63,10 @@ bitnet_a48_status a48_launch_linear_simple(const bitnet_a48_weight* w, const int
                                            int M, float* Y, int32_t* acc, cudaStream_t st);
 
 // ---- gemm_tcgen05.cu
-bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M);
+// ss = true: both operands from shared memory (needs the int8 copy); false: weights expanded into tensor memory.
+bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss);
 bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
-                                          float* Y, int32_t* acc, cudaStream_t st);
+                                          float* Y, int32_t* acc, bool ss, cudaStream_t st);
 bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]);
 
 // ---- decode.cu

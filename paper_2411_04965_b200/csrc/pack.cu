@@ -108,6 +108,15 @@ __global__ void unpack_layout_kernel(const uint32_t* __restrict__ src, int N, in
     }
 }
 
+// int8 codes [Np][Kp], zero outside [N][K]
+__global__ void expand_i8_kernel(const uint8_t* __restrict__ l0, int N, int K, int K4, int Np, int Kp,
+                                 int8_t* __restrict__ dst) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)Np * Kp) return;
+    int n = (int)(idx / Kp), k = (int)(idx % Kp);
+    dst[idx] = (n < N && k < K) ? (int8_t)a48_l0_code(l0, K4, n, k) : (int8_t)0;
+}
+
 template <class Layout>
 void run_relayout(const bitnet_a48_weight* w, Layout lay, uint8_t* dst, size_t bytes, cudaStream_t st) {
     size_t nwords = bytes / 4;
@@ -137,6 +146,10 @@ bitnet_a48_status a48_launch_pack(bitnet_a48_weight* w, const float* W_dev, floa
     if (w->gemm) run_relayout(w, GemmLayout{w->Kp}, w->gemm, (size_t)w->Np * w->Kp / 4, st);
     if (w->decode) run_relayout(w, DecodeLayout{w->Kp}, w->decode, w->decode_bytes, st);
     if (w->sparse) run_relayout(w, SparseLayout{w->Np}, w->sparse, w->sparse_bytes, st);
+    if (w->i8) {
+        size_t n8 = (size_t)w->Np * w->Kp;
+        expand_i8_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(w->l0, w->N, w->K, w->K4, w->Np, w->Kp, w->i8);
+    }
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }

@@ -1,0 +1,89 @@
+"""tcgen05 prefill kernel (both operand variants) against the oracle: int32 accumulators bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from parity import max_rel_err
+from paper_2411_04965_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-5
+# (M, N, K): one tile; several k-blocks; ragged M and N tails; K a multiple of 64 but not 128 (like 8640);
+# K a multiple of 16 only; several tiles per CTA wave
+SHAPES = [(256, 128, 128), (256, 128, 1024), (300, 200, 384), (70, 130, 320), (513, 257, 144), (1, 128, 256),
+          (1100, 1536, 1536)]
+
+
+def _algos(a48):
+    return {"tmem": a48.ALGO_GEMM_TCGEN05, "smem_i8": a48.ALGO_GEMM_TCGEN05_I8}
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("variant", ["tmem", "smem_i8"])
+@pytest.mark.parametrize("kind", ["int4", "topk"])
+def test_gemm_tcgen05_matches_oracle(a48, oracle, cuda_dev, M, N, K, variant, kind):
+    W = synth.latent_weights(N, K, seed=N + K)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_ALL | a48.LAYOUT_I8)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=M)
+        codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+        c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS, nthreads=8)
+        act = a48.ACT_INT4
+    else:
+        x = synth.student_t3(M, K, seed=M)
+        codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+        c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS, nthreads=8)
+        act = a48.ACT_TOPK_INT8
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    y, acc = a48.linear(w, codes, scale, act, _algos(a48)[variant], want_acc=True)
+    torch.cuda.synchronize()
+    assert a48.kernel_status() == [0, 0, 0, 0]
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+
+
+def test_gemm_extreme_codes_do_not_overflow(a48, oracle, cuda_dev):
+    # all codes +-127 against all-(+1) weights: |acc| = 127*K, the largest accumulator this path can see
+    M, N, K = 256, 128, 11008
+    W = torch.full((N, K), 0.05)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_GEMM)
+    codes = torch.full((M, K), 127, dtype=torch.int8)
+    codes[1::2] = -127
+    scale = torch.ones(M)
+    y, acc = a48.linear(w, codes.to(cuda_dev), scale.to(cuda_dev), a48.ACT_TOPK_INT8, a48.ALGO_GEMM_TCGEN05,
+                        want_acc=True)
+    acc = acc.cpu()
+    assert (acc[0::2] == 127 * K).all() and (acc[1::2] == -127 * K).all()
+
+
+def test_gemm_full_size_sampled(a48, oracle, cuda_dev):
+    # The benchmark's launch configuration: 7B gate projection (4096 -> 11008) over 16384 tokens.  The oracle
+    # recomputes a sample: 24 whole token rows and 24 whole output columns.
+    M, N, K = 16384, 11008, 4096
+    W = synth.ternary_latents(N, K, seed=4, device=cuda_dev)
+    w = a48.pack_ternary(W, EPS, a48.LAYOUT_GEMM)
+    t_dev, alpha = a48.weight_unpack(w)
+    x = synth.gaussian_outlier_activations(M, K, seed=40, device=cuda_dev)
+    codes, scale = a48.quant_int4(x, EPS)
+    y, acc = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05, want_acc=True)
+    torch.cuda.synchronize()
+    assert a48.kernel_status() == [0, 0, 0, 0]
+    g = torch.Generator().manual_seed(0)
+    rows = torch.cat([torch.tensor([0, 255, 256, M - 1]), torch.randint(0, M, (20,), generator=g)]).to(cuda_dev)
+    cols = torch.cat([torch.tensor([0, 127, 128, N - 1]), torch.randint(0, N, (20,), generator=g)]).to(cuda_dev)
+    t_ref, a_ref = oracle.ternarise(W.cpu().numpy(), EPS)
+    assert np.array_equal(t_dev.cpu().numpy(), t_ref) and alpha == np.float32(a_ref)
+    x_rows = x[rows].cpu().numpy()
+    q_ref, d_ref = oracle.quant_int4(x_rows, EPS, nthreads=8)
+    assert np.array_equal(codes[rows].cpu().numpy(), q_ref)
+    acc_ref, y_ref = oracle.linear(q_ref, d_ref, t_ref, a_ref, nthreads=8)
+    assert np.array_equal(acc[rows].cpu().numpy().astype(np.int64), acc_ref)
+    assert max_rel_err(y[rows].cpu().numpy(), y_ref) <= 1e-5
+    # whole columns: every token against 24 weight rows (codes already checked on the sampled rows; here the
+    # GPU codes feed the oracle contraction, which checks the contraction at every token)
+    codes_h, scale_h = codes.cpu().numpy(), scale.cpu().numpy().astype(np.float64)
+    acc_c, _ = oracle.linear(codes_h, scale_h, t_ref[cols.cpu().numpy()], a_ref, nthreads=8, want_y=False)
+    assert np.array_equal(acc[:, cols].cpu().numpy().astype(np.int64), acc_c)
