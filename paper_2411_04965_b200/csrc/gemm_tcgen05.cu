@@ -1,25 +1,31 @@
 // Prefill BitLinear contraction (Eq. 1 / Eq. 6) on the 5th-generation tensor cores:
 // tcgen05.mma kind::i8 (s8 x s8 -> s32) with the accumulators in tensor memory.
 //
-// Orientation.  The MMA computes D[128 x 256] = A[128 x K] * B[K x 256] with
+// Orientation.  The MMA computes D[128 x 192] = A[128 x K] * B[K x 192] with
 //   A = a tile of 128 weight rows (output features n), expanded to int8 codes,
-//   B = a tile of 256 tokens of activation codes (row-major [M,K] is exactly the
+//   B = a tile of 192 tokens of activation codes (row-major [M,K] is exactly the
 //       K-major operand layout the MMA wants),
 // so the accumulator holds Y^T: TMEM lane = output feature, TMEM column = token.
 // The epilogue thread that owns lane n writes Y[m, n] for consecutive m, which
 // makes every warp store a contiguous 128-byte run of one output row.
 //
 // Two variants share the pipeline:
-//   TS (default): the 2-bit weights are read straight from global memory (L2
-//       resident) by four expander warps, widened to int8 in registers with a
+//   TS (default): the 2-bit weights are staged into shared memory by a bulk
+//       copy on the same pipeline stage as the activation tile (4 KB per 128
+//       channels), widened to int8 in registers by four expander warps with a
 //       byte-permute lookup, and written into tensor memory with tcgen05.st; the
-//       MMA takes A from tensor memory.  The weights never occupy shared memory,
-//       whose bandwidth is left to the activation operand.
+//       MMA takes A from tensor memory.  Only the packed form touches shared
+//       memory, whose bandwidth is left to the activation operand.
 //   SS: both operands come from shared memory via TMA; A is a pre-expanded int8
 //       copy of the weights (BITNET_A48_LAYOUT_I8).  Comparison / bring-up variant.
 //
+// Tensor memory (512 columns) holds two 192-column accumulators, so the epilogue
+// of one tile drains while the MMAs of the next tile run, and four 32-column
+// stages of the expanded weight operand.
+//
 // Warp roles (one persistent CTA per SM): warp 0 TMA producer, warp 1 MMA issuer
-// and TMEM owner, warps 2-5 weight expanders (TS only), warps 6-9 epilogue.
+// and TMEM owner, warps 2-9 weight expanders (TS only; two groups of four that
+// alternate over the 128-channel blocks), warps 10-13 epilogue.
 // Every mbarrier wait is bounded; a wait that gives up records a status word and
 // the CTA drains and exits without touching tensor memory again.
 #include <cuda.h>
@@ -29,22 +35,28 @@
 namespace {
 
 constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
-constexpr int TILE_M = 256;  // tokens per tile       (MMA N)
+constexpr int TILE_M = 192;  // tokens per tile       (MMA N)
 constexpr int BK = 128;      // channels per pipeline stage = one 128-byte swizzle row of int8
 constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
-constexpr int A_STAGES = 8;  // tensor-memory stages of the expanded weight operand (32 columns each)
+constexpr int A_STAGES = 4;  // tensor-memory stages of the expanded weight operand (32 columns each)
 constexpr int A_COLS = BK / 4;
 constexpr int ACC_COLS = TILE_M;
+constexpr int ACC_BUFS = 2;
 constexpr int TMEM_COLS = 512;
+static_assert(ACC_BUFS * ACC_COLS + A_STAGES * A_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int B_TILE_BYTES = TILE_M * BK;
 constexpr int A_TILE_BYTES = TILE_N * BK;
-constexpr int NUM_THREADS = 320;
+constexpr int W_PACKED_BYTES = TILE_N * BK / 4;  // one tile of 2-bit codes
+constexpr int NUM_THREADS = 448;
+constexpr int EXPAND_GROUPS = 2;
 constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
 
 template <bool TS>
 struct Cfg {
-    static constexpr int STAGES = TS ? 6 : 4;
-    static constexpr int STAGE_BYTES = B_TILE_BYTES + (TS ? 0 : A_TILE_BYTES);
+    static constexpr int STAGES = TS ? 7 : 5;
+    static constexpr int STAGE_BYTES = B_TILE_BYTES + (TS ? W_PACKED_BYTES : A_TILE_BYTES);
+    // a stage is released by the MMA commit and, for TS, by one lane of each expander warp
+    static constexpr int EMPTY_ARRIVALS = TS ? 5 : 1;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 1024 /*barriers*/;
 };
 
@@ -75,9 +87,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns false when the CTA is aborting or the wait ran out of
 // time; in the latter case the first such event is recorded in g_status.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id,
-                                       uint32_t iter) {
-    if (mbar_try(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id,
+                                            uint32_t iter) {
     const unsigned long long t0 = clock64();
     uint32_t spins = 0;
     while (true) {
@@ -97,11 +108,48 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile u
     }
 }
 
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id,
+                                          uint32_t iter) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, id, iter);
+}
+
+// Non-blocking look at a barrier phase (used to start the next wait early).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// True in exactly one lane of a converged warp (the same lane on every call).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
+}
+
+// Untiled bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -213,21 +261,23 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_afull = bar_empty + 8 * STAGES, bar_aempty = bar_afull + 8 * A_STAGES;
-    const uint32_t bar_acc_full = bar_aempty + 8 * A_STAGES, bar_acc_empty = bar_acc_full + 8;
+    const uint32_t bar_acc_full = bar_aempty + 8 * A_STAGES, bar_acc_empty = bar_acc_full + 8 * ACC_BUFS;
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, C::EMPTY_ARRIVALS);
         }
         for (int s = 0; s < A_STAGES; ++s) {
             mbar_init(bar_afull + 8 * s, 128);
             mbar_init(bar_aempty + 8 * s, 1);
         }
-        mbar_init(bar_acc_full, 1);
-        mbar_init(bar_acc_empty, 128);
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 128);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -242,7 +292,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_acc = tmem_base;
-    const uint32_t tmem_a = tmem_base + ACC_COLS;
+    const uint32_t tmem_a = tmem_base + ACC_BUFS * ACC_COLS;
     const int total_tiles = p.n_tiles * p.m_tiles;
 
     if (warp == 0) {
@@ -252,13 +302,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
+                const uint8_t* wtile = p.wt + (size_t)(tile % p.n_tiles) * p.kblocks * W_PACKED_BYTES;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
                     const uint32_t dst = smem_base + s * C::STAGE_BYTES;
                     mbar_expect_tx(bar_full + 8 * s, C::STAGE_BYTES);
                     tma_load_2d(dst, &tm_act, kb * BK, m0, bar_full + 8 * s);
-                    if (!TS) tma_load_2d(dst + B_TILE_BYTES, &tm_w, kb * BK, n0, bar_full + 8 * s);
+                    if (TS) bulk_load(dst + B_TILE_BYTES, wtile + (size_t)kb * W_PACKED_BYTES, W_PACKED_BYTES, bar_full + 8 * s);
+                    else tma_load_2d(dst + B_TILE_BYTES, &tm_w, kb * BK, n0, bar_full + 8 * s);
                 }
             }
             if (!ok) {
@@ -273,19 +325,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_i8(TILE_N, TILE_M);
-            uint32_t it = 0, tcount = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-                if (!(ok = mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag, 2, tcount))) break;
+        // The whole warp walks the loop in lockstep so that indices and descriptors stay
+        // warp-uniform; one elected lane issues the MMAs and the commits.  With TS the
+        // issuer waits only for the expanded weights: the expanders arrive on that barrier
+        // after they have themselves seen the stage's TMA barrier complete.
+        constexpr uint32_t idesc = idesc_i8(TILE_N, TILE_M);
+        uint32_t it = 0, tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+            const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
+            const uint32_t d_tmem = tmem_acc + ab * ACC_COLS;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8 * ab, pab ^ 1, abort_flag, 2, tcount));
+            if (!ok) break;
+            tc_fence_after();
+            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
+                const uint32_t bar_in = TS ? bar_afull + 8 * sa : bar_full + 8 * s;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_in, TS ? pha : ph, abort_flag, TS ? 4 : 3, it));
+                if (!ok) break;
                 tc_fence_after();
-                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                    const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
-                    if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_flag, 3, it))) break;
-                    if (TS && !(ok = mbar_wait(bar_afull + 8 * sa, pha, abort_flag, 4, it))) break;
-                    tc_fence_after();
+                if (elect_one()) {
                     const uint32_t b_addr = smem_base + s * C::STAGE_BYTES;
                     const uint64_t b_desc = smem_desc_sw128(b_addr);
                     const uint64_t a_desc = smem_desc_sw128(b_addr + B_TILE_BYTES);
@@ -293,29 +353,34 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                     for (int j = 0; j < BK / UMMA_K; ++j) {
                         const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
                         // advancing 32 channels = 32 bytes inside the swizzle row = +2 in the address field
-                        if (TS) mma_ts(tmem_acc, tmem_a + sa * A_COLS + j * (UMMA_K / 4), b_desc + 2 * j, idesc, accum);
-                        else mma_ss(tmem_acc, a_desc + 2 * j, b_desc + 2 * j, idesc, accum);
+                        if (TS) mma_ts(d_tmem, tmem_a + sa * A_COLS + j * (UMMA_K / 4), b_desc + 2 * j, idesc, accum);
+                        else mma_ss(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, accum);
                     }
                     tc_commit(bar_empty + 8 * s);
                     if (TS) tc_commit(bar_aempty + 8 * sa);
                 }
-                if (ok) tc_commit(bar_acc_full);
+                __syncwarp();
             }
+            if (ok && elect_one()) tc_commit(bar_acc_full + 8 * ab);
+            __syncwarp();
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + 4 * EXPAND_GROUPS) {
         // ------------------------------------------------------------- weight expanders (TS)
         if (TS) {
             const int quad = warp & 3;            // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
             const int row = quad * 32 + lane;     // weight row inside the tile = TMEM lane
+            const uint32_t group = (uint32_t)(warp - 2) >> 2;  // this group takes the blocks with it % groups == group
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int nt = tile % p.n_tiles;
-                const uint8_t* tile_base = p.wt + (size_t)nt * p.kblocks * 4096;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    if (it % EXPAND_GROUPS != group) continue;
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
-                    const uint4* src = reinterpret_cast<const uint4*>(tile_base + (size_t)kb * 4096);
-                    const uint4 lo = __ldg(src + row), hi = __ldg(src + 128 + row);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag, 7, it));
+                    if (!ok) break;
+                    const uint4* src = reinterpret_cast<const uint4*>(smem + s * C::STAGE_BYTES + B_TILE_BYTES);
+                    const uint4 lo = src[row], hi = src[128 + row];
                     uint32_t v[32];
                     expand_word(lo.x, v + 0);
                     expand_word(lo.y, v + 4);
@@ -325,6 +390,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                     expand_word(hi.y, v + 20);
                     expand_word(hi.z, v + 24);
                     expand_word(hi.w, v + 28);
+                    __syncwarp();  // every lane has consumed its packed words: the stage's weight bytes are free
+                    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1, abort_flag, 5, it));
                     if (!ok) break;
                     tc_fence_after();
@@ -343,7 +410,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
             const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, tcount & 1, abort_flag, 6, tcount));
+            const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, pab, abort_flag, 6, tcount));
             if (!ok) break;
             tc_fence_after();
             const int n = n0 + quad * 32 + lane;
@@ -351,7 +419,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 #pragma unroll 1
             for (int c0 = 0; c0 < TILE_M; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + c0, r);
+                tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + ab * ACC_COLS + c0, r);
                 // lane j fetches the rescale factor of token m0+c0+j (Eq. 2/3/7 prefactors); shared by shuffle
                 const int mj = m0 + c0 + lane;
                 const float sv = mj < p.M ? __ldg(p.scale + mj) * alpha : 0.f;
@@ -368,7 +436,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                 }
             }
             tc_fence_before();
-            mbar_arrive(bar_acc_empty);
+            mbar_arrive(bar_acc_empty + 8 * ab);
         }
     }
     tc_fence_before();

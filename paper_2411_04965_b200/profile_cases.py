@@ -1,0 +1,100 @@
+"""Small single-kernel cases for profiler captures (ncu) and quick timing.
+
+    python -m paper_2411_04965_b200.profile_cases gemm   --M 8192 --N 11008 --K 4096 --kind int4 --reps 3
+    python -m paper_2411_04965_b200.profile_cases quant  --M 16384 --K 4096 --kind topk --reps 3
+    python -m paper_2411_04965_b200.profile_cases decode --M 1 --N 11008 --K 4096 --kind topk --copies 32 --reps 3
+
+Each case builds seeded synthetic inputs (the same recipes the benchmark uses),
+runs the kernel `reps` times after one warm-up call and prints the mean time
+from CUDA events on the launching stream.  `decode` cycles over `copies`
+distinct weight matrices so that the weight bytes come from HBM, not L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as a48
+from . import build as a48_build
+from . import synth
+
+EPS = 1e-5
+
+
+def _time(fn, reps, stream):
+    fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def _acts(kind, M, K, dev, k_frac=0.5):
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=11, device=dev)
+        codes, scale = a48.quant_int4(x, EPS)
+        return x, codes, scale, a48.ACT_INT4
+    x = synth.student_t3(M, K, seed=12, device=dev)
+    codes, scale, _ = a48.topk_quant_int8(x, max(1, int(K * k_frac)), EPS)
+    return x, codes, scale, a48.ACT_TOPK_INT8
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["gemm", "quant", "decode"])
+    ap.add_argument("--M", type=int, default=8192)
+    ap.add_argument("--N", type=int, default=11008)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--kind", choices=["int4", "topk"], default="int4")
+    ap.add_argument("--algo", type=int, default=a48.ALGO_AUTO)
+    ap.add_argument("--copies", type=int, default=32)
+    ap.add_argument("--reps", type=int, default=3)
+    args = ap.parse_args()
+    a48_build.build()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.current_stream()
+    M, N, K = args.M, args.N, args.K
+    out = {"case": args.case, "M": M, "N": N, "K": K, "kind": args.kind}
+    if args.case == "quant":
+        x = (synth.gaussian_outlier_activations if args.kind == "int4" else synth.student_t3)(M, K, 11, device=dev)
+        codes = torch.empty(M, K, dtype=torch.int8, device=dev)
+        scale = torch.empty(M, dtype=torch.float32, device=dev)
+        if args.kind == "int4":
+            ms = _time(lambda: a48.quant_int4(x, EPS, codes, scale), args.reps, stream)
+        else:
+            ms = _time(lambda: a48.topk_quant_int8(x, K // 2, EPS, codes, scale), args.reps, stream)
+        out.update(ms=ms, gbs=(5.0 * M * K + 4 * M) / ms / 1e6)
+    elif args.case == "gemm":
+        algo = args.algo or a48.ALGO_GEMM_TCGEN05
+        layouts = a48.LAYOUT_GEMM | (a48.LAYOUT_I8 if algo == a48.ALGO_GEMM_TCGEN05_I8 else 0)
+        w = a48.pack_ternary(synth.ternary_latents(N, K, seed=4, device=dev), EPS, layouts)
+        _, codes, scale, act = _acts(args.kind, M, K, dev)
+        y = torch.empty(M, N, dtype=torch.float32, device=dev)
+        ms = _time(lambda: a48.linear(w, codes, scale, act, algo, Y=y), args.reps, stream)
+        out.update(ms=ms, tops=2.0 * M * N * K / ms / 1e9)
+    else:
+        ws = [a48.pack_ternary(synth.ternary_latents(N, K, seed=100 + i, device=dev), EPS,
+                               a48.LAYOUT_DECODE | a48.LAYOUT_SPARSE) for i in range(args.copies)]
+        _, codes, scale, act = _acts(args.kind, M, K, dev)
+        y = torch.empty(M, N, dtype=torch.float32, device=dev)
+        need = a48.linear_workspace_bytes(ws[0], M)
+        wsp = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+
+        def run():
+            for w in ws:
+                a48.linear(w, codes, scale, act, args.algo, Y=y, workspace=wsp)
+
+        ms = _time(run, args.reps, stream) / len(ws)
+        out.update(ms=ms, dense_gbs=ws[0].packed_bytes / ms / 1e6)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
