@@ -67,7 +67,7 @@ bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, floa
     w->K = K;
     w->K4 = (K + 3) / 4;
     w->Np = a48_round_up(N, 256);
-    w->Kp = a48_round_up(K, 128);
+    w->Kp = a48_round_up(K, 256);
     w->flags = layout_flags;
     w->decode_bytes = (size_t)w->Np * w->Kp / 4;
     w->sparse_bytes = (size_t)K * w->Np / 4;

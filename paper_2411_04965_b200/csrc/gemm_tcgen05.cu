@@ -11,21 +11,31 @@
 //
 // Two variants share the pipeline:
 //   TS (default): the 2-bit weights are staged into shared memory by a bulk
-//       copy on the same pipeline stage as the activation tile (4 KB per 128
-//       channels), widened to int8 in registers by four expander warps with a
+//       copy on the same pipeline stage as the activation tile (8 KB per 256
+//       channels), widened to int8 in registers by eight expander warps with a
 //       byte-permute lookup, and written into tensor memory with tcgen05.st; the
 //       MMA takes A from tensor memory.  Only the packed form touches shared
 //       memory, whose bandwidth is left to the activation operand.
 //   SS: both operands come from shared memory via TMA; A is a pre-expanded int8
 //       copy of the weights (BITNET_A48_LAYOUT_I8).  Comparison / bring-up variant.
 //
-// Tensor memory (512 columns) holds two 192-column accumulators, so the epilogue
-// of one tile drains while the MMAs of the next tile run, and four 32-column
-// stages of the expanded weight operand.
+// A pipeline stage ("unit") covers 256 channels for TS (two 128-byte swizzle
+// rows of the activation tile and 8 KB of packed weights): one thread issues all
+// MMAs, and what it pays per stage (one barrier wait, one commit, the loop) is
+// spread over eight MMAs instead of four.  Tensor memory (512 columns) holds two
+// 192-column accumulators, so the epilogue of one tile drains while the MMAs of
+// the next tile run, and two 64-column slots of the expanded weight operand.
+//
+// Barriers per stage s: full[s] (TMA bytes landed), empty[s] (the MMAs that read
+// the stage have completed - one tcgen05.commit - and the expanders have read
+// its packed weights).  The same commit frees the tensor-memory slot the stage's
+// expanded weights sat in, so the expanders wait on empty[] of the stage two
+// units back instead of on a barrier of their own.  afull[g]: slot g written.
 //
 // Warp roles (one persistent CTA per SM): warp 0 TMA producer, warp 1 MMA issuer
-// and TMEM owner, warps 2-9 weight expanders (TS only; two groups of four that
-// alternate over the 128-channel blocks), warps 10-13 epilogue.
+// and TMEM owner, warps 2-9 weight expanders (TS only; two groups of four, group
+// g takes every second unit and owns slot g), warps 10-17 epilogue (two per
+// tensor-memory lane quadrant, each draining half of the accumulator columns).
 // Every mbarrier wait is bounded; a wait that gives up records a status word and
 // the CTA drains and exits without touching tensor memory again.
 #include <cuda.h>
@@ -36,28 +46,35 @@ namespace {
 
 constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
 constexpr int TILE_M = 192;  // tokens per tile       (MMA N)
-constexpr int BK = 128;      // channels per pipeline stage = one 128-byte swizzle row of int8
+constexpr int BK = 128;      // channels per 128-byte swizzle row of int8
 constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
-constexpr int A_STAGES = 4;  // tensor-memory stages of the expanded weight operand (32 columns each)
-constexpr int A_COLS = BK / 4;
+constexpr int A_SLOTS = 2;   // tensor-memory slots of the expanded weight operand
 constexpr int ACC_COLS = TILE_M;
 constexpr int ACC_BUFS = 2;
 constexpr int TMEM_COLS = 512;
-static_assert(ACC_BUFS * ACC_COLS + A_STAGES * A_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int B_TILE_BYTES = TILE_M * BK;
 constexpr int A_TILE_BYTES = TILE_N * BK;
-constexpr int W_PACKED_BYTES = TILE_N * BK / 4;  // one tile of 2-bit codes
-constexpr int NUM_THREADS = 448;
+constexpr int W_PACKED_BYTES = TILE_N * BK / 4;  // 128 rows x 128 channels of 2-bit codes
 constexpr int EXPAND_GROUPS = 2;
+constexpr int EPI_SPLIT = 2;  // epilogue warps per lane quadrant
+constexpr int EPI_COLS = TILE_M / EPI_SPLIT;
+static_assert(EPI_COLS % 32 == 0, "the epilogue drains 32 columns at a time");
+constexpr int NUM_THREADS = 32 * (2 + 4 * EXPAND_GROUPS + 4 * EPI_SPLIT);
+static_assert(A_SLOTS == EXPAND_GROUPS, "expander group g owns slot g");
 constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
 
 template <bool TS>
 struct Cfg {
-    static constexpr int STAGES = TS ? 7 : 5;
-    static constexpr int STAGE_BYTES = B_TILE_BYTES + (TS ? W_PACKED_BYTES : A_TILE_BYTES);
-    // a stage is released by the MMA commit and, for TS, by one lane of each expander warp
+    static constexpr int KBU = TS ? 2 : 1;  // 128-channel blocks per pipeline stage
+    static constexpr int STAGES = TS ? 4 : 5;
+    static constexpr int STAGE_BYTES = KBU * (B_TILE_BYTES + (TS ? W_PACKED_BYTES : A_TILE_BYTES));
+    static constexpr int A_SLOT_COLS = KBU * BK / 4;
+    // a stage is released by the MMA commit and, for TS, by one lane of each expander warp of one group
     static constexpr int EMPTY_ARRIVALS = TS ? 5 : 1;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 1024 /*barriers*/;
+    static_assert(ACC_BUFS * ACC_COLS + (TS ? A_SLOTS * A_SLOT_COLS : 0) <= TMEM_COLS, "tensor memory budget");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(STAGES > A_SLOTS, "the stage two units back must still be distinct");
 };
 
 __device__ unsigned int g_status[4];
@@ -114,19 +131,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_slow(bar, parity, abort_flag, id, iter);
 }
 
-// Non-blocking look at a barrier phase (used to start the next wait early).
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
 // True in exactly one lane of a converged warp (the same lane on every call).
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred = 0;
@@ -166,6 +170,15 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] += A[tmem] * B[smem desc given as two words]
+__device__ __forceinline__ void mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 d;\n\tsetp.eq.b32 p, 0, 0;\n\tmov.b64 d, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], d, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
@@ -251,17 +264,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                         const GemmParams p) {
     using C = Cfg<TS>;
-    constexpr int STAGES = C::STAGES;
+    constexpr int STAGES = C::STAGES, KBU = C::KBU;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ctrl = smem + STAGES * C::STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] aempty[A] acc_full acc_empty
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] acc_full[2] acc_empty[2]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 512);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 516);
 
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
-    const uint32_t bar_afull = bar_empty + 8 * STAGES, bar_aempty = bar_afull + 8 * A_STAGES;
-    const uint32_t bar_acc_full = bar_aempty + 8 * A_STAGES, bar_acc_empty = bar_acc_full + 8 * ACC_BUFS;
+    const uint32_t bar_afull = bar_empty + 8 * STAGES;
+    const uint32_t bar_acc_full = bar_afull + 8 * A_SLOTS, bar_acc_empty = bar_acc_full + 8 * ACC_BUFS;
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -270,13 +283,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, C::EMPTY_ARRIVALS);
         }
-        for (int s = 0; s < A_STAGES; ++s) {
-            mbar_init(bar_afull + 8 * s, 128);
-            mbar_init(bar_aempty + 8 * s, 1);
-        }
+        for (int s = 0; s < A_SLOTS; ++s) mbar_init(bar_afull + 8 * s, 128);
         for (int b = 0; b < ACC_BUFS; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, 128);
+            mbar_init(bar_acc_empty + 8 * b, 128 * EPI_SPLIT);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -294,31 +304,39 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     const uint32_t tmem_acc = tmem_base;
     const uint32_t tmem_a = tmem_base + ACC_BUFS * ACC_COLS;
     const int total_tiles = p.n_tiles * p.m_tiles;
+    const int kunits = p.kblocks / KBU;  // the packed layouts pad K so that this is exact
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, ph = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
                 const uint8_t* wtile = p.wt + (size_t)(tile % p.n_tiles) * p.kblocks * W_PACKED_BYTES;
-                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int u = 0; u < kunits; ++u, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
-                    const uint32_t dst = smem_base + s * C::STAGE_BYTES;
-                    mbar_expect_tx(bar_full + 8 * s, C::STAGE_BYTES);
-                    tma_load_2d(dst, &tm_act, kb * BK, m0, bar_full + 8 * s);
-                    if (TS) bulk_load(dst + B_TILE_BYTES, wtile + (size_t)kb * W_PACKED_BYTES, W_PACKED_BYTES, bar_full + 8 * s);
-                    else tma_load_2d(dst + B_TILE_BYTES, &tm_w, kb * BK, n0, bar_full + 8 * s);
+                    const uint32_t dst = smem_base + s * C::STAGE_BYTES, bar = bar_full + 8 * s;
+                    mbar_expect_tx(bar, C::STAGE_BYTES);
+#pragma unroll
+                    for (int h = 0; h < KBU; ++h) tma_load_2d(dst + h * B_TILE_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
+                    if (TS) {
+                        bulk_load(dst + KBU * B_TILE_BYTES, wtile + (size_t)u * KBU * W_PACKED_BYTES, KBU * W_PACKED_BYTES,
+                                  bar);
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < KBU; ++h)
+                            tma_load_2d(dst + KBU * B_TILE_BYTES + h * A_TILE_BYTES, &tm_w, (u * KBU + h) * BK, n0, bar);
+                    }
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
             }
             if (!ok) {
                 // aborting: let the copies already issued land before the CTA exits
                 for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
-                    const uint32_t j = it - back, s = j % STAGES, ph = (j / STAGES) & 1;
+                    const uint32_t j = it - back, sj = j % STAGES, pj = (j / STAGES) & 1;
                     const unsigned long long t0 = clock64();
-                    while (!mbar_try(bar_full + 8 * s, ph) && clock64() - t0 < kWaitClocks) {
+                    while (!mbar_try(bar_full + 8 * sj, pj) && clock64() - t0 < kWaitClocks) {
                     }
                 }
             }
@@ -330,7 +348,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         // issuer waits only for the expanded weights: the expanders arrive on that barrier
         // after they have themselves seen the stage's TMA barrier complete.
         constexpr uint32_t idesc = idesc_i8(TILE_N, TILE_M);
+        const bool leader = elect_one();  // the same lane issues every MMA and commit
         uint32_t it = 0, tcount = 0;
+        uint32_t s = 0, ph = 0;  // stage ring position and phase, advanced without divisions
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
@@ -338,30 +358,39 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
             ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8 * ab, pab ^ 1, abort_flag, 2, tcount));
             if (!ok) break;
             tc_fence_after();
-            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
-                const uint32_t bar_in = TS ? bar_afull + 8 * sa : bar_full + 8 * s;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_in, TS ? pha : ph, abort_flag, TS ? 4 : 3, it));
+            for (int u = 0; u < kunits; ++u, ++it) {
+                const uint32_t slot = it % A_SLOTS, pslot = (it / A_SLOTS) & 1;
+                const uint32_t bar_in = TS ? bar_afull + 8 * slot : bar_full + 8 * s;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_in, TS ? pslot : ph, abort_flag, TS ? 4 : 3, it));
                 if (!ok) break;
                 tc_fence_after();
-                if (elect_one()) {
+                if (leader) {
                     const uint32_t b_addr = smem_base + s * C::STAGE_BYTES;
-                    const uint64_t b_desc = smem_desc_sw128(b_addr);
-                    const uint64_t a_desc = smem_desc_sw128(b_addr + B_TILE_BYTES);
 #pragma unroll
-                    for (int j = 0; j < BK / UMMA_K; ++j) {
-                        const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
+                    for (int h = 0; h < KBU; ++h) {
+                        const uint64_t b_desc = smem_desc_sw128(b_addr + h * B_TILE_BYTES);
                         // advancing 32 channels = 32 bytes inside the swizzle row = +2 in the address field
-                        if (TS) mma_ts(d_tmem, tmem_a + sa * A_COLS + j * (UMMA_K / 4), b_desc + 2 * j, idesc, accum);
-                        else mma_ss(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, accum);
+                        if (TS) {
+                            const uint32_t b_lo = (uint32_t)b_desc, b_hi = (uint32_t)(b_desc >> 32);
+                            const uint32_t a_t = tmem_a + slot * C::A_SLOT_COLS + h * (BK / 4);
+#pragma unroll
+                            for (int j = 0; j < BK / UMMA_K; ++j) {
+                                if (h == 0 && j == 0 && u == 0) mma_ts(d_tmem, a_t, b_desc, idesc, 0u);
+                                else mma_ts_acc(d_tmem, a_t + j * (UMMA_K / 4), b_lo + 2 * j, b_hi, idesc);
+                            }
+                        } else {
+                            const uint64_t a_desc = smem_desc_sw128(b_addr + KBU * B_TILE_BYTES + h * A_TILE_BYTES);
+#pragma unroll
+                            for (int j = 0; j < BK / UMMA_K; ++j)
+                                mma_ss(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (u > 0 || h > 0 || j > 0) ? 1u : 0u);
+                        }
                     }
                     tc_commit(bar_empty + 8 * s);
-                    if (TS) tc_commit(bar_aempty + 8 * sa);
                 }
                 __syncwarp();
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
-            if (ok && elect_one()) tc_commit(bar_acc_full + 8 * ab);
+            if (ok && leader) tc_commit(bar_acc_full + 8 * ab);
             __syncwarp();
         }
     } else if (warp < 2 + 4 * EXPAND_GROUPS) {
@@ -369,42 +398,49 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         if (TS) {
             const int quad = warp & 3;            // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
             const int row = quad * 32 + lane;     // weight row inside the tile = TMEM lane
-            const uint32_t group = (uint32_t)(warp - 2) >> 2;  // this group takes the blocks with it % groups == group
-            uint32_t it = 0;
+            const uint32_t group = (uint32_t)(warp - 2) >> 2;  // takes the units with it % groups == group; owns slot `group`
+            const uint32_t a_dst = tmem_a + ((uint32_t)(quad * 32) << 16) + group * C::A_SLOT_COLS;
+            const long long total_units = (long long)kunits * ((total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x);
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                    if (it % EXPAND_GROUPS != group) continue;
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                    const uint32_t sa = it % A_STAGES, pha = (it / A_STAGES) & 1;
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag, 7, it));
-                    if (!ok) break;
-                    const uint4* src = reinterpret_cast<const uint4*>(smem + s * C::STAGE_BYTES + B_TILE_BYTES);
-                    const uint4 lo = src[row], hi = src[128 + row];
-                    uint32_t v[32];
-                    expand_word(lo.x, v + 0);
-                    expand_word(lo.y, v + 4);
-                    expand_word(lo.z, v + 8);
-                    expand_word(lo.w, v + 12);
-                    expand_word(hi.x, v + 16);
-                    expand_word(hi.y, v + 20);
-                    expand_word(hi.z, v + 24);
-                    expand_word(hi.w, v + 28);
-                    __syncwarp();  // every lane has consumed its packed words: the stage's weight bytes are free
-                    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1, abort_flag, 5, it));
-                    if (!ok) break;
-                    tc_fence_after();
-                    tmem_st32(tmem_a + ((uint32_t)(quad * 32) << 16) + sa * A_COLS, v);
-                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                    tc_fence_before();
-                    mbar_arrive(bar_afull + 8 * sa);
+            for (long long it64 = group; it64 < total_units && ok; it64 += EXPAND_GROUPS) {
+                const uint32_t it = (uint32_t)it64;
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag, 7, it));
+                if (!ok) break;
+                const uint4* src = reinterpret_cast<const uint4*>(smem + s * C::STAGE_BYTES + KBU * B_TILE_BYTES);
+                uint32_t v[KBU][32];
+#pragma unroll
+                for (int h = 0; h < KBU; ++h) {
+                    const uint4 lo = src[h * 256 + row], hi = src[h * 256 + 128 + row];
+                    expand_word(lo.x, v[h] + 0);
+                    expand_word(lo.y, v[h] + 4);
+                    expand_word(lo.z, v[h] + 8);
+                    expand_word(lo.w, v[h] + 12);
+                    expand_word(hi.x, v[h] + 16);
+                    expand_word(hi.y, v[h] + 20);
+                    expand_word(hi.z, v[h] + 24);
+                    expand_word(hi.w, v[h] + 28);
                 }
+                __syncwarp();  // every lane has consumed its packed words: the stage's weight bytes are free
+                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+                if (it >= (uint32_t)A_SLOTS) {
+                    // slot `group` was last read by the MMAs of unit it - A_SLOTS; their commit completes that stage's empty phase
+                    const uint32_t j = it - A_SLOTS, sj = j % STAGES, pj = (j / STAGES) & 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * sj, pj, abort_flag, 5, it));
+                    if (!ok) break;
+                }
+                tc_fence_after();
+#pragma unroll
+                for (int h = 0; h < KBU; ++h) tmem_st32(a_dst + h * (BK / 4), v[h]);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(bar_afull + 8 * group);
             }
         }
     } else {
         // ------------------------------------------------------------- epilogue
         const int quad = warp & 3;
+        const int cbase = ((warp - (2 + 4 * EXPAND_GROUPS)) >> 2) * EPI_COLS;  // this warp's share of the token columns
         const float alpha = *p.alpha;
         uint32_t tcount = 0;
         bool ok = true;
@@ -417,21 +453,33 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
             const int n = n0 + quad * 32 + lane;
             const bool n_ok = n < p.N;
 #pragma unroll 1
-            for (int c0 = 0; c0 < TILE_M; c0 += 32) {
+            for (int c0 = cbase; c0 < cbase + EPI_COLS; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + ab * ACC_COLS + c0, r);
-                // lane j fetches the rescale factor of token m0+c0+j (Eq. 2/3/7 prefactors); shared by shuffle
-                const int mj = m0 + c0 + lane;
-                const float sv = mj < p.M ? __ldg(p.scale + mj) * alpha : 0.f;
+                const int mrow = m0 + c0;
+                const int valid = p.M - mrow;  // tokens of this chunk that exist
+                const size_t o = (size_t)mrow * p.N + n;
+                float* yp = p.Y + o;
+                const float* sp = p.scale + mrow;
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (n_ok) {
+                    // y = fp32(acc) * (scale[m] * alpha): the prefactors of Eq. 2, 3 and 7
+                    if (valid >= 32) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float sc = __shfl_sync(0xffffffffu, sv, j);
-                    const int m = m0 + c0 + j;
-                    if (n_ok && m < p.M) {
-                        const size_t o = (size_t)m * p.N + n;
-                        p.Y[o] = (float)(int)r[j] * sc;
-                        if (p.acc) p.acc[o] = (int)r[j];
+                        for (int j = 0; j < 32; ++j) {
+                            *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                            yp += p.N;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < valid) yp[(size_t)j * p.N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                    }
+                    if (p.acc) {
+                        int32_t* ap = p.acc + o;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < valid) ap[(size_t)j * p.N] = (int)r[j];
                     }
                 }
             }

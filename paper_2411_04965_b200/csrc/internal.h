@@ -23,7 +23,7 @@ static inline int a48_round_up(int x, int m) { return (x + m - 1) / m * m; }
 struct bitnet_a48_weight {
     int N, K;
     int K4;          // bytes per canonical row
-    int Np, Kp;      // N rounded up to 256, K rounded up to 128 (tiled layouts)
+    int Np, Kp;      // N rounded up to 256, K rounded up to 256 (tiled layouts)
     unsigned flags;  // BITNET_A48_LAYOUT_* present
     float* alpha_dev;      // fp32 alpha
     double* alpha64_dev;   // float64 alpha (packing only)
