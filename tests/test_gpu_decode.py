@@ -1,0 +1,67 @@
+"""Decode kernel (up to 8 tokens, weight-streaming) against the oracle: int32 accumulators bit-exact,
+fp32 outputs within 1e-5 relative (Eq. 1 / Eq. 6)."""
+import numpy as np
+import pytest
+import torch
+
+from parity import max_rel_err
+from paper_2411_04965_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-5
+# (N, K): tiny; ragged N (not a multiple of 16) with K a multiple of 16 only; one, two and four CTAs per cluster;
+# the 3B and 7B projection shapes
+SHAPES = [(16, 128), (130, 144), (257, 400), (256, 512), (768, 2048), (3200, 3200), (8640, 3200), (3200, 8640),
+          (4096, 4096), (11008, 4096), (4096, 11008)]
+
+
+@pytest.mark.parametrize("N,K", SHAPES)
+@pytest.mark.parametrize("M", [1, 3, 8])
+@pytest.mark.parametrize("kind", ["int4", "topk"])
+def test_decode_matches_oracle(a48, oracle, cuda_dev, N, K, M, kind):
+    if N * K > 2e7 and M == 3:
+        pytest.skip("large shapes run at M = 1 and M = 8")
+    W = synth.latent_weights(N, K, seed=N + K)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_DECODE)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=M + K)
+        codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+        c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS)
+        act = a48.ACT_INT4
+    else:
+        x = synth.student_t3(M, K, seed=M + K)
+        codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+        c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS)
+        act = a48.ACT_TOPK_INT8
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    y, acc = a48.linear(w, codes, scale, act, a48.ALGO_DECODE, want_acc=True)
+    torch.cuda.synchronize()
+    assert a48.kernel_status() == [0, 0, 0, 0]
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+    y2 = a48.linear(w, codes, scale, act, a48.ALGO_AUTO)  # AUTO takes the same kernel: identical bits
+    assert torch.equal(y, y2)
+    w.free()
+
+
+def test_decode_extreme_codes(a48, cuda_dev):
+    # every code -127 against all-(+1) weights, then all-(-1) weights: the largest accumulators this path can see
+    N, K = 64, 11008
+    for sign in (1.0, -1.0):
+        w = a48.pack_ternary(torch.full((N, K), 0.05 * sign).to(cuda_dev), EPS, a48.LAYOUT_DECODE)
+        codes = torch.full((8, K), -127, dtype=torch.int8, device=cuda_dev)
+        scale = torch.ones(8, device=cuda_dev)
+        _, acc = a48.linear(w, codes, scale, a48.ACT_TOPK_INT8, a48.ALGO_DECODE, want_acc=True)
+        assert (acc.cpu() == int(-127 * K * sign)).all()
+
+
+def test_decode_rejects_more_than_eight_tokens(a48, cuda_dev):
+    w = a48.pack_ternary(synth.latent_weights(64, 128, seed=1).to(cuda_dev), EPS, a48.LAYOUT_DECODE)
+    codes = torch.zeros(9, 128, dtype=torch.int8, device=cuda_dev)
+    scale = torch.ones(9, device=cuda_dev)
+    with pytest.raises(a48.A48Error) as e:
+        a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_DECODE)
+    assert e.value.code == 4  # BITNET_A48_ERR_UNSUPPORTED
