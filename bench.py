@@ -370,7 +370,7 @@ def bench_decode(a48, synth, dev, stream, peaks, rank):
     c8f, d8f, _ = a48.topk_quant_int8(s_f, F // 2, EPS)
     y = torch.empty(1, F, dtype=torch.float32, device=dev)
     ws_need = max(a48.linear_workspace_bytes(w, 1) for w, *_ in weights)
-    ws = torch.empty(max(ws_need, 16), dtype=torch.uint8, device=dev)
+    ws = torch.zeros(max(ws_need, 16), dtype=torch.uint8, device=dev)
     packed_bytes = sum(w.packed_bytes for w, *_ in weights)
     nz = {"int4": float((c4 != 0).float().mean()), "topk_h": float((c8h != 0).float().mean()),
           "topk_f": float((c8f != 0).float().mean())}

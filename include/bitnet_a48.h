@@ -62,7 +62,7 @@ typedef enum {
     BITNET_A48_ALGO_AUTO = 0,
     BITNET_A48_ALGO_SIMPLE = 1,       /* tiled dp4a kernel, any shape; the in-tree cross-check */
     BITNET_A48_ALGO_GEMM_TCGEN05 = 2, /* prefill: tcgen05 kind::i8, int32 accumulators in TMEM */
-    BITNET_A48_ALGO_DECODE = 3,       /* M <= 64: streams every weight byte once */
+    BITNET_A48_ALGO_DECODE = 3,       /* M <= 8: streams every weight byte once */
     BITNET_A48_ALGO_DECODE_SPARSE = 4, /* M == 1: fetches only channels whose code is non-zero */
     BITNET_A48_ALGO_GEMM_TCGEN05_I8 = 5 /* comparison variant: int8 weight copy staged through shared memory */
 } bitnet_a48_algo;
@@ -136,7 +136,11 @@ bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t*
  * quantiser made the codes (it selects the zero-skipping decode path for
  * top-K inputs at M == 1; the result does not depend on it).
  * workspace_dev: at least bitnet_a48_linear_workspace_bytes(w, M) bytes, or NULL
- * when that is 0.  Nothing is allocated and nothing synchronises.
+ * when that is 0.  The decode kernel (M <= 8) adds the partial sums of tiles that
+ * two CTAs share into this scratch: it must be zero-filled before its first use
+ * (cudaMemset), every call leaves it zero-filled again, and two calls that may
+ * overlap on the device must not share it.  Nothing is allocated and nothing
+ * synchronises.
  */
 bitnet_a48_status bitnet_a48_linear(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
                                     int M, bitnet_a48_act kind, float* Y_dev, int32_t* acc_dev,

@@ -198,7 +198,7 @@ def linear(w: Weight, codes: torch.Tensor, scale: torch.Tensor, kind: int = ACT_
         acc = torch.empty(M, w.N, dtype=torch.int32, device=codes.device)
     need = linear_workspace_bytes(w, M)
     if workspace is None and need:
-        workspace = torch.empty(need, dtype=torch.uint8, device=codes.device)
+        workspace = torch.zeros(need, dtype=torch.uint8, device=codes.device)  # the decode scratch starts zeroed
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(lib().bitnet_a48_linear_ex(c_void_p(w.handle), _ptr(codes), _ptr(scale), M, kind, algo, _ptr(Y), _ptr(acc),
                                       _ptr(workspace), ws_bytes, _stream(stream)), "linear")

@@ -251,6 +251,8 @@ bitnet_a48_status bitnet_a48_bitlinear_host(const bitnet_a48_weight* w, const fl
     else if (kind == BITNET_A48_ACT_FP4) s = bitnet_a48_quant_fp4(X, M, w->K, codes, scale, stream);
     else return BITNET_A48_ERR_INVALID_ARG;
     if (s != BITNET_A48_OK) return s;
+    const size_t lin_bytes = a48_decode_workspace_bytes(w, M);
+    if (lin_bytes) A48_CUDA_TRY(cudaMemsetAsync(base + off[4], 0, lin_bytes, st));
     s = bitnet_a48_linear(w, codes, scale, M, kind, Y, nullptr, base + off[4], workspace_bytes - off[4], stream);
     if (s != BITNET_A48_OK) return s;
     A48_CUDA_TRY(cudaMemcpyAsync(Y_host, Y, (size_t)M * w->N * 4, cudaMemcpyDeviceToHost, st));

@@ -361,6 +361,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         return bitnet_a48_linear_ex(blk->w[wi], codes, scale, M, kind, BITNET_A48_ALGO_AUTO, out, nullptr, lin,
                                     lin_bytes, st);
     };
+    // the decode kernel wants its scratch zero on entry and leaves it zero
+    if (o.total > o.lin) A48_CUDA_TRY(cudaMemsetAsync(lin, 0, o.total - o.lin, st));
     // attention sub-layer
     A48_TRY(a48_launch_quant_int4(X, M, H, c.quant_eps, codes, scale, blk->g_attn, c.norm_eps, st));
     A48_TRY(linear(0, BITNET_A48_ACT_INT4, q));

@@ -85,7 +85,7 @@ def main():
         _, codes, scale, act = _acts(args.kind, M, K, dev)
         y = torch.empty(M, N, dtype=torch.float32, device=dev)
         need = a48.linear_workspace_bytes(ws[0], M)
-        wsp = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+        wsp = torch.zeros(max(need, 16), dtype=torch.uint8, device=dev)
 
         def run():
             for w in ws:

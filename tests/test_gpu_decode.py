@@ -65,3 +65,23 @@ def test_decode_rejects_more_than_eight_tokens(a48, cuda_dev):
     with pytest.raises(a48.A48Error) as e:
         a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_DECODE)
     assert e.value.code == 4  # BITNET_A48_ERR_UNSUPPORTED
+
+
+def test_decode_leaves_its_scratch_zeroed(a48, oracle, cuda_dev):
+    # one scratch buffer, zeroed once, serves several calls in a row (different tokens, different matrices of one shape)
+    N, K = 1100, 1536
+    Ws = [synth.latent_weights(N, K, seed=70 + i) for i in range(2)]
+    ws = [a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_DECODE) for W in Ws]
+    scratch = torch.zeros(a48.linear_workspace_bytes(ws[0], 5), dtype=torch.uint8, device=cuda_dev)
+    assert scratch.numel() > 0
+    for rep in range(4):
+        W, w = Ws[rep % 2], ws[rep % 2]
+        M = 1 + rep
+        x = synth.gaussian_outlier_activations(M, K, seed=80 + rep)
+        codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+        c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS)
+        t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+        acc_ref, _ = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8, want_y=False)
+        _, acc = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_DECODE, want_acc=True, workspace=scratch)
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert int(scratch.count_nonzero()) == 0
