@@ -6,17 +6,20 @@
 // busy.  The packed matrix is a sequence of 512-byte units (16 output rows x 128
 // channels, ordered tile by tile, see DecodeLayout).  The sequence is cut into one
 // contiguous, equally long piece per CTA whatever the tile boundaries ("stream-K"),
-// and every thread requests its 16 bytes of every unit of its warp's share with
-// cp.async right at the start, before anything else happens.  Inside a piece a warp
-// takes every sixteenth 128-channel chunk, over all tiles of the piece, so that it
-// loads the token codes of a chunk once and reuses them for each tile.
+// and the CTA requests its whole piece with cp.async right at the start, before
+// anything else happens (and, under programmatic dependent launch, before the
+// kernel ahead of it in the stream has finished).  Inside a piece a warp takes
+// every eighth 128-channel chunk, over all tiles of the piece, so that it loads the
+// token codes of a chunk once and reuses them for each tile.
 //
 // A warp turns each unit into int32 partial sums with four mma.sync m16n8k32
 // (u8 x s8): one 128-bit shared-memory load per lane is the A fragments of the four
 // MMAs, the 2-bit fields e = t+1 being isolated with a shift and a mask; the token
 // codes are the B fragments, copied once per CTA into shared memory (rows padded by
-// 16 bytes, which keeps the fragment loads free of bank conflicts) by the first
-// cp.async group, ahead of the weights.  Sums of a tile are added up in shared memory.
+// 16 bytes, which keeps the fragment loads free of bank conflicts) by bulk copies
+// with a barrier of their own.  With a single token the same fields go through dp4a
+// on the CUDA cores instead, which wastes no MMA columns.  Sums of a tile are added
+// up in shared memory.
 // A tile that lies wholly inside the CTA's piece is finished there.  The at most
 // two tiles a piece shares with its neighbours go through a global scratch array
 // of 64-bit words, one per (row, token): a contributor adds its partial sum
@@ -32,12 +35,12 @@
 
 namespace {
 
-constexpr int WARPS = 16;
+constexpr int WARPS = 8;
 constexpr int THREADS = 32 * WARPS;
 constexpr int UNIT_BYTES = 512;   // 16 rows x 128 channels of 2-bit codes
 constexpr int TOK = 8;            // tokens per launch (one MMA column group)
 constexpr int MAX_SHARE = 288;    // units per CTA (144 KB of packed weights)
-constexpr int MAX_TILES = 64;     // tiles a CTA's piece may touch (bounds the shared partial-sum array)
+constexpr int MAX_TILES = 24;     // tiles a CTA's piece may touch (bounds the shared partial-sum array)
 constexpr int MAX_GROUPS = 8;     // cp.async commit groups of weights per thread
 constexpr int NTL = 6;            // tiles whose accumulators a warp carries in registers at a time
 
@@ -72,6 +75,43 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ unsigned int g_decode_status[4];
+constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
+
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; when it runs out of time the first such event is recorded and the caller carries on.
+__device__ __noinline__ void mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    const unsigned long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try(bar, parity)) {
+        if ((++spins & 255u) == 0 && clock64() - t0 > kWaitClocks) {
+            if (atomicCAS(&g_decode_status[0], 0u, (unsigned)BITNET_A48_ERR_TIMEOUT) == 0u) {
+                g_decode_status[1] = 100;
+                g_decode_status[2] = blockIdx.x;
+                g_decode_status[3] = 0;
+            }
+            return;
+        }
+    }
+}
+
+// sum of four u8 x s8 products plus c
+__device__ __forceinline__ int dp4a_u8s8(uint32_t a, int b, int c) {
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 struct DecodeParams {
     const uint8_t* wdec;  // fragment-major packed weights
     const int8_t* codes;  // [M, K]
@@ -84,6 +124,7 @@ struct DecodeParams {
     int kchunks;          // units per tile (128-channel chunks of the padded K)
     int units;            // ntiles * kchunks
     int grid;             // CTAs
+    int tile_aligned;     // pieces end on tile boundaries: no tile is shared, the scratch stays untouched
     int act_row_bytes;    // padded K + 16
 };
 
@@ -99,78 +140,156 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     uint8_t* act = wbuf + (size_t)share_max * UNIT_BYTES;
     int* sacc = reinterpret_cast<int*>(act + (size_t)p.M * p.act_row_bytes);
     int* csum = sacc + MAX_TILES * 16 * TOK;
+    __shared__ uint64_t act_bar;  // completes when the token codes have landed
+    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&act_bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int u0 = (int)((long long)blockIdx.x * p.units / p.grid), u1 = (int)((long long)(blockIdx.x + 1) * p.units / p.grid);
+    int u0 = (int)((long long)blockIdx.x * p.units / p.grid), u1 = (int)((long long)(blockIdx.x + 1) * p.units / p.grid);
+    if (p.tile_aligned) {
+        const int ntiles = p.units / p.kchunks;
+        u0 = (int)((long long)blockIdx.x * ntiles / p.grid) * p.kchunks;
+        u1 = (int)((long long)(blockIdx.x + 1) * ntiles / p.grid) * p.kchunks;
+    }
     const int share = u1 - u0;
     const int first_tile = u0 / p.kchunks;
     const int ntl = share > 0 ? (u1 - 1) / p.kchunks - first_tile + 1 : 0;  // tiles this piece touches
 
-    // ---- first group: the token codes, rows of K bytes in 16-byte pieces (pieces past K are written as zeros)
-    const int row_pieces = p.kchunks * 8, real_pieces = p.K / 16;
-    for (int idx = threadIdx.x; idx < p.M * row_pieces; idx += THREADS) {
-        const int m = idx / row_pieces, c = idx % row_pieces;
-        uint8_t* dst = act + (size_t)m * p.act_row_bytes + c * 16;
-        if (c < real_pieces) cp_async16(dst, p.codes + (size_t)m * p.K + c * 16);
-        else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-    }
-    cp_async_commit();
-    // ---- then this warp's units: chunks warp, warp + WARPS, ... of every tile of the piece.  Nothing here
-    // depends on anything but the weights.
-    const int my_chunks = p.kchunks > warp ? (p.kchunks - warp + WARPS - 1) / WARPS : 0;
-    const int per_group = (my_chunks + MAX_GROUPS - 1) / MAX_GROUPS;  // chunks per commit group
-    const int ngroups = per_group ? (my_chunks + per_group - 1) / per_group : 0;
-    for (int j = 0; j < my_chunks; ++j) {
-        const int kc = warp + j * WARPS;
+    // ---- request the whole piece.  Copy group gq is chunks [gq*cg, (gq+1)*cg) of every tile of the piece (cg a
+    // multiple of the warp count); the CTA's threads share each contiguous run 16 bytes at a time.  Nothing here
+    // depends on anything but the weights, so it runs before the wait for the kernel ahead of this one in the
+    // stream (programmatic dependent launch): the weight stream of this call overlaps the tail of the previous one.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int cg = WARPS * ((p.kchunks + WARPS * MAX_GROUPS - 1) / (WARPS * MAX_GROUPS));
+    const int ngroups = (p.kchunks + cg - 1) / cg;
+    for (int gq = 0; gq < ngroups; ++gq) {
+        const int c_lo = gq * cg, c_hi = min(c_lo + cg, p.kchunks);
         for (int tl = 0; tl < ntl; ++tl) {
-            const int u = (first_tile + tl) * p.kchunks + kc;
-            if (u >= u0 && u < u1)
-                cp_async16(wbuf + (size_t)(u - u0) * UNIT_BYTES + lane * 16, p.wdec + (size_t)u * UNIT_BYTES + lane * 16);
+            const int base = (first_tile + tl) * p.kchunks;
+            const int lo = max(base + c_lo, u0), hi = min(base + c_hi, u1);
+            const uint8_t* src = p.wdec + (size_t)lo * UNIT_BYTES;
+            uint8_t* dst = wbuf + (size_t)(lo - u0) * UNIT_BYTES;
+            for (int o = threadIdx.x * 16; o < (hi - lo) * UNIT_BYTES; o += THREADS * 16) cp_async16(dst + o, src + o);
         }
-        if (j % per_group == per_group - 1 || j == my_chunks - 1) cp_async_commit();
+        cp_async_commit();
+    }
+    // ---- the token codes: one bulk copy per row, tracked by a barrier of their own so that waiting for them does
+    // not mean waiting for the weights (pieces past K are written as zeros).  They, the scratch and the outputs may
+    // belong to the previous kernel until it has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int row_pieces = p.kchunks * 8, real_pieces = p.K / 16;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(p.M * p.K)) : "memory");
+        for (int m = 0; m < p.M; ++m)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"((uint32_t)__cvta_generic_to_shared(act + (size_t)m * p.act_row_bytes)),
+                         "l"(p.codes + (size_t)m * p.K), "r"((uint32_t)p.K), "r"(bar)
+                         : "memory");
+    }
+    for (int idx = threadIdx.x; idx < p.M * (row_pieces - real_pieces); idx += THREADS) {
+        const int m = idx / (row_pieces - real_pieces), c = real_pieces + idx % (row_pieces - real_pieces);
+        *reinterpret_cast<uint4*>(act + (size_t)m * p.act_row_bytes + c * 16) = make_uint4(0, 0, 0, 0);
     }
 
-    for (int i = threadIdx.x; i < MAX_TILES * 16 * TOK; i += THREADS) sacc[i] = 0;
+    for (int i = threadIdx.x; i < ntl * 16 * TOK; i += THREADS) sacc[i] = 0;
     if (threadIdx.x < TOK) csum[threadIdx.x] = 0;
     __syncthreads();
-    // sum of the codes of every token (the offset of the e = t+1 encoding): each thread adds up the pieces it copied
-    cp_async_wait(ngroups);
-    {
-        int s = 0, cur = -1;
-        for (int idx = threadIdx.x; idx < p.M * row_pieces; idx += THREADS) {
-            const int m = idx / row_pieces, c = idx % row_pieces;
-            if (m != cur) {
-                if (cur >= 0) atomicAdd(csum + cur, s);
-                cur = m;
-                s = 0;
-            }
-            const uint4 v = *reinterpret_cast<const uint4*>(act + (size_t)m * p.act_row_bytes + c * 16);
-            s = __dp4a((int)v.x, 0x01010101, s);
-            s = __dp4a((int)v.y, 0x01010101, s);
-            s = __dp4a((int)v.z, 0x01010101, s);
-            s = __dp4a((int)v.w, 0x01010101, s);
-        }
-        if (cur >= 0) atomicAdd(csum + cur, s);
-    }
-    __syncthreads();
+    mbar_wait_bounded(bar, 0);  // the token codes are in shared memory
 
     // ---- this warp's units -> partial sums of their tiles.  Up to NTL tiles are carried in registers at a time
     // and walked side by side, so that consecutive MMAs are independent; one flush per tile at the end.
     const int g = lane >> 2, tig = lane & 3;
     const bool tok_ok = g < p.M;  // B-fragment column g is token g; columns of missing tokens stay zero
     const uint8_t* arow = act + (size_t)(tok_ok ? g : 0) * p.act_row_bytes + tig * 4;
+    if (p.M == 1) {
+        // One token: the MMA would spend seven of its eight columns on nothing, so the CUDA cores do it with dp4a.
+        // A word masked with 0x03030303 << 2q is four u8 fields e * 4^q of one row and one 32-channel slice; the
+        // sums of slice q carry the factor 4^q, which an exact shift removes at the end.  Rows g (words 0, 2) and
+        // g+8 (words 1, 3); the four lanes of a quad hold different channels of the same rows.
+        int xsum = 0;
+        for (int tb = 0; tb < ntl; tb += NTL) {
+            int lo[NTL][4], hi[NTL][4];
+#pragma unroll
+            for (int t = 0; t < NTL; ++t)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) lo[t][q] = hi[t][q] = 0;
+            for (int gq = 0; gq < ngroups; ++gq) {
+                if (tb == 0) {  // group gq has landed for every thread
+                    cp_async_wait(ngroups - 1 - gq);
+                    __syncthreads();
+                }
+                for (int kc = gq * cg + warp; kc < min((gq + 1) * cg, p.kchunks); kc += WARPS) {
+                int b[4][2];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    b[q][0] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + tig * 4);
+                    b[q][1] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + 16 + tig * 4);
+                }
+                if (tb == 0) {  // this chunk's share of sum_k x[k]: every quad holds the same words, quad 0 reports
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) xsum = __dp4a(b[q][1], 0x01010101, __dp4a(b[q][0], 0x01010101, xsum));
+                }
+                // all tiles are loaded, units outside the piece from a valid address and then blanked: no branches
+                uint4 a[NTL];
+#pragma unroll
+                for (int t = 0; t < NTL; ++t) {
+                    const int u = (first_tile + tb + t) * p.kchunks + kc;
+                    const bool have = tb + t < ntl && u >= u0 && u < u1;
+                    a[t] = *reinterpret_cast<const uint4*>(wbuf + (size_t)(have ? u - u0 : 0) * UNIT_BYTES + lane * 16);
+                    if (!have) a[t] = make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int t = 0; t < NTL; ++t) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t mq = 0x03030303u << (2 * q);
+                        lo[t][q] = dp4a_u8s8(a[t].x & mq, b[q][0], lo[t][q]);
+                        lo[t][q] = dp4a_u8s8(a[t].z & mq, b[q][1], lo[t][q]);
+                        hi[t][q] = dp4a_u8s8(a[t].y & mq, b[q][0], hi[t][q]);
+                        hi[t][q] = dp4a_u8s8(a[t].w & mq, b[q][1], hi[t][q]);
+                    }
+                }
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < NTL; ++t) {
+                if (tb + t >= ntl) continue;
+                int r0 = lo[t][0] + (lo[t][1] >> 2) + (lo[t][2] >> 4) + (lo[t][3] >> 6);
+                int r1 = hi[t][0] + (hi[t][1] >> 2) + (hi[t][2] >> 4) + (hi[t][3] >> 6);
+                r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
+                r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
+                if (tig == 0) {
+                    atomicAdd(sacc + ((size_t)(tb + t) * 16 + g) * TOK, r0);
+                    atomicAdd(sacc + ((size_t)(tb + t) * 16 + g + 8) * TOK, r1);
+                }
+            }
+        }
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+        if (lane == 0) atomicAdd(csum, xsum);
+    } else {
+    int xsum = 0;  // this lane's share of sum_k x[g][k]
     for (int tb = 0; tb < ntl; tb += NTL) {
         int c[NTL][4];
 #pragma unroll
         for (int t = 0; t < NTL; ++t) c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0;
-        for (int j = 0; j < my_chunks; ++j) {
-            const int kc = warp + j * WARPS;
-            if (tb == 0 && j % per_group == 0) cp_async_wait(ngroups - 1 - j / per_group);  // a lane reads only its own copies
+        for (int gq = 0; gq < ngroups; ++gq) {
+            if (tb == 0) {  // group gq has landed for every thread
+                cp_async_wait(ngroups - 1 - gq);
+                __syncthreads();
+            }
+            for (int kc = gq * cg + warp; kc < min((gq + 1) * cg, p.kchunks); kc += WARPS) {
             // B fragments of MMA q: channels 32q + 4tig .. +3 and 32q + 16 + 4tig .. +3 of token g
             uint32_t b[4][2];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 b[q][0] = tok_ok ? *reinterpret_cast<const uint32_t*>(arow + kc * 128 + q * 32) : 0u;
                 b[q][1] = tok_ok ? *reinterpret_cast<const uint32_t*>(arow + kc * 128 + q * 32 + 16) : 0u;
+                if (tb == 0) xsum = __dp4a((int)b[q][1], 0x01010101, __dp4a((int)b[q][0], 0x01010101, xsum));
             }
             uint4 a[NTL];
             bool have[NTL];
@@ -190,6 +309,7 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
                         mma_u8s8(c[t], (a[t].x >> (2 * q)) & kMask, (a[t].y >> (2 * q)) & kMask, (a[t].z >> (2 * q)) & kMask,
                                  (a[t].w >> (2 * q)) & kMask, b[q][0], b[q][1]);
             }
+            }
         }
 #pragma unroll
         for (int t = 0; t < NTL; ++t) {
@@ -205,6 +325,10 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
                 atomicAdd(dst + 8 * TOK + 1, c[t][3]);
             }
         }
+    }
+    xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+    xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+    if (tig == 0 && tok_ok) atomicAdd(csum + g, xsum);
     }
     __syncthreads();
 
@@ -288,7 +412,12 @@ bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* co
     if (tile_cap < cap) cap = tile_cap;
     if ((p.units + grid - 1) / grid > cap) grid = (p.units + cap - 1) / cap;
     p.grid = (int)grid;
-    const int share_max = (int)((p.units + grid - 1) / grid);
+    int share_max = (int)((p.units + grid - 1) / grid);
+    // With at least one tile per SM, whole tiles per piece cost a little balance (a piece is at most one tile longer
+    // than the average) and save the round trip through the scratch, which is the longer of the two at these sizes.
+    const long long aligned_share = ((ntiles + grid - 1) / grid) * p.kchunks;
+    p.tile_aligned = grid == sm_count() && ntiles >= grid && aligned_share <= cap;
+    if (p.tile_aligned) share_max = (int)aligned_share;
     const size_t smem = (size_t)share_max * UNIT_BYTES + (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
     if (smem > 227 * 1024 - 64) return BITNET_A48_ERR_UNSUPPORTED;
     static size_t smem_set = 0;
@@ -296,8 +425,25 @@ bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* co
         A48_CUDA_TRY(cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         smem_set = smem;
     }
-    decode_kernel<<<(unsigned)grid, THREADS, smem, st>>>(p, share_max);
-    A48_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = w->decode_prefetch_ok ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel, p, share_max));
+    w->decode_prefetch_ok = true;
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_read_decode_status(unsigned int words_host[4]) {
+    A48_CUDA_TRY(cudaMemcpyFromSymbol(words_host, g_decode_status, sizeof(unsigned int) * 4));
+    const unsigned int zero[4] = {0, 0, 0, 0};
+    A48_CUDA_TRY(cudaMemcpyToSymbol(g_decode_status, zero, sizeof(zero)));
     return BITNET_A48_OK;
 }
 

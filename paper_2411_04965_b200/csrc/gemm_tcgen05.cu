@@ -587,5 +587,10 @@ bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]) {
     A48_CUDA_TRY(cudaMemcpyFromSymbol(words_host, g_status, sizeof(unsigned int) * 4));
     const unsigned int zero[4] = {0, 0, 0, 0};
     A48_CUDA_TRY(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
+    unsigned int dec[4];
+    bitnet_a48_status ds = a48_read_decode_status(dec);
+    if (ds != BITNET_A48_OK) return ds;
+    if (words_host[0] == 0 && dec[0] != 0)
+        for (int i = 0; i < 4; ++i) words_host[i] = dec[i];
     return BITNET_A48_OK;
 }

@@ -34,6 +34,9 @@ struct bitnet_a48_weight {
     uint8_t* sparse;       // channel-major layout (or NULL)
     int8_t* i8;            // int8 codes [Np][Kp], zero padded (or NULL)
     size_t decode_bytes, sparse_bytes;
+    // false until the first decode launch: that one is fully ordered after the packing kernels, later ones may
+    // start fetching weights while the kernel ahead of them in the stream is still finishing
+    mutable bool decode_prefetch_ok;
 };
 
 struct bitnet_a48_block {
@@ -75,6 +78,7 @@ bool a48_decode_sparse_supported(const bitnet_a48_weight* w, int M);
 size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                     float* Y, int32_t* acc, void* ws, size_t ws_bytes, cudaStream_t st);
+bitnet_a48_status a48_read_decode_status(unsigned int words_host[4]);
 bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int8_t* codes, const float* scale,
                                            int M, float* Y, int32_t* acc, void* ws, size_t ws_bytes,
                                            cudaStream_t st);
