@@ -152,6 +152,26 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
                                        int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
 
+/* Decode BitLinear (M <= 8 tokens, weights packed with BITNET_A48_LAYOUT_DECODE) for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is a convenience of this library.)
+ * Some hosts of this code may not call cudaMalloc or any allocator at all once they are running: a plugin
+ * inside a serving process whose memory is handed out once at start-up and then frozen, a real-time loop
+ * that must not take the allocator's locks, a call made while a stream is being captured.  Such callers
+ * cannot give bitnet_a48_linear the scratch it asks for.  Here the scratch is an array inside the library
+ * image (1 MiB on every GPU that loads the library, until the process exits); the caller passes only the
+ * inputs and the output, and the call performs no cudaMalloc, cudaFree or other allocating call.
+ *   - Result: identical, bit for bit, to bitnet_a48_linear_ex(..., BITNET_A48_ALGO_DECODE, ...).
+ *   - Limits: N <= 16384 output features (BITNET_A48_ERR_LIMIT beyond), M <= 8 and the DECODE layout
+ *     (BITNET_A48_ERR_UNSUPPORTED otherwise).
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the part it uses on `stream` and then
+ *     runs the kernel on `stream`; two calls that can overlap on the GPU (different streams) race on it
+ *     and give wrong results - serialise them.
+ * Enqueues on `stream` and returns without synchronising. */
+bitnet_a48_status bitnet_a48_linear_decode_static(const bitnet_a48_weight* w, const int8_t* codes_dev,
+                                                  const float* scale_dev, int M, float* Y_dev, void* stream);
+
 /* One BitLinear end to end from HOST buffers (Eq. 6 with kind INT4, Eq. 1 with
  * kind TOPK_INT8 and top-k count k): copies X_host fp32 [M,K] to the device,
  * quantises, contracts, rescales and copies Y back to Y_host fp32 [M,N].

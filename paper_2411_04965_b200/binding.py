@@ -28,7 +28,7 @@ EXPORTS = [
     "bitnet_a48_linear", "bitnet_a48_linear_ex", "bitnet_a48_linear_workspace_bytes",
     "bitnet_a48_bitlinear_host", "bitnet_a48_bitlinear_host_workspace_bytes", "bitnet_a48_block_create",
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
-    "bitnet_a48_kernel_status",
+    "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_block_forward.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                                c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_kernel_status.argtypes = [POINTER(c_uint)]
+        L.bitnet_a48_linear_decode_static.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -203,6 +204,15 @@ def linear(w: Weight, codes: torch.Tensor, scale: torch.Tensor, kind: int = ACT_
     _check(lib().bitnet_a48_linear_ex(c_void_p(w.handle), _ptr(codes), _ptr(scale), M, kind, algo, _ptr(Y), _ptr(acc),
                                       _ptr(workspace), ws_bytes, _stream(stream)), "linear")
     return (Y, acc) if want_acc else Y
+
+
+def linear_decode_static(w: Weight, codes: torch.Tensor, scale: torch.Tensor, Y: torch.Tensor, stream=None):
+    """Decode BitLinear with the library's built-in scratch: allocates nothing, Y must be passed in."""
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.is_contiguous() and codes.shape[1] == w.K
+    assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and tuple(Y.shape) == (codes.shape[0], w.N)
+    _check(lib().bitnet_a48_linear_decode_static(c_void_p(w.handle), _ptr(codes), _ptr(scale), codes.shape[0], _ptr(Y),
+                                                 _stream(stream)), "linear_decode_static")
+    return Y
 
 
 def bitlinear_host_workspace_bytes(w: Weight, M: int) -> int:

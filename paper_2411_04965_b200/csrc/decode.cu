@@ -451,3 +451,41 @@ bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight*, const int8_
                                            void*, size_t, cudaStream_t) {
     return BITNET_A48_ERR_UNSUPPORTED;
 }
+
+// ---------------------------------------------------------------------------------------------------------------
+// Decode without any allocation: the scratch of the decode kernel lives in the library image.
+namespace {
+
+constexpr int kStaticMaxN = 16384;  // output features the built-in scratch covers
+// 64-bit fix-up words, one per (row, token): 1 MiB that every device loading the library holds until exit.
+static __device__ __align__(256) unsigned long long g_static_scratch[(size_t)kStaticMaxN * TOK];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices];  // device address of the array, per device, filled on first use
+
+}  // namespace
+
+extern "C" bitnet_a48_status bitnet_a48_linear_decode_static(const bitnet_a48_weight* w, const int8_t* codes_dev,
+                                                             const float* scale_dev, int M, float* Y_dev,
+                                                             void* stream) {
+    if (!w || !codes_dev || !scale_dev || !Y_dev) return BITNET_A48_ERR_INVALID_ARG;
+    if (M <= 0) return BITNET_A48_ERR_SHAPE;
+    if (!a48_aligned16(codes_dev) || !a48_aligned16(scale_dev) || !a48_aligned16(Y_dev)) return BITNET_A48_ERR_ALIGNMENT;
+    if (w->N > kStaticMaxN) return BITNET_A48_ERR_LIMIT;
+    if (!a48_decode_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return BITNET_A48_ERR_CUDA;
+    }
+    if (!g_static_scratch_ptr[dev]) {
+        // In host code the array's name is only a handle; kernels need the address the runtime gives for it.
+        void* ptr = nullptr;
+        A48_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    const size_t bytes = a48_decode_workspace_bytes(w, M);  // <= sizeof(g_static_scratch) because N <= kStaticMaxN
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the last call left (zeros, unless a call was cut short): start from zeros
+    A48_CUDA_TRY(cudaMemsetAsync(g_static_scratch_ptr[dev], 0, bytes, st));
+    return a48_launch_decode(w, codes_dev, scale_dev, M, Y_dev, nullptr, g_static_scratch_ptr[dev], bytes, st);
+}
