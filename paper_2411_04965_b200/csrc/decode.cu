@@ -31,6 +31,8 @@
 // per row) and applying scale[m]*alpha.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "internal.h"
 
 namespace {
@@ -209,65 +211,71 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         // sums of slice q carry the factor 4^q, which an exact shift removes at the end.  Rows g (words 0, 2) and
         // g+8 (words 1, 3); the four lanes of a quad hold different channels of the same rows.
         int xsum = 0;
-        for (int tb = 0; tb < ntl; tb += NTL) {
-            int lo[NTL][4], hi[NTL][4];
-#pragma unroll
-            for (int t = 0; t < NTL; ++t)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) lo[t][q] = hi[t][q] = 0;
-            for (int gq = 0; gq < ngroups; ++gq) {
-                if (tb == 0) {  // group gq has landed for every thread
-                    cp_async_wait(ngroups - 1 - gq);
-                    __syncthreads();
-                }
-                for (int kc = gq * cg + warp; kc < min((gq + 1) * cg, p.kchunks); kc += WARPS) {
-                int b[4][2];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    b[q][0] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + tig * 4);
-                    b[q][1] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + 16 + tig * 4);
-                }
-                if (tb == 0) {  // this chunk's share of sum_k x[k]: every quad holds the same words, quad 0 reports
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) xsum = __dp4a(b[q][1], 0x01010101, __dp4a(b[q][0], 0x01010101, xsum));
-                }
-                // all tiles are loaded, units outside the piece from a valid address and then blanked: no branches
-                uint4 a[NTL];
-#pragma unroll
-                for (int t = 0; t < NTL; ++t) {
-                    const int u = (first_tile + tb + t) * p.kchunks + kc;
-                    const bool have = tb + t < ntl && u >= u0 && u < u1;
-                    a[t] = *reinterpret_cast<const uint4*>(wbuf + (size_t)(have ? u - u0 : 0) * UNIT_BYTES + lane * 16);
-                    if (!have) a[t] = make_uint4(0, 0, 0, 0);
-                }
-#pragma unroll
-                for (int t = 0; t < NTL; ++t) {
-#pragma unroll
+        // the walk is compiled for 3 and for 6 tiles side by side: a piece of a long-K matrix touches few tiles
+        auto walk = [&](auto nt_c) {
+            constexpr int NT = decltype(nt_c)::value;
+            for (int tb = 0; tb < ntl; tb += NT) {
+                int lo[NT][4], hi[NT][4];
+    #pragma unroll
+                for (int t = 0; t < NT; ++t)
+    #pragma unroll
+                    for (int q = 0; q < 4; ++q) lo[t][q] = hi[t][q] = 0;
+                for (int gq = 0; gq < ngroups; ++gq) {
+                    if (tb == 0) {  // group gq has landed for every thread
+                        cp_async_wait(ngroups - 1 - gq);
+                        __syncthreads();
+                    }
+                    for (int kc = gq * cg + warp; kc < min((gq + 1) * cg, p.kchunks); kc += WARPS) {
+                    int b[4][2];
+    #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const uint32_t mq = 0x03030303u << (2 * q);
-                        lo[t][q] = dp4a_u8s8(a[t].x & mq, b[q][0], lo[t][q]);
-                        lo[t][q] = dp4a_u8s8(a[t].z & mq, b[q][1], lo[t][q]);
-                        hi[t][q] = dp4a_u8s8(a[t].y & mq, b[q][0], hi[t][q]);
-                        hi[t][q] = dp4a_u8s8(a[t].w & mq, b[q][1], hi[t][q]);
+                        b[q][0] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + tig * 4);
+                        b[q][1] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + 16 + tig * 4);
+                    }
+                    if (tb == 0) {  // this chunk's share of sum_k x[k]: every quad holds the same words, quad 0 reports
+    #pragma unroll
+                        for (int q = 0; q < 4; ++q) xsum = __dp4a(b[q][1], 0x01010101, __dp4a(b[q][0], 0x01010101, xsum));
+                    }
+                    // all tiles are loaded, units outside the piece from a valid address and then blanked: no branches
+                    uint4 a[NT];
+    #pragma unroll
+                    for (int t = 0; t < NT; ++t) {
+                        const int u = (first_tile + tb + t) * p.kchunks + kc;
+                        const bool have = tb + t < ntl && u >= u0 && u < u1;
+                        a[t] = *reinterpret_cast<const uint4*>(wbuf + (size_t)(have ? u - u0 : 0) * UNIT_BYTES + lane * 16);
+                        if (!have) a[t] = make_uint4(0, 0, 0, 0);
+                    }
+    #pragma unroll
+                    for (int t = 0; t < NT; ++t) {
+    #pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t mq = 0x03030303u << (2 * q);
+                            lo[t][q] = dp4a_u8s8(a[t].x & mq, b[q][0], lo[t][q]);
+                            lo[t][q] = dp4a_u8s8(a[t].z & mq, b[q][1], lo[t][q]);
+                            hi[t][q] = dp4a_u8s8(a[t].y & mq, b[q][0], hi[t][q]);
+                            hi[t][q] = dp4a_u8s8(a[t].w & mq, b[q][1], hi[t][q]);
+                        }
+                    }
                     }
                 }
+    #pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    if (tb + t >= ntl) continue;
+                    int r0 = lo[t][0] + (lo[t][1] >> 2) + (lo[t][2] >> 4) + (lo[t][3] >> 6);
+                    int r1 = hi[t][0] + (hi[t][1] >> 2) + (hi[t][2] >> 4) + (hi[t][3] >> 6);
+                    r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                    r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                    r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
+                    r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
+                    if (tig == 0) {
+                        atomicAdd(sacc + ((size_t)(tb + t) * 16 + g) * TOK, r0);
+                        atomicAdd(sacc + ((size_t)(tb + t) * 16 + g + 8) * TOK, r1);
+                    }
                 }
             }
-#pragma unroll
-            for (int t = 0; t < NTL; ++t) {
-                if (tb + t >= ntl) continue;
-                int r0 = lo[t][0] + (lo[t][1] >> 2) + (lo[t][2] >> 4) + (lo[t][3] >> 6);
-                int r1 = hi[t][0] + (hi[t][1] >> 2) + (hi[t][2] >> 4) + (hi[t][3] >> 6);
-                r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
-                r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
-                r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
-                r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
-                if (tig == 0) {
-                    atomicAdd(sacc + ((size_t)(tb + t) * 16 + g) * TOK, r0);
-                    atomicAdd(sacc + ((size_t)(tb + t) * 16 + g + 8) * TOK, r1);
-                }
-            }
-        }
+        };
+        if (ntl <= 3) walk(std::integral_constant<int, 3>{});
+        else walk(std::integral_constant<int, NTL>{});
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         if (lane == 0) atomicAdd(csum, xsum);
