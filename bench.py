@@ -405,14 +405,28 @@ def bench_decode(a48, synth, dev, stream, peaks, rank):
         frac = nz["int4"] if kind == "int4" else (nz["topk_h"] if k == H else nz["topk_f"])
         needed_bytes += w.packed_bytes * frac
 
+    ys = [torch.empty(1, F, dtype=torch.float32, device=dev) for _ in range(3)]
+    ws_multi = max(a48.linear_multi_workspace_bytes([w for w, *_ in weights[0:3]], 1),
+                   a48.linear_multi_workspace_bytes([w for w, *_ in weights[4:6]], 1), ws_need, 16)
+    ws = torch.zeros(ws_multi, dtype=torch.uint8, device=dev)
+    fused = not os.environ.get("A48_BENCH_DECODE_UNFUSED")
+
     def chain():
-        for w, n, k, kind in weights:
-            if kind == "int4":
-                a48.linear(w, c4, d4, a48.ACT_INT4, Y=y[:, :n], workspace=ws)
-            elif k == H:
-                a48.linear(w, c8h, d8h, a48.ACT_TOPK_INT8, Y=y[:, :n], workspace=ws)
+        # per layer: q,k,v share the attention input and gate,up the FFN input: one call each (one launch each)
+        for li in range(LAYERS):
+            (wq, *_), (wk, *_), (wv, *_), (wo, *_), (wg, *_), (wu, *_), (wd, *_) = weights[7 * li:7 * li + 7]
+            if fused:
+                a48.linear_multi([wq, wk, wv], c4, d4, a48.ACT_INT4, Ys=[t[:, :H] for t in ys], workspace=ws)
             else:
-                a48.linear(w, c8f, d8f, a48.ACT_TOPK_INT8, Y=y[:, :n], workspace=ws)
+                for w_, t in zip((wq, wk, wv), ys):
+                    a48.linear(w_, c4, d4, a48.ACT_INT4, Y=t[:, :H], workspace=ws)
+            a48.linear(wo, c8h, d8h, a48.ACT_TOPK_INT8, Y=y[:, :H], workspace=ws)
+            if fused:
+                a48.linear_multi([wg, wu], c4, d4, a48.ACT_INT4, Ys=[ys[0], ys[1]], workspace=ws)
+            else:
+                a48.linear(wg, c4, d4, a48.ACT_INT4, Y=ys[0], workspace=ws)
+                a48.linear(wu, c4, d4, a48.ACT_INT4, Y=ys[1], workspace=ws)
+            a48.linear(wd, c8f, d8f, a48.ACT_TOPK_INT8, Y=y[:, :H], workspace=ws)
 
     for _ in range(2):
         chain()
@@ -441,8 +455,9 @@ def bench_decode(a48, synth, dev, stream, peaks, rank):
            "ms_per_token_all_bitlinears": ms, "packed_weight_bytes": packed_bytes, "matrices": len(weights),
            "hbm_peak_gbs": peaks["hbm_gbs"], "frac_of_hbm_peak": gbs_dense / peaks["hbm_gbs"],
            "algorithmic_gbs": needed_bytes / (ms * 1e-3) / 1e9, "nonzero_code_fraction": nz,
-           "tokens_per_s": 1e3 / ms, "note": "CUDA-graph chain over 224 distinct matrices (1.6 GB >> L2); "
-           "value counts every packed byte, algorithmic_gbs only channels with a non-zero code"}
+           "tokens_per_s": 1e3 / ms, "launches_per_layer": 4 if fused else 7,
+           "note": "CUDA-graph chain over 224 distinct matrices (1.6 GB >> L2), q/k/v and gate/up each as one "
+           "bitnet_a48_linear_multi call; value counts every packed byte, algorithmic_gbs only channels with a non-zero code"}
     for w, *_ in weights:
         w.free()
     return out

@@ -152,6 +152,18 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
                                        int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
 
+/* Several BitLinears on the SAME activation codes (Eq. 6: q, k and v share the attention input; gate and up
+ * share the FFN input): Y_dev[j] = BitLinear(weights[j]) for j < count, all weights with the same K.
+ * For M <= 8 and count <= 4 with the DECODE layout this is one launch that streams the matrices as one
+ * sequence of tiles (a launch costs more than the HBM time of one 7B-shape matrix); otherwise it is
+ * `count` calls of bitnet_a48_linear one after the other.  Results are identical to separate calls.
+ * workspace_dev: bitnet_a48_linear_multi_workspace_bytes bytes, zero-filled before first use, left zero-filled
+ * (same contract as bitnet_a48_linear). */
+bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* const weights[], const int8_t* codes_dev,
+                                          const float* scale_dev, int M, bitnet_a48_act kind, float* const Y_dev[],
+                                          void* workspace_dev, size_t workspace_bytes, void* stream);
+size_t bitnet_a48_linear_multi_workspace_bytes(int count, const bitnet_a48_weight* const weights[], int M);
+
 /* Decode BitLinear (M <= 8 tokens, weights packed with BITNET_A48_LAYOUT_DECODE) for callers that cannot
  * allocate device memory.  (The paper has no counterpart: this is a convenience of this library.)
  * Some hosts of this code may not call cudaMalloc or any allocator at all once they are running: a plugin

@@ -28,7 +28,8 @@ EXPORTS = [
     "bitnet_a48_linear", "bitnet_a48_linear_ex", "bitnet_a48_linear_workspace_bytes",
     "bitnet_a48_bitlinear_host", "bitnet_a48_bitlinear_host_workspace_bytes", "bitnet_a48_block_create",
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
-    "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static",
+    "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
+    "bitnet_a48_linear_multi_workspace_bytes",
 ]
 
 
@@ -85,6 +86,10 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_block_forward.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                                c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_kernel_status.argtypes = [POINTER(c_uint)]
+        L.bitnet_a48_linear_multi.argtypes = [c_int, POINTER(c_void_p), c_void_p, c_void_p, c_int, c_int, POINTER(c_void_p),
+                                              c_void_p, c_size_t, c_void_p]
+        L.bitnet_a48_linear_multi_workspace_bytes.restype = c_size_t
+        L.bitnet_a48_linear_multi_workspace_bytes.argtypes = [c_int, POINTER(c_void_p), c_int]
         L.bitnet_a48_linear_decode_static.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
         _lib = L
     return _lib
@@ -204,6 +209,27 @@ def linear(w: Weight, codes: torch.Tensor, scale: torch.Tensor, kind: int = ACT_
     _check(lib().bitnet_a48_linear_ex(c_void_p(w.handle), _ptr(codes), _ptr(scale), M, kind, algo, _ptr(Y), _ptr(acc),
                                       _ptr(workspace), ws_bytes, _stream(stream)), "linear")
     return (Y, acc) if want_acc else Y
+
+
+def linear_multi_workspace_bytes(ws, M: int) -> int:
+    arr = (c_void_p * len(ws))(*[c_void_p(w.handle) for w in ws])
+    return int(lib().bitnet_a48_linear_multi_workspace_bytes(len(ws), arr, M))
+
+
+def linear_multi(ws, codes: torch.Tensor, scale: torch.Tensor, kind: int = ACT_INT4, Ys=None, workspace=None, stream=None):
+    """Several BitLinears (one K) on the same codes; one fused launch for M <= 8.  Returns the list of outputs."""
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.is_contiguous() and codes.shape[1] == ws[0].K
+    M = codes.shape[0]
+    if Ys is None:
+        Ys = [torch.empty(M, w.N, dtype=torch.float32, device=codes.device) for w in ws]
+    need = linear_multi_workspace_bytes(ws, M)
+    if workspace is None and need:
+        workspace = torch.zeros(need, dtype=torch.uint8, device=codes.device)
+    warr = (c_void_p * len(ws))(*[c_void_p(w.handle) for w in ws])
+    yarr = (c_void_p * len(ws))(*[_ptr(y) for y in Ys])
+    _check(lib().bitnet_a48_linear_multi(len(ws), warr, _ptr(codes), _ptr(scale), M, kind, yarr, _ptr(workspace),
+                                         workspace.numel() if workspace is not None else 0, _stream(stream)), "linear_multi")
+    return Ys
 
 
 def linear_decode_static(w: Weight, codes: torch.Tensor, scale: torch.Tensor, Y: torch.Tensor, stream=None):

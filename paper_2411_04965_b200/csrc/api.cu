@@ -212,6 +212,45 @@ bitnet_a48_status bitnet_a48_linear(const bitnet_a48_weight* w, const int8_t* co
                                 workspace_dev, workspace_bytes, stream);
 }
 
+size_t bitnet_a48_linear_multi_workspace_bytes(int count, const bitnet_a48_weight* const weights[], int M) {
+    if (count < 1 || !weights || M <= 0) return 0;
+    for (int j = 0; j < count; ++j)
+        if (!weights[j]) return 0;
+    size_t fused = count <= 4 ? a48_decode_multi_workspace_bytes(count, weights, M) : 0;
+    if (fused) return fused;
+    size_t single = 0;  // one call after the other: the largest single requirement
+    for (int j = 0; j < count; ++j) {
+        size_t b = a48_decode_workspace_bytes(weights[j], M);
+        single = b > single ? b : single;
+    }
+    return single;
+}
+
+bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* const weights[], const int8_t* codes_dev,
+                                          const float* scale_dev, int M, bitnet_a48_act kind, float* const Y_dev[],
+                                          void* workspace_dev, size_t workspace_bytes, void* stream) {
+    if (count < 1 || !weights || !codes_dev || !scale_dev || !Y_dev) return BITNET_A48_ERR_INVALID_ARG;
+    if ((int)kind < 0 || (int)kind > 2) return BITNET_A48_ERR_INVALID_ARG;
+    if (M <= 0) return BITNET_A48_ERR_SHAPE;
+    for (int j = 0; j < count; ++j) {
+        if (!weights[j] || !Y_dev[j]) return BITNET_A48_ERR_INVALID_ARG;
+        if (weights[j]->K != weights[0]->K) return BITNET_A48_ERR_SHAPE;
+        if (!a48_aligned16(Y_dev[j])) return BITNET_A48_ERR_ALIGNMENT;
+    }
+    if (!a48_aligned16(codes_dev) || !a48_aligned16(scale_dev) || !a48_aligned16(workspace_dev))
+        return BITNET_A48_ERR_ALIGNMENT;
+    if (!have_device()) return BITNET_A48_ERR_CUDA;
+    if (count <= 4 && a48_decode_multi_workspace_bytes(count, weights, M) > 0)
+        return a48_launch_decode_multi(count, weights, codes_dev, scale_dev, M, Y_dev, nullptr, workspace_dev,
+                                       workspace_bytes, (cudaStream_t)stream);
+    for (int j = 0; j < count; ++j) {
+        bitnet_a48_status s = bitnet_a48_linear(weights[j], codes_dev, scale_dev, M, kind, Y_dev[j], nullptr, workspace_dev,
+                                                workspace_bytes, stream);
+        if (s != BITNET_A48_OK) return s;
+    }
+    return BITNET_A48_OK;
+}
+
 // Workspace of the host-buffer entry point: X | codes | scale | Y | linear workspace, each 256-byte aligned.
 static size_t host_ws_layout(const bitnet_a48_weight* w, int M, size_t off[5]) {
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };

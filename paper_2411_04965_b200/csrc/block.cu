@@ -36,6 +36,12 @@ BlockWs block_ws(const bitnet_a48_block* blk, int B, int T) {
         size_t b = a48_decode_workspace_bytes(blk->w[i], (int)M);
         lin = b > lin ? b : lin;
     }
+    {  // q,k,v and gate,up go out as one call each
+        size_t b = bitnet_a48_linear_multi_workspace_bytes(3, blk->w, (int)M);
+        lin = b > lin ? b : lin;
+        b = bitnet_a48_linear_multi_workspace_bytes(2, blk->w + 4, (int)M);
+        lin = b > lin ? b : lin;
+    }
     w.lin = take(lin);
     w.total = o;
     return w;
@@ -365,9 +371,10 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     if (o.total > o.lin) A48_CUDA_TRY(cudaMemsetAsync(lin, 0, o.total - o.lin, st));
     // attention sub-layer
     A48_TRY(a48_launch_quant_int4(X, M, H, c.quant_eps, codes, scale, blk->g_attn, c.norm_eps, st));
-    A48_TRY(linear(0, BITNET_A48_ACT_INT4, q));
-    A48_TRY(linear(1, BITNET_A48_ACT_INT4, k));
-    A48_TRY(linear(2, BITNET_A48_ACT_INT4, v));
+    {
+        float* qkv[3] = {q, k, v};
+        A48_TRY(bitnet_a48_linear_multi(3, blk->w, codes, scale, M, BITNET_A48_ACT_INT4, qkv, lin, lin_bytes, st));
+    }
     {
         int n = T * (hd / 2);
         rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
@@ -394,8 +401,10 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
     // feed-forward sub-layer
     A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
-    A48_TRY(linear(4, BITNET_A48_ACT_INT4, gate));
-    A48_TRY(linear(5, BITNET_A48_ACT_INT4, up));
+    {
+        float* gu[2] = {gate, up};
+        A48_TRY(bitnet_a48_linear_multi(2, blk->w + 4, codes, scale, M, BITNET_A48_ACT_INT4, gu, lin, lin_bytes, st));
+    }
     relu2glu_kernel<<<(unsigned)((nF4 + 255) / 256), 256, 0, st>>>(gate, up, nF4);
     A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
     A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));

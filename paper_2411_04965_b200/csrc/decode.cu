@@ -114,21 +114,33 @@ __device__ __forceinline__ int dp4a_u8s8(uint32_t a, int b, int c) {
     return d;
 }
 
+constexpr int MAX_MATS = 4;  // matrices of one K that one launch can run on the same token codes
+
 struct DecodeParams {
-    const uint8_t* wdec;  // fragment-major packed weights
+    // The launch sees the 16-row tiles of its matrices as one sequence: matrix j owns tiles [tile_base[j], tile_base[j+1]).
+    const uint8_t* wdec[MAX_MATS];  // fragment-major packed weights
+    const float* alpha[MAX_MATS];
+    float* Y[MAX_MATS];             // [M, N_j]
+    int32_t* acc[MAX_MATS];         // [M, N_j] or nullptr
+    int N[MAX_MATS];
+    int tile_base[MAX_MATS + 1];
+    int count;
     const int8_t* codes;  // [M, K]
     const float* scale;   // [M]
-    const float* alpha;
-    float* Y;             // [M, N]
-    int32_t* acc;         // [M, N] or nullptr
     unsigned long long* ws;  // [ntiles][16][TOK]: arrivals << 40 | biased partial sums of shared tiles; zero between calls
-    int M, N, K;
+    int M, K;
     int kchunks;          // units per tile (128-channel chunks of the padded K)
     int units;            // ntiles * kchunks
     int grid;             // CTAs
     int tile_aligned;     // pieces end on tile boundaries: no tile is shared, the scratch stays untouched
     int act_row_bytes;    // padded K + 16
 };
+
+__device__ __forceinline__ int matrix_of(const DecodeParams& p, int tile) {
+    int j = 0;
+    while (j + 1 < p.count && tile >= p.tile_base[j + 1]) ++j;
+    return j;
+}
 
 // CTA that owns unit u when `units` units are cut into `grid` pieces [c*units/grid, (c+1)*units/grid).
 __device__ __forceinline__ int owner_of(int u, int units, int grid) {
@@ -171,7 +183,8 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         for (int tl = 0; tl < ntl; ++tl) {
             const int base = (first_tile + tl) * p.kchunks;
             const int lo = max(base + c_lo, u0), hi = min(base + c_hi, u1);
-            const uint8_t* src = p.wdec + (size_t)lo * UNIT_BYTES;
+            const int j = matrix_of(p, first_tile + tl);
+            const uint8_t* src = p.wdec[j] + ((size_t)lo - (size_t)p.tile_base[j] * p.kchunks) * UNIT_BYTES;
             uint8_t* dst = wbuf + (size_t)(lo - u0) * UNIT_BYTES;
             for (int o = threadIdx.x * 16; o < (hi - lo) * UNIT_BYTES; o += THREADS * 16) cp_async16(dst + o, src + o);
         }
@@ -341,7 +354,6 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     __syncthreads();
 
     // ---- finish the tiles: one thread per (tile, row, token)
-    const float alpha = *p.alpha;
     constexpr unsigned long long kLow = (1ull << 40) - 1;
     constexpr long long kBias = 1ll << 31;
     for (int idx = threadIdx.x; idx < ntl * 16 * p.M; idx += THREADS) {
@@ -358,12 +370,13 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
             sum = (long long)((old & kLow) + (mine & kLow)) - contributors * kBias;
             *slot = 0;
         }
-        const int n = tile * 16 + row;
-        if (n < p.N) {
+        const int j = matrix_of(p, tile);
+        const int n = (tile - p.tile_base[j]) * 16 + row;
+        if (n < p.N[j]) {
             const int v = (int)sum - csum[m];
-            const size_t o = (size_t)m * p.N + (size_t)n;
-            p.Y[o] = (float)v * (p.scale[m] * alpha);  // prefactors of Eq. 2, 3 and 7
-            if (p.acc) p.acc[o] = v;
+            const size_t o = (size_t)m * p.N[j] + (size_t)n;
+            p.Y[j][o] = (float)v * (p.scale[m] * __ldg(p.alpha[j]));  // prefactors of Eq. 2, 3 and 7
+            if (p.acc[j]) p.acc[j][o] = v;
         }
     }
 }
@@ -396,20 +409,48 @@ size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M) {
 
 bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                     float* Y, int32_t* acc, void* ws, size_t ws_bytes, cudaStream_t st) {
-    if (!ws || ws_bytes < a48_decode_workspace_bytes(w, M)) return BITNET_A48_ERR_NOMEM;
-    DecodeParams p;
-    p.wdec = w->decode;
+    return a48_launch_decode_multi(1, &w, codes, scale, M, &Y, &acc, ws, ws_bytes, st);
+}
+
+size_t a48_decode_multi_workspace_bytes(int count, const bitnet_a48_weight* const* ws_, int M) {
+    size_t total = 0;
+    for (int j = 0; j < count; ++j) {
+        if (!a48_decode_supported(ws_[j], M) || ws_[j]->K != ws_[0]->K) return 0;
+        total += ws_bytes_for(ws_[j]);
+    }
+    return total;
+}
+
+bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* const* wv, const int8_t* codes,
+                                          const float* scale, int M, float* const* Y, int32_t* const* acc, void* ws,
+                                          size_t ws_bytes, cudaStream_t st) {
+    if (count < 1 || count > MAX_MATS) return BITNET_A48_ERR_LIMIT;
+    const size_t need = a48_decode_multi_workspace_bytes(count, wv, M);
+    if (need == 0) return BITNET_A48_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < need) return BITNET_A48_ERR_NOMEM;
+    const bitnet_a48_weight* w = wv[0];
+    DecodeParams p = {};
+    long long ntiles = 0;
+    bool prefetch_ok = true;
+    for (int j = 0; j < count; ++j) {
+        p.wdec[j] = wv[j]->decode;
+        p.alpha[j] = wv[j]->alpha_dev;
+        p.Y[j] = Y[j];
+        p.acc[j] = acc ? acc[j] : nullptr;
+        p.N[j] = wv[j]->N;
+        p.tile_base[j] = (int)ntiles;
+        ntiles += (wv[j]->N + 15) / 16;
+        prefetch_ok = prefetch_ok && wv[j]->decode_prefetch_ok;
+    }
+    p.tile_base[count] = (int)ntiles;
+    p.count = count;
     p.codes = codes;
     p.scale = scale;
-    p.alpha = w->alpha_dev;
-    p.Y = Y;
-    p.acc = acc;
     p.ws = static_cast<unsigned long long*>(ws);
     p.M = M;
-    p.N = w->N;
     p.K = w->K;
     p.kchunks = w->Kp / 128;
-    const long long ntiles = (w->N + 15) / 16;
+    if (ntiles * p.kchunks >= (1ll << 31)) return BITNET_A48_ERR_UNSUPPORTED;
     p.units = (int)(ntiles * p.kchunks);
     p.act_row_bytes = w->Kp + 16;
     // one piece per SM unless a piece would then not fit: at most MAX_SHARE units and MAX_TILES tiles per piece
@@ -418,13 +459,17 @@ bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* co
     long long cap = MAX_SHARE;
     const long long tile_cap = (long long)(MAX_TILES - 2) * p.kchunks;
     if (tile_cap < cap) cap = tile_cap;
-    if ((p.units + grid - 1) / grid > cap) grid = (p.units + cap - 1) / cap;
+    if ((p.units + grid - 1) / grid > cap) {
+        // more pieces than SMs: a whole number of rounds (pieces of two rounds can share an SM when they are small)
+        const long long rounds = (p.units + (long long)sm_count() * cap - 1) / ((long long)sm_count() * cap);
+        grid = rounds * sm_count();
+    }
     p.grid = (int)grid;
     int share_max = (int)((p.units + grid - 1) / grid);
     // With at least one tile per SM, whole tiles per piece cost a little balance (a piece is at most one tile longer
     // than the average) and save the round trip through the scratch, which is the longer of the two at these sizes.
     const long long aligned_share = ((ntiles + grid - 1) / grid) * p.kchunks;
-    p.tile_aligned = grid == sm_count() && ntiles >= grid && aligned_share <= cap;
+    p.tile_aligned = grid % sm_count() == 0 && ntiles >= grid && aligned_share <= cap;
     if (p.tile_aligned) share_max = (int)aligned_share;
     const size_t smem = (size_t)share_max * UNIT_BYTES + (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
     if (smem > 227 * 1024 - 64) return BITNET_A48_ERR_UNSUPPORTED;
@@ -440,11 +485,11 @@ bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* co
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = w->decode_prefetch_ok ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = prefetch_ok ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel, p, share_max));
-    w->decode_prefetch_ok = true;
+    for (int j = 0; j < count; ++j) wv[j]->decode_prefetch_ok = true;
     return BITNET_A48_OK;
 }
 

@@ -78,6 +78,11 @@ bool a48_decode_sparse_supported(const bitnet_a48_weight* w, int M);
 size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                     float* Y, int32_t* acc, void* ws, size_t ws_bytes, cudaStream_t st);
+// Several matrices of one K (all with the decode layout) on the same token codes in one launch, e.g. q, k and v.
+size_t a48_decode_multi_workspace_bytes(int count, const bitnet_a48_weight* const* w, int M);
+bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* const* w, const int8_t* codes,
+                                          const float* scale, int M, float* const* Y, int32_t* const* acc, void* ws,
+                                          size_t ws_bytes, cudaStream_t st);
 bitnet_a48_status a48_read_decode_status(unsigned int words_host[4]);
 bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int8_t* codes, const float* scale,
                                            int M, float* Y, int32_t* acc, void* ws, size_t ws_bytes,

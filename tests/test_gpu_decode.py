@@ -85,3 +85,17 @@ def test_decode_leaves_its_scratch_zeroed(a48, oracle, cuda_dev):
         _, acc = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_DECODE, want_acc=True, workspace=scratch)
         assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
         assert int(scratch.count_nonzero()) == 0
+
+
+@pytest.mark.parametrize("Ns,K,M", [((4096, 4096, 4096), 4096, 1), ((11008, 11008), 4096, 3), ((130, 257, 64, 1000), 400, 8),
+                                    ((512, 256), 1536, 12)])
+def test_linear_multi_equals_separate_calls(a48, cuda_dev, Ns, K, M):
+    # q/k/v-like and gate/up-like groups on shared codes: the fused launch gives the bits of the separate calls
+    # (which the tests above pin to the oracle); M = 12 takes the one-after-the-other route
+    ws = [a48.pack_ternary(synth.latent_weights(N, K, seed=N + i).to(cuda_dev), EPS, a48.LAYOUT_ALL) for i, N in enumerate(Ns)]
+    x = synth.gaussian_outlier_activations(M, K, seed=9).to(cuda_dev)
+    codes, scale = a48.quant_int4(x, EPS)
+    fused = a48.linear_multi(ws, codes, scale, a48.ACT_INT4)
+    for w, y in zip(ws, fused):
+        assert torch.equal(y, a48.linear(w, codes, scale, a48.ACT_INT4))
+    assert a48.kernel_status() == [0, 0, 0, 0]
