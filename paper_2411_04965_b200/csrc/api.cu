@@ -160,7 +160,8 @@ bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t*
 
 size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M) {
     if (!w || M <= 0) return 0;
-    return a48_decode_workspace_bytes(w, M);
+    const size_t dense = a48_decode_workspace_bytes(w, M), sparse = a48_decode_sparse_workspace_bytes(w, M);
+    return dense > sparse ? dense : sparse;
 }
 
 bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
@@ -175,10 +176,12 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
     if (!have_device()) return BITNET_A48_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
     if (algo == BITNET_A48_ALGO_AUTO) {
-        if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M))
-            algo = BITNET_A48_ALGO_DECODE_SPARSE;
-        else if (a48_decode_supported(w, M))
+        // At the 3B/7B shapes one launch is latency-bound, and the dense kernel (dp4a on whole rows) beats the
+        // zero-skipping one although it moves twice the bytes; the latter is taken when it is the only one possible.
+        if (a48_decode_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE;
+        else if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M))
+            algo = BITNET_A48_ALGO_DECODE_SPARSE;
         else if (a48_gemm_tcgen05_supported(w, M, false))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05;
         else

@@ -402,7 +402,6 @@ bool a48_decode_supported(const bitnet_a48_weight* w, int M) {
     return w->decode != nullptr && M >= 1 && M <= TOK && w->K % 16 == 0 && (size_t)M * (w->Kp + 16) <= 96 * 1024 &&
            (long long)((w->N + 15) / 16) * (w->Kp / 128) < (1ll << 31);
 }
-bool a48_decode_sparse_supported(const bitnet_a48_weight*, int) { return false; }
 size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M) {
     return a48_decode_supported(w, M) ? ws_bytes_for(w) : 0;
 }
@@ -500,10 +499,6 @@ bitnet_a48_status a48_read_decode_status(unsigned int words_host[4]) {
     return BITNET_A48_OK;
 }
 
-bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight*, const int8_t*, const float*, int, float*, int32_t*,
-                                           void*, size_t, cudaStream_t) {
-    return BITNET_A48_ERR_UNSUPPORTED;
-}
 
 // ---------------------------------------------------------------------------------------------------------------
 // Decode without any allocation: the scratch of the decode kernel lives in the library image.

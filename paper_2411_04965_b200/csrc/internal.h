@@ -76,6 +76,7 @@ bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]);
 bool a48_decode_supported(const bitnet_a48_weight* w, int M);
 bool a48_decode_sparse_supported(const bitnet_a48_weight* w, int M);
 size_t a48_decode_workspace_bytes(const bitnet_a48_weight* w, int M);
+size_t a48_decode_sparse_workspace_bytes(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_decode(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                     float* Y, int32_t* acc, void* ws, size_t ws_bytes, cudaStream_t st);
 // Several matrices of one K (all with the decode layout) on the same token codes in one launch, e.g. q, k and v.

@@ -99,3 +99,25 @@ def test_linear_multi_equals_separate_calls(a48, cuda_dev, Ns, K, M):
     for w, y in zip(ws, fused):
         assert torch.equal(y, a48.linear(w, codes, scale, a48.ACT_INT4))
     assert a48.kernel_status() == [0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("N,K", [(16, 128), (130, 144), (1000, 250), (3200, 3200), (4096, 11008), (11008, 4096)])
+@pytest.mark.parametrize("kfrac", [0.5, 0.05, 1.0])
+def test_decode_sparse_matches_oracle(a48, oracle, cuda_dev, N, K, kfrac):
+    # zero-skipping kernel: one token, top-K codes (about kfrac of the channels survive)
+    W = synth.latent_weights(N, K, seed=N + K)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_SPARSE)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    x = synth.student_t3(1, K, seed=K)
+    k = max(1, int(K * kfrac))
+    codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), k, EPS)
+    c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), k, EPS)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    scratch = torch.zeros(a48.linear_workspace_bytes(w, 1), dtype=torch.uint8, device=cuda_dev)
+    for _ in range(2):  # twice on one scratch: it is left zeroed
+        y, acc = a48.linear(w, codes, scale, a48.ACT_TOPK_INT8, a48.ALGO_DECODE_SPARSE, want_acc=True, workspace=scratch)
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+        assert int(scratch.count_nonzero()) == 0
+    w.free()
