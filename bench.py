@@ -196,6 +196,43 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- replicas (N > 1)
+class Replicas:
+    """The only cross-rank steps of the benchmark: a barrier, and the slowest rank's time.
+
+    Every rank runs an independent replica (tokens shard with no exchange); the job's throughput is the work
+    of all ranks divided by the slowest rank's time.  Backend "nccl" on GPUs, "gloo" in the CPU tests.
+    """
+
+    def __init__(self, world, backend="nccl", device=None):
+        self.world, self.device = world, device
+        if world > 1:
+            import torch.distributed as dist
+            self.dist = dist
+            if not dist.is_initialized():
+                kw = {"device_id": device} if backend == "nccl" else {}
+                dist.init_process_group(backend, **kw)
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+
+    def max_ms(self, ms):
+        if self.world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def job_value(self, units_per_rank, ms_per_step_max):
+        """Whole-job throughput: all ranks' units per second of the slowest rank's step."""
+        return units_per_rank * self.world / (ms_per_step_max * 1e-3)
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
 # --------------------------------------------------------------------------- our arm
 class Layer:
     """Packed weights of one 7B-shape layer plus resident activation buffers."""
@@ -219,29 +256,20 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the BitLinear path has no CPU fallback")
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    reps = Replicas(world, "nccl", dev)
     if rank == 0:
         a48_build.build()
-    if world > 1:
-        dist.barrier()
+    reps.barrier()
     a48.lib()
     peaks = load_peaks()
     M = M_PREFILL
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = reps.max_ms
 
     # ---- resident inputs: larger than L2 (268 MB + 268 MB + 721 MB of fp32 activations per step)
     layer = Layer(a48, dev, seed=4 + rank, layouts=a48.LAYOUT_ALL)
@@ -295,7 +323,7 @@ def run_ours(args):
     clocks = sampler.stop(t_begin, t_end)
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     ms_per_step = ms_total / args.steps
-    tops = STEP_OPS * world / (ms_per_step * 1e-3) / 1e12
+    tops = reps.job_value(STEP_OPS, ms_per_step) / 1e12
 
     gemm_ms = sum(a.elapsed_time(b) for _, a, b in gemm_events)
     gemm_ops = sum(2 * M * n * k for name, _, _ in gemm_events for pn, n, k, _ in PROJ if pn == name)
@@ -376,8 +404,7 @@ def run_ours(args):
             "cpu_baseline": cpu_baseline, "decode": decode, "block": block,
         }
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 def bench_decode(a48, synth, dev, stream, peaks, rank):

@@ -99,3 +99,26 @@ def test_pack_ternary_ties_and_ternary_latents(a48, oracle, cuda_dev):
     codes, alpha = a48.weight_unpack(w)
     t_ref, a_ref = oracle.ternarise(W.numpy(), EPS)
     assert np.array_equal(codes.cpu().numpy(), t_ref) and alpha == np.float32(a_ref)
+
+
+@pytest.mark.parametrize("K,kind", [(4096, "int4"), (4096, "topk"), (11008, "topk")])
+def test_quantisers_at_benchmark_size_sampled(a48, oracle, cuda_dev, K, kind):
+    # The benchmark's launch configuration (16384 tokens of the 7B shape); the oracle recomputes 48 sampled rows,
+    # and every row is checked for what holds at any size: code range, at most k survivors, the maximum coded +-127.
+    M = 16384
+    g = torch.Generator().manual_seed(K)
+    rows = torch.cat([torch.tensor([0, 1, M - 1]), torch.randint(0, M, (45,), generator=g)]).to(cuda_dev)
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=40, device=cuda_dev)
+        codes, scale = a48.quant_int4(x, EPS)
+        q_ref, d_ref = oracle.quant_int4(x[rows].cpu().numpy(), EPS, nthreads=8)
+        assert int(codes.min()) >= -8 and int(codes.max()) <= 7
+    else:
+        x = synth.student_t3(M, K, seed=41, device=cuda_dev)
+        codes, scale, _ = a48.topk_quant_int8(x, K // 2, EPS)
+        q_ref, d_ref, _ = oracle.topk_quant_int8(x[rows].cpu().numpy(), K // 2, EPS, nthreads=8)
+        nz = (codes != 0).sum(1)
+        assert int(nz.max()) <= K // 2  # at most k survivors (kept entries below gamma/254 still code to 0)
+        assert bool((codes.abs().amax(1) == 127).all())
+    assert np.array_equal(codes[rows].cpu().numpy(), q_ref)
+    assert np.array_equal(scale[rows].cpu().numpy(), d_ref.astype(np.float32))
