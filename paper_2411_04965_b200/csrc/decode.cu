@@ -178,17 +178,24 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int cg = WARPS * ((p.kchunks + WARPS * MAX_GROUPS - 1) / (WARPS * MAX_GROUPS));
     const int ngroups = (p.kchunks + cg - 1) / cg;
-    for (int gq = 0; gq < ngroups; ++gq) {
-        const int c_lo = gq * cg, c_hi = min(c_lo + cg, p.kchunks);
-        for (int tl = 0; tl < ntl; ++tl) {
-            const int base = (first_tile + tl) * p.kchunks;
-            const int lo = max(base + c_lo, u0), hi = min(base + c_hi, u1);
-            const int j = matrix_of(p, first_tile + tl);
-            const uint8_t* src = p.wdec[j] + ((size_t)lo - (size_t)p.tile_base[j] * p.kchunks) * UNIT_BYTES;
-            uint8_t* dst = wbuf + (size_t)(lo - u0) * UNIT_BYTES;
-            for (int o = threadIdx.x * 16; o < (hi - lo) * UNIT_BYTES; o += THREADS * 16) cp_async16(dst + o, src + o);
+    {
+        // a warp takes whole units (lane l the l-th 16 bytes of each), so that one cp.async instruction moves 512
+        // contiguous bytes and the only arithmetic per copy is the unit index
+        const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16 - (uint32_t)u0 * UNIT_BYTES;
+        for (int gq = 0; gq < ngroups; ++gq) {
+            const int c_lo = gq * cg, c_hi = min(c_lo + cg, p.kchunks);
+            for (int tl = 0; tl < ntl; ++tl) {
+                const int base = (first_tile + tl) * p.kchunks;
+                const int j = matrix_of(p, first_tile + tl);
+                const uint8_t* src0 = p.wdec[j] + lane * 16 - (size_t)p.tile_base[j] * p.kchunks * UNIT_BYTES;
+                for (int u = base + c_lo + warp; u < base + c_hi; u += WARPS)
+                    if (u >= u0 && u < u1)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)u * UNIT_BYTES),
+                                     "l"(src0 + (size_t)u * UNIT_BYTES)
+                                     : "memory");
+            }
+            cp_async_commit();
         }
-        cp_async_commit();
     }
     // ---- the token codes: one bulk copy per row, tracked by a barrier of their own so that waiting for them does
     // not mean waiting for the weights (pieces past K are written as zeros).  They, the scratch and the outputs may
@@ -224,7 +231,7 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         // sums of slice q carry the factor 4^q, which an exact shift removes at the end.  Rows g (words 0, 2) and
         // g+8 (words 1, 3); the four lanes of a quad hold different channels of the same rows.
         int xsum = 0;
-        // the walk is compiled for 3 and for 6 tiles side by side: a piece of a long-K matrix touches few tiles
+        // the walk is compiled for 3, 4, 5 and 6 tiles side by side: blank slots would cost as much as real ones
         auto walk = [&](auto nt_c) {
             constexpr int NT = decltype(nt_c)::value;
             for (int tb = 0; tb < ntl; tb += NT) {
@@ -288,6 +295,8 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
             }
         };
         if (ntl <= 3) walk(std::integral_constant<int, 3>{});
+        else if (ntl == 4) walk(std::integral_constant<int, 4>{});
+        else if (ntl == 5) walk(std::integral_constant<int, 5>{});
         else walk(std::integral_constant<int, NTL>{});
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
