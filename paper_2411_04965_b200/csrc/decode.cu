@@ -303,10 +303,12 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         if (lane == 0) atomicAdd(csum, xsum);
     } else {
     int xsum = 0;  // this lane's share of sum_k x[g][k]
-    for (int tb = 0; tb < ntl; tb += NTL) {
-        int c[NTL][4];
+    auto walk = [&](auto nt_c) {
+    constexpr int NT = decltype(nt_c)::value;
+    for (int tb = 0; tb < ntl; tb += NT) {
+        int c[NT][4];
 #pragma unroll
-        for (int t = 0; t < NTL; ++t) c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0;
+        for (int t = 0; t < NT; ++t) c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0;
         for (int gq = 0; gq < ngroups; ++gq) {
             if (tb == 0) {  // group gq has landed for every thread
                 cp_async_wait(ngroups - 1 - gq);
@@ -321,28 +323,28 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
                 b[q][1] = tok_ok ? *reinterpret_cast<const uint32_t*>(arow + kc * 128 + q * 32 + 16) : 0u;
                 if (tb == 0) xsum = __dp4a((int)b[q][1], 0x01010101, __dp4a((int)b[q][0], 0x01010101, xsum));
             }
-            uint4 a[NTL];
-            bool have[NTL];
+            // all tiles are loaded, units outside the piece from a valid address and then blanked (a zero A fragment
+            // adds nothing), so that no MMA sits behind a branch
+            uint4 a[NT];
 #pragma unroll
-            for (int t = 0; t < NTL; ++t) {
+            for (int t = 0; t < NT; ++t) {
                 const int u = (first_tile + tb + t) * p.kchunks + kc;
-                have[t] = tb + t < ntl && u >= u0 && u < u1;
-                a[t] = make_uint4(0, 0, 0, 0);
-                if (have[t]) a[t] = *reinterpret_cast<const uint4*>(wbuf + (size_t)(u - u0) * UNIT_BYTES + lane * 16);
+                const bool have = tb + t < ntl && u >= u0 && u < u1;
+                a[t] = *reinterpret_cast<const uint4*>(wbuf + (size_t)(have ? u - u0 : 0) * UNIT_BYTES + lane * 16);
+                if (!have) a[t] = make_uint4(0, 0, 0, 0);
             }
             constexpr uint32_t kMask = 0x03030303u;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
 #pragma unroll
-                for (int t = 0; t < NTL; ++t)
-                    if (have[t])
+                for (int t = 0; t < NT; ++t)
                         mma_u8s8(c[t], (a[t].x >> (2 * q)) & kMask, (a[t].y >> (2 * q)) & kMask, (a[t].z >> (2 * q)) & kMask,
                                  (a[t].w >> (2 * q)) & kMask, b[q][0], b[q][1]);
             }
             }
         }
 #pragma unroll
-        for (int t = 0; t < NTL; ++t) {
+        for (int t = 0; t < NT; ++t) {
             if (tb + t >= ntl) continue;
             // rows g and g+8 of the tile, tokens 2*tig and 2*tig+1
             int* dst = sacc + ((size_t)(tb + t) * 16 + g) * TOK + 2 * tig;
@@ -356,6 +358,11 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
             }
         }
     }
+    };
+    if (ntl <= 3) walk(std::integral_constant<int, 3>{});
+    else if (ntl == 4) walk(std::integral_constant<int, 4>{});
+    else if (ntl == 5) walk(std::integral_constant<int, 5>{});
+    else walk(std::integral_constant<int, NTL>{});
     xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
     xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
     if (tig == 0 && tok_ok) atomicAdd(csum + g, xsum);
@@ -472,6 +479,12 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
         const long long rounds = (p.units + (long long)sm_count() * cap - 1) / ((long long)sm_count() * cap);
         grid = rounds * sm_count();
     }
+    // Two CTAs must fit on an SM for a launch to request its weights while its predecessor still computes: with
+    // many tokens the staged codes take room, so the pieces get shorter (more rounds of pieces) until they do.
+    const size_t fixed_smem = (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
+    while (fixed_smem <= 64 * 1024 && grid % sm_count() == 0 && grid < 2ll * sm_count() && p.units / grid > 32 &&
+           fixed_smem + (size_t)((p.units + grid - 1) / grid) * UNIT_BYTES > 112 * 1024)
+        grid += sm_count();
     p.grid = (int)grid;
     int share_max = (int)((p.units + grid - 1) / grid);
     // With at least one tile per SM, whole tiles per piece cost a little balance (a piece is at most one tile longer
