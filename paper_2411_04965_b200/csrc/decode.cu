@@ -398,13 +398,12 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
 }
 
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return n;
+    static int n[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int& c = n[dev & 63];
+    if (!c) cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev);
+    return c;
 }
 
 size_t align256(size_t v) { return (v + 255) / 256 * 256; }
@@ -494,7 +493,10 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     if (p.tile_aligned) share_max = (int)aligned_share;
     const size_t smem = (size_t)share_max * UNIT_BYTES + (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
     if (smem > 227 * 1024 - 64) return BITNET_A48_ERR_UNSUPPORTED;
-    static size_t smem_set = 0;
+    static size_t smem_set_dev[64] = {};  // the attribute is per device
+    int dev = 0;
+    A48_CUDA_TRY(cudaGetDevice(&dev));
+    size_t& smem_set = smem_set_dev[dev & 63];
     if (smem > smem_set) {
         A48_CUDA_TRY(cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         smem_set = smem;

@@ -89,13 +89,12 @@ __global__ void __launch_bounds__(THREADS) decode_sparse_kernel(const uint32_t* 
 }
 
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return n;
+    static int n[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int& c = n[dev & 63];
+    if (!c) cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev);
+    return c;
 }
 
 }  // namespace

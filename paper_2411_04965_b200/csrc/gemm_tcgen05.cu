@@ -526,23 +526,24 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, 
 }
 
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return n;
+    static int n[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int& c = n[dev & 63];
+    if (!c) cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev);
+    return c;
 }
 
 template <bool TS>
 bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
                          int32_t* acc, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};  // the attribute is per device
+    int dev = 0;
+    A48_CUDA_TRY(cudaGetDevice(&dev));
+    if (!attr_set[dev & 63]) {
         A48_CUDA_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<TS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           Cfg<TS>::SMEM_BYTES));
-        attr_set = true;
+        attr_set[dev & 63] = true;
     }
     CUtensorMap tm_act, tm_w;
     if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TILE_M)) return BITNET_A48_ERR_CUDA;
