@@ -215,6 +215,78 @@ __device__ __forceinline__ Select radix_select(int k, unsigned* hist, unsigned* 
     return Select{prefix, kr, eq_total};
 }
 
+// The same selection for a whole block working on one row, with far fewer instructions per element: the first
+// pass (the 8 exponent bits) runs over the registers as above; the elements of the chosen binade - about a third
+// of a row of real data - are then copied into shared memory, and the three remaining passes (8, 8 and 7 mantissa
+// bits) walk that list instead of testing every element of the row again.
+// hist: 256 bins; sel: 4 words; cand: room for every key of the row.
+template <class ForEachKey>
+__device__ __forceinline__ Select radix_select_compact(int k, unsigned* hist, unsigned* sel, unsigned* cand, int t,
+                                                       ForEachKey for_each_key) {
+    unsigned prefix = 0, kr = (unsigned)k, eq_total = 0, n_cand = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+        const int bits = pass == 3 ? 7 : 8;
+        const int shift = pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0));
+        hist[t] = 0;
+        if (pass == 0 && t == 0) sel[3] = 0;
+        __syncthreads();
+        if (pass == 0) {
+            for_each_key([&](unsigned u) { atomicAdd(&hist[u >> 23], 1u); });
+        } else {
+            for (unsigned j = t; j < n_cand; j += kBlock) {
+                const unsigned u = cand[j];
+                if ((u >> (shift + bits)) == prefix) atomicAdd(&hist[(u >> shift) & ((1u << bits) - 1u)], 1u);
+            }
+        }
+        __syncthreads();
+        if (t < 32) {
+            // lane l owns bins 255-8l-7 .. 255-8l; lanes ascend as digits descend
+            unsigned h[8], c = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                h[i] = hist[255 - 8 * t - i];
+                c += h[i];
+            }
+            unsigned incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (t >= o) incl += n;
+            }
+            unsigned excl = incl - c;
+            if (incl >= kr && excl < kr) {
+                unsigned cum = excl;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (cum < kr && cum + h[i] >= kr) {
+                        sel[0] = 255 - 8 * t - i;
+                        sel[1] = kr - cum;
+                        sel[2] = h[i];
+                    }
+                    cum += h[i];
+                }
+            }
+        }
+        __syncthreads();
+        prefix = (prefix << bits) | sel[0];
+        kr = sel[1];
+        eq_total = sel[2];
+        if (pass == 0) {
+            // this thread's elements of the chosen binade go to a range of the list reserved with one atomic
+            unsigned mine = 0;
+            for_each_key([&](unsigned u) { mine += (u >> 23) == prefix; });
+            unsigned pos = mine ? atomicAdd(&sel[3], mine) : 0u;
+            for_each_key([&](unsigned u) {
+                if ((u >> 23) == prefix) cand[pos++] = u;
+            });
+            __syncthreads();
+            n_cand = sel[3];
+        }
+    }
+    return Select{prefix, kr, eq_total};
+}
+
 // Exclusive scan of cnt over the TPR threads of a group in thread order; returns
 // the exclusive prefix and the group total.
 template <int TPR>
@@ -251,9 +323,11 @@ __global__ void __launch_bounds__(kBlock, V >= 12 ? 3 : (V >= 8 ? 4 : 6))
     topk_quant_int8_kernel(const float* __restrict__ X, int M, int K, int k, double eps, int8_t* __restrict__ codes,
                            float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
+    constexpr bool ONE_ROW = TPR == kBlock;  // the block owns one row: candidate list in dynamic shared memory
     __shared__ unsigned hist[G][256];
     __shared__ unsigned sel[G][4];
     __shared__ unsigned red[kBlock / 32];
+    extern __shared__ unsigned cand[];  // K words when ONE_ROW
     const int group = threadIdx.x / TPR, t = threadIdx.x % TPR;
     const int row = blockIdx.x * G + group;
     if (row >= M) return;
@@ -274,7 +348,7 @@ __global__ void __launch_bounds__(kBlock, V >= 12 ? 3 : (V >= 8 ? 4 : 6))
     const double gamma = (double)__uint_as_float(gmax);
     const double mult = 127.0 / (gamma + eps);
 
-    Select s = radix_select<TPR>(k, hist[group], sel[group], group, t, [&](auto f) {
+    auto for_each_key = [&](auto f) {
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             if (i * TPR + t < nv) {
@@ -284,7 +358,10 @@ __global__ void __launch_bounds__(kBlock, V >= 12 ? 3 : (V >= 8 ? 4 : 6))
                 f(key(v[i].w));
             }
         }
-    });
+    };
+    Select s;
+    if constexpr (ONE_ROW) s = radix_select_compact(k, hist[0], sel[0], cand, t, for_each_key);
+    else s = radix_select<TPR>(k, hist[group], sel[group], group, t, for_each_key);
     const bool ordered = s.eq_total != s.keep_eq;  // a tie straddles the k-th place: lowest indices win
     unsigned running = 0;
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
@@ -421,9 +498,15 @@ bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k
     const int nv = K / 4;
     const bool fast = (K % 4 == 0) && nv <= 256 * 12;
     const double e = (double)eps;
-#define A48_TK(TPR, V)                                                                                          \
-    topk_quant_int8_kernel<TPR, V><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(X, M, K, k, e, codes, \
-                                                                                              scale, mask_bits)
+#define A48_TK(TPR, V)                                                                                              \
+    do {                                                                                                            \
+        const size_t dyn = TPR == kBlock ? (size_t)K * sizeof(unsigned) : 0; /* candidate list of the one-row kernels */ \
+        if (dyn > 40 * 1024)                                                                                        \
+            cudaFuncSetAttribute(topk_quant_int8_kernel<TPR, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); \
+        topk_quant_int8_kernel<TPR, V><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, dyn, st>>>(X, M, K, k, e,  \
+                                                                                                    codes, scale,   \
+                                                                                                    mask_bits);     \
+    } while (0)
     if (!fast) topk_quant_int8_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, k, e, codes, scale, mask_bits);
     else if (nv <= 32 * 4) A48_TK(32, 4);
     else if (nv <= 64 * 4) A48_TK(64, 4);
