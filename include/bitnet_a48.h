@@ -193,6 +193,12 @@ bitnet_a48_status bitnet_a48_linear_decode_static(const bitnet_a48_weight* w, co
 bitnet_a48_status bitnet_a48_bitlinear_host(const bitnet_a48_weight* w, const float* X_host, int M,
                                             bitnet_a48_act kind, int k, float eps, float* Y_host,
                                             void* workspace_dev, size_t workspace_bytes, void* stream);
+/* The same without the final synchronisation: everything is enqueued on `stream`, Y_host is valid once the
+ * stream has been synchronised.  Calls on different streams (each with its own workspace, page-locked host
+ * buffers) overlap their host-to-device copy, compute and device-to-host copy. */
+bitnet_a48_status bitnet_a48_bitlinear_host_async(const bitnet_a48_weight* w, const float* X_host, int M,
+                                                  bitnet_a48_act kind, int k, float eps, float* Y_host,
+                                                  void* workspace_dev, size_t workspace_bytes, void* stream);
 size_t bitnet_a48_bitlinear_host_workspace_bytes(const bitnet_a48_weight* w, int M);
 
 /* ---------------------------------------------------------------------------

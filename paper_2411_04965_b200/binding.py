@@ -29,7 +29,7 @@ EXPORTS = [
     "bitnet_a48_bitlinear_host", "bitnet_a48_bitlinear_host_workspace_bytes", "bitnet_a48_block_create",
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
-    "bitnet_a48_linear_multi_workspace_bytes",
+    "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
 ]
 
 
@@ -79,6 +79,7 @@ def lib() -> ctypes.CDLL:
                                            c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_bitlinear_host.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_float, c_void_p, c_void_p,
                                                 c_size_t, c_void_p]
+        L.bitnet_a48_bitlinear_host_async.argtypes = L.bitnet_a48_bitlinear_host.argtypes
         L.bitnet_a48_block_create.argtypes = [POINTER(BlockConfig), POINTER(c_void_p), c_void_p, c_void_p,
                                               POINTER(c_void_p)]
         L.bitnet_a48_block_free.argtypes = [c_void_p]
@@ -253,6 +254,16 @@ def bitlinear_host(w: Weight, X_host: torch.Tensor, Y_host: torch.Tensor, kind: 
     _check(lib().bitnet_a48_bitlinear_host(c_void_p(w.handle), _ptr(X_host), M, kind, k, eps, _ptr(Y_host),
                                            _ptr(workspace), workspace.numel() * workspace.element_size(),
                                            _stream(stream)), "bitlinear_host")
+    return Y_host
+
+
+def bitlinear_host_async(w: Weight, X_host: torch.Tensor, Y_host: torch.Tensor, kind: int, k: int, eps: float,
+                         workspace: torch.Tensor, stream=None):
+    """As bitlinear_host, but only enqueues: synchronise the stream before reading Y_host."""
+    assert not X_host.is_cuda and not Y_host.is_cuda and X_host.is_contiguous() and Y_host.is_contiguous()
+    _check(lib().bitnet_a48_bitlinear_host_async(c_void_p(w.handle), _ptr(X_host), X_host.shape[0], kind, k, eps,
+                                                 _ptr(Y_host), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                 _stream(stream)), "bitlinear_host_async")
     return Y_host
 
 

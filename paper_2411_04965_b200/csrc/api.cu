@@ -275,6 +275,16 @@ size_t bitnet_a48_bitlinear_host_workspace_bytes(const bitnet_a48_weight* w, int
 bitnet_a48_status bitnet_a48_bitlinear_host(const bitnet_a48_weight* w, const float* X_host, int M,
                                             bitnet_a48_act kind, int k, float eps, float* Y_host,
                                             void* workspace_dev, size_t workspace_bytes, void* stream) {
+    bitnet_a48_status s = bitnet_a48_bitlinear_host_async(w, X_host, M, kind, k, eps, Y_host, workspace_dev,
+                                                          workspace_bytes, stream);
+    if (s != BITNET_A48_OK) return s;
+    A48_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status bitnet_a48_bitlinear_host_async(const bitnet_a48_weight* w, const float* X_host, int M,
+                                                  bitnet_a48_act kind, int k, float eps, float* Y_host,
+                                                  void* workspace_dev, size_t workspace_bytes, void* stream) {
     if (!w || !X_host || !Y_host || !workspace_dev) return BITNET_A48_ERR_INVALID_ARG;
     if (M <= 0) return BITNET_A48_ERR_SHAPE;
     if (!a48_aligned16(workspace_dev)) return BITNET_A48_ERR_ALIGNMENT;
@@ -298,7 +308,6 @@ bitnet_a48_status bitnet_a48_bitlinear_host(const bitnet_a48_weight* w, const fl
     s = bitnet_a48_linear(w, codes, scale, M, kind, Y, nullptr, base + off[4], workspace_bytes - off[4], stream);
     if (s != BITNET_A48_OK) return s;
     A48_CUDA_TRY(cudaMemcpyAsync(Y_host, Y, (size_t)M * w->N * 4, cudaMemcpyDeviceToHost, st));
-    A48_CUDA_TRY(cudaStreamSynchronize(st));
     return BITNET_A48_OK;
 }
 

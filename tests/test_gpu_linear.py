@@ -45,3 +45,23 @@ def test_linear_simple_matches_oracle(a48, oracle, cuda_dev, M, N, K, kind):
     assert max_rel_err(y.cpu().numpy(), y_ref) <= REL_TOL
     y2 = a48.linear(w, codes, scale, act, a48.ALGO_AUTO)  # whatever AUTO picks must agree bit for bit
     assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("M", [5, 300])
+def test_host_buffer_entry_points_match_the_device_path(a48, cuda_dev, M):
+    # bitnet_a48_bitlinear_host and its asynchronous form: upload, quantise, contract, download
+    N, K = 384, 512
+    w = a48.pack_ternary(synth.latent_weights(N, K, seed=3).to(cuda_dev), EPS, a48.LAYOUT_ALL)
+    x = synth.student_t3(M, K, seed=4)
+    codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+    expected = a48.linear(w, codes, scale, a48.ACT_TOPK_INT8).cpu()
+    ws = torch.zeros(a48.bitlinear_host_workspace_bytes(w, M), dtype=torch.uint8, device=cuda_dev)
+    xp = x.pin_memory()
+    y1 = torch.empty(M, N).pin_memory()
+    a48.bitlinear_host(w, xp, y1, a48.ACT_TOPK_INT8, K // 2, EPS, ws)
+    assert torch.equal(y1, expected)
+    y2 = torch.full((M, N), float("nan")).pin_memory()
+    side = torch.cuda.Stream()
+    a48.bitlinear_host_async(w, xp, y2, a48.ACT_TOPK_INT8, K // 2, EPS, ws, stream=side)
+    side.synchronize()
+    assert torch.equal(y2, expected)
