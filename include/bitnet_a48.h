@@ -97,6 +97,11 @@ bitnet_a48_status bitnet_a48_weight_unpack_layout(const bitnet_a48_weight* w, un
 bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int* K, unsigned* layout_flags);
 /* Bytes of packed weight data a kernel reads for this matrix (N*K/4 rounded up per row). */
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w);
+/* Asks the GPU to pull one packed layout of the matrix (BITNET_A48_LAYOUT_DECODE or _GEMM) into its L2 cache.
+ * A hint with no effect on results: a decode loop calls it on a second stream for the matrix it will need next,
+ * so that the bytes leave HBM while the current BitLinear still runs (at batch 1 a 7B-shape matrix is about
+ * 1.7 us of HBM time but several us of launch and dependency latency).  Enqueues one small kernel on `stream`. */
+bitnet_a48_status bitnet_a48_weight_prefetch(const bitnet_a48_weight* w, unsigned layout, void* stream);
 void bitnet_a48_weight_free(bitnet_a48_weight* w);
 
 /* ---------------------------------------------------------------------------

@@ -124,6 +124,12 @@ bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int
 
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w) { return w ? (size_t)w->N * w->K4 : 0; }
 
+bitnet_a48_status bitnet_a48_weight_prefetch(const bitnet_a48_weight* w, unsigned layout, void* stream) {
+    if (!w) return BITNET_A48_ERR_INVALID_ARG;
+    if (!have_device()) return BITNET_A48_ERR_CUDA;
+    return a48_launch_prefetch(w, layout, (cudaStream_t)stream);
+}
+
 void bitnet_a48_weight_free(bitnet_a48_weight* w) {
     if (!w) return;
     free_weight_buffers(w);

@@ -133,6 +133,7 @@ struct DecodeParams {
     int units;            // ntiles * kchunks
     int grid;             // CTAs
     int tile_aligned;     // pieces end on tile boundaries: no tile is shared, the scratch stays untouched
+    int piece_q, piece_r; // the first piece_r pieces hold piece_q + 1 items (tiles if tile_aligned, else units), the rest piece_q
     int act_row_bytes;    // padded K + 16
 };
 
@@ -142,9 +143,12 @@ __device__ __forceinline__ int matrix_of(const DecodeParams& p, int tile) {
     return j;
 }
 
-// CTA that owns unit u when `units` units are cut into `grid` pieces [c*units/grid, (c+1)*units/grid).
-__device__ __forceinline__ int owner_of(int u, int units, int grid) {
-    return (int)((((long long)u + 1) * grid + units - 1) / units) - 1;
+// First item of piece c when the items are dealt as piece_r pieces of piece_q + 1 followed by pieces of piece_q.
+__device__ __forceinline__ int piece_begin(const DecodeParams& p, int c) { return c * p.piece_q + min(c, p.piece_r); }
+// Piece that owns unit u (stream-K pieces, items = units).
+__device__ __forceinline__ int owner_of(const DecodeParams& p, int u) {
+    const int big = p.piece_r * (p.piece_q + 1);
+    return u < big ? u / (p.piece_q + 1) : p.piece_r + (u - big) / p.piece_q;
 }
 
 // Dynamic shared memory: wbuf [share][512] | act [M][act_row_bytes] | sacc [MAX_TILES][16][TOK] s32 | csum [TOK] s32
@@ -161,11 +165,10 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int u0 = (int)((long long)blockIdx.x * p.units / p.grid), u1 = (int)((long long)(blockIdx.x + 1) * p.units / p.grid);
+    int u0 = piece_begin(p, blockIdx.x), u1 = piece_begin(p, blockIdx.x + 1);  // no divisions on the way to the first copy
     if (p.tile_aligned) {
-        const int ntiles = p.units / p.kchunks;
-        u0 = (int)((long long)blockIdx.x * ntiles / p.grid) * p.kchunks;
-        u1 = (int)((long long)(blockIdx.x + 1) * ntiles / p.grid) * p.kchunks;
+        u0 *= p.kchunks;
+        u1 *= p.kchunks;
     }
     const int share = u1 - u0;
     const int first_tile = u0 / p.kchunks;
@@ -378,7 +381,7 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         const int tb = tile * p.kchunks, te = tb + p.kchunks;
         long long sum = sacc[(tl * 16 + row) * TOK + m];
         if (tb < u0 || te > u1) {  // shared with neighbours
-            const long long contributors = owner_of(te - 1, p.units, p.grid) - owner_of(tb, p.units, p.grid) + 1;
+            const long long contributors = owner_of(p, te - 1) - owner_of(p, tb) + 1;
             unsigned long long* slot = p.ws + ((size_t)tile * 16 + row) * TOK + m;
             const unsigned long long mine = (1ull << 40) | (unsigned long long)(sum + kBias);
             const unsigned long long old = atomicAdd(slot, mine);
@@ -491,6 +494,9 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     const long long aligned_share = ((ntiles + grid - 1) / grid) * p.kchunks;
     p.tile_aligned = grid % sm_count() == 0 && ntiles >= grid && aligned_share <= cap;
     if (p.tile_aligned) share_max = (int)aligned_share;
+    const long long items = p.tile_aligned ? ntiles : (long long)p.units;
+    p.piece_q = (int)(items / grid);
+    p.piece_r = (int)(items % grid);
     const size_t smem = (size_t)share_max * UNIT_BYTES + (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
     if (smem > 227 * 1024 - 64) return BITNET_A48_ERR_UNSUPPORTED;
     static size_t smem_set_dev[64] = {};  // the attribute is per device
@@ -560,4 +566,42 @@ extern "C" bitnet_a48_status bitnet_a48_linear_decode_static(const bitnet_a48_we
     // the array keeps whatever the last call left (zeros, unless a call was cut short): start from zeros
     A48_CUDA_TRY(cudaMemsetAsync(g_static_scratch_ptr[dev], 0, bytes, st));
     return a48_launch_decode(w, codes_dev, scale_dev, M, Y_dev, nullptr, g_static_scratch_ptr[dev], bytes, st);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// L2 prefetch of a packed matrix: lets a decode loop pull the next matrix out of HBM while the current one computes.
+namespace {
+
+constexpr uint32_t kPrefetchChunk = 8192;
+
+__global__ void __launch_bounds__(32) prefetch_l2_kernel(const uint8_t* __restrict__ base, size_t bytes) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x * kPrefetchChunk;
+    for (size_t off = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * kPrefetchChunk; off < bytes; off += stride) {
+        const size_t left = bytes - off;
+        const uint32_t size = (uint32_t)(left < kPrefetchChunk ? left : kPrefetchChunk) & ~15u;  // a multiple of 16 bytes
+        if (size) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(size) : "memory");
+    }
+}
+
+}  // namespace
+
+bitnet_a48_status a48_launch_prefetch(const bitnet_a48_weight* w, unsigned layout, cudaStream_t st) {
+    const uint8_t* base = nullptr;
+    size_t bytes = 0;
+    if (layout == BITNET_A48_LAYOUT_DECODE && w->decode) {
+        base = w->decode;
+        bytes = (size_t)((w->N + 15) / 16) * (w->Kp / 128) * UNIT_BYTES;  // the tiles that hold real rows
+    } else if (layout == BITNET_A48_LAYOUT_GEMM && w->gemm) {
+        base = w->gemm;
+        bytes = (size_t)w->Np * w->Kp / 4;
+    } else {
+        return BITNET_A48_ERR_UNSUPPORTED;
+    }
+    const size_t chunks = (bytes + kPrefetchChunk - 1) / kPrefetchChunk;
+    unsigned blocks = (unsigned)((chunks + 31) / 32);
+    if (blocks > (unsigned)sm_count()) blocks = (unsigned)sm_count();
+    if (blocks == 0) return BITNET_A48_OK;
+    prefetch_l2_kernel<<<blocks, 32, 0, st>>>(base, bytes);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
 }
