@@ -181,7 +181,43 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int cg = WARPS * ((p.kchunks + WARPS * MAX_GROUPS - 1) / (WARPS * MAX_GROUPS));
     const int ngroups = (p.kchunks + cg - 1) / cg;
-    {
+    // Pieces of one to six whole tiles (the usual case at model shapes) run code compiled for their tile count,
+    // with the per-tile addresses in registers: a copy or a fragment load then costs one multiply-add.
+    const bool whole = p.tile_aligned && ntl >= 1 && ntl <= NTL;
+    auto for_tile_count = [&](auto f) {
+        switch (ntl) {
+            case 1: f(std::integral_constant<int, 1>{}); break;
+            case 2: f(std::integral_constant<int, 2>{}); break;
+            case 3: f(std::integral_constant<int, 3>{}); break;
+            case 4: f(std::integral_constant<int, 4>{}); break;
+            case 5: f(std::integral_constant<int, 5>{}); break;
+            default: f(std::integral_constant<int, 6>{}); break;
+        }
+    };
+    if (whole) {
+        for_tile_count([&](auto nt_c) {
+            constexpr int NT = decltype(nt_c)::value;
+            const uint8_t* src[NT];
+            uint32_t dst[NT];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) {
+                const int tile = first_tile + t, j = matrix_of(p, tile);
+                src[t] = p.wdec[j] + lane * 16 + (size_t)(tile - p.tile_base[j]) * p.kchunks * UNIT_BYTES;
+                dst[t] = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16 + (uint32_t)(t * p.kchunks) * UNIT_BYTES;
+            }
+            for (int gq = 0; gq < ngroups; ++gq) {
+                const int c_hi = min(gq * cg + cg, p.kchunks);
+                for (int kc = gq * cg + warp; kc < c_hi; kc += WARPS) {
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst[t] + (uint32_t)kc * UNIT_BYTES),
+                                     "l"(src[t] + (size_t)kc * UNIT_BYTES)
+                                     : "memory");
+                }
+                cp_async_commit();
+            }
+        });
+    } else {
         // a warp takes whole units (lane l the l-th 16 bytes of each), so that one cp.async instruction moves 512
         // contiguous bytes and the only arithmetic per copy is the unit index
         const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16 - (uint32_t)u0 * UNIT_BYTES;
@@ -234,6 +270,60 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         // sums of slice q carry the factor 4^q, which an exact shift removes at the end.  Rows g (words 0, 2) and
         // g+8 (words 1, 3); the four lanes of a quad hold different channels of the same rows.
         int xsum = 0;
+        if (whole) {
+            for_tile_count([&](auto nt_c) {
+                constexpr int NT = decltype(nt_c)::value;
+                int lo[NT][4], hi[NT][4];
+#pragma unroll
+                for (int t = 0; t < NT; ++t)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) lo[t][q] = hi[t][q] = 0;
+                const uint8_t* a0 = wbuf + lane * 16;
+                const uint32_t tile_bytes = (uint32_t)p.kchunks * UNIT_BYTES;
+                for (int gq = 0; gq < ngroups; ++gq) {
+                    cp_async_wait(ngroups - 1 - gq);  // group gq has landed for every thread
+                    __syncthreads();
+                    const int c_hi = min(gq * cg + cg, p.kchunks);
+                    for (int kc = gq * cg + warp; kc < c_hi; kc += WARPS) {
+                        int b[4][2];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            b[q][0] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + tig * 4);
+                            b[q][1] = *reinterpret_cast<const int*>(act + kc * 128 + q * 32 + 16 + tig * 4);
+                            xsum = __dp4a(b[q][1], 0x01010101, __dp4a(b[q][0], 0x01010101, xsum));
+                        }
+                        uint4 a[NT];
+#pragma unroll
+                        for (int t = 0; t < NT; ++t)
+                            a[t] = *reinterpret_cast<const uint4*>(a0 + t * tile_bytes + (uint32_t)kc * UNIT_BYTES);
+#pragma unroll
+                        for (int t = 0; t < NT; ++t) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const uint32_t mq = 0x03030303u << (2 * q);
+                                lo[t][q] = dp4a_u8s8(a[t].x & mq, b[q][0], lo[t][q]);
+                                lo[t][q] = dp4a_u8s8(a[t].z & mq, b[q][1], lo[t][q]);
+                                hi[t][q] = dp4a_u8s8(a[t].y & mq, b[q][0], hi[t][q]);
+                                hi[t][q] = dp4a_u8s8(a[t].w & mq, b[q][1], hi[t][q]);
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    int r0 = lo[t][0] + (lo[t][1] >> 2) + (lo[t][2] >> 4) + (lo[t][3] >> 6);
+                    int r1 = hi[t][0] + (hi[t][1] >> 2) + (hi[t][2] >> 4) + (hi[t][3] >> 6);
+                    r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                    r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                    r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
+                    r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
+                    if (tig == 0) {
+                        atomicAdd(sacc + ((size_t)t * 16 + g) * TOK, r0);
+                        atomicAdd(sacc + ((size_t)t * 16 + g + 8) * TOK, r1);
+                    }
+                }
+            });
+        } else {
         // the walk is compiled for 3, 4, 5 and 6 tiles side by side: blank slots would cost as much as real ones
         auto walk = [&](auto nt_c) {
             constexpr int NT = decltype(nt_c)::value;
@@ -301,6 +391,7 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         else if (ntl == 4) walk(std::integral_constant<int, 4>{});
         else if (ntl == 5) walk(std::integral_constant<int, 5>{});
         else walk(std::integral_constant<int, NTL>{});
+        }
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         if (lane == 0) atomicAdd(csum, xsum);
