@@ -229,7 +229,7 @@ size_t bitnet_a48_linear_multi_workspace_bytes(int count, const bitnet_a48_weigh
     if (fused) return fused;
     size_t single = 0;  // one call after the other: the largest single requirement
     for (int j = 0; j < count; ++j) {
-        size_t b = a48_decode_workspace_bytes(weights[j], M);
+        size_t b = bitnet_a48_linear_workspace_bytes(weights[j], M);
         single = b > single ? b : single;
     }
     return single;
@@ -268,7 +268,7 @@ static size_t host_ws_layout(const bitnet_a48_weight* w, int M, size_t off[5]) {
     off[1] = o; o += up((size_t)M * w->K);
     off[2] = o; o += up((size_t)M * 4);
     off[3] = o; o += up((size_t)M * w->N * 4);
-    off[4] = o; o += up(a48_decode_workspace_bytes(w, M));
+    off[4] = o; o += up(bitnet_a48_linear_workspace_bytes(w, M));
     return o;
 }
 
@@ -309,7 +309,7 @@ bitnet_a48_status bitnet_a48_bitlinear_host_async(const bitnet_a48_weight* w, co
     else if (kind == BITNET_A48_ACT_FP4) s = bitnet_a48_quant_fp4(X, M, w->K, codes, scale, stream);
     else return BITNET_A48_ERR_INVALID_ARG;
     if (s != BITNET_A48_OK) return s;
-    const size_t lin_bytes = a48_decode_workspace_bytes(w, M);
+    const size_t lin_bytes = bitnet_a48_linear_workspace_bytes(w, M);
     if (lin_bytes) A48_CUDA_TRY(cudaMemsetAsync(base + off[4], 0, lin_bytes, st));
     s = bitnet_a48_linear(w, codes, scale, M, kind, Y, nullptr, base + off[4], workspace_bytes - off[4], stream);
     if (s != BITNET_A48_OK) return s;

@@ -33,7 +33,7 @@ BlockWs block_ws(const bitnet_a48_block* blk, int B, int T) {
     w.vc = take(M * H * 4);
     size_t lin = 0;
     for (int i = 0; i < 7; ++i) {
-        size_t b = a48_decode_workspace_bytes(blk->w[i], (int)M);
+        size_t b = bitnet_a48_linear_workspace_bytes(blk->w[i], (int)M);
         lin = b > lin ? b : lin;
     }
     {  // q,k,v and gate,up go out as one call each

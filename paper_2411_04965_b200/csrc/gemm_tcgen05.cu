@@ -45,28 +45,37 @@
 namespace {
 
 constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
-constexpr int TILE_M = 192;  // tokens per tile       (MMA N)
+constexpr int TILE_M_WIDE = 192;   // tokens per tile (MMA N) of the prefill kernel
+constexpr int TILE_M_SKINNY = 64;  // ... and of the kernel for at most 64 tokens
 constexpr int BK = 128;      // channels per 128-byte swizzle row of int8
 constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
-constexpr int A_SLOTS = 2;   // tensor-memory slots of the expanded weight operand
-constexpr int ACC_COLS = TILE_M;
 constexpr int ACC_BUFS = 2;
 constexpr int TMEM_COLS = 512;
-constexpr int B_TILE_BYTES = TILE_M * BK;
 constexpr int A_TILE_BYTES = TILE_N * BK;
 constexpr int W_PACKED_BYTES = TILE_N * BK / 4;  // 128 rows x 128 channels of 2-bit codes
-constexpr int EXPAND_GROUPS = 2;
-constexpr int EPI_SPLIT = 2;  // epilogue warps per lane quadrant
-constexpr int EPI_COLS = TILE_M / EPI_SPLIT;
-static_assert(EPI_COLS % 32 == 0, "the epilogue drains 32 columns at a time");
-constexpr int NUM_THREADS = 32 * (2 + 4 * EXPAND_GROUPS + 4 * EPI_SPLIT);
-static_assert(A_SLOTS == EXPAND_GROUPS, "expander group g owns slot g");
+constexpr int kMaxSplit = 8;  // CTAs that may share a tile's channels: the portable cluster size
 constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
 
-template <bool TS>
+template <bool TS, int TM>
 struct Cfg {
+    static constexpr int TILE_M = TM;
+    static constexpr int ACC_COLS = TM;
+    static constexpr int B_TILE_BYTES = TM * BK;
+    // Expander groups of four warps (TS).  A group spends about 740 clocks on a unit; at 64 tokens the kernel is
+    // bound by the fill rate of shared memory (24 KB per unit and CTA), so two groups are enough there too.
+    static constexpr int EXPAND_GROUPS = 2;
+    static constexpr int EPI_SPLIT = 2;  // epilogue warps per lane quadrant
+    static constexpr int NUM_THREADS = 32 * (2 + 4 * EXPAND_GROUPS + 4 * EPI_SPLIT);
+    static constexpr int EPI_COLS = TM / EPI_SPLIT;
+    static_assert(EPI_COLS % 32 == 0, "the epilogue drains 32 columns at a time");
     static constexpr int KBU = TS ? 2 : 1;  // 128-channel blocks per pipeline stage
-    static constexpr int STAGES = TS ? 4 : 5;
+    // the narrow activation tile leaves room for a deeper ring: more weight bytes in flight per SM
+    static constexpr int STAGES = TM == TILE_M_SKINNY ? 8 : (TS ? 4 : 5);
+    // Tensor-memory slots of the expanded weight operand, 64 columns each.  A slot is busy from the expanders'
+    // store until the MMAs that read it have completed, a round trip of well over a thousand clocks whatever
+    // the MMA's size; two slots leave that round trip exposed, the narrow accumulators make room for more.
+    static constexpr int A_SLOTS = TM == TILE_M_SKINNY ? 6 : 2;
+    static_assert(A_SLOTS % EXPAND_GROUPS == 0, "unit it goes to group it % groups and to slot it % slots");
     static constexpr int STAGE_BYTES = KBU * (B_TILE_BYTES + (TS ? W_PACKED_BYTES : A_TILE_BYTES));
     static constexpr int A_SLOT_COLS = KBU * BK / 4;
     // a stage is released by the MMA commit and, for TS, by one lane of each expander warp of one group
@@ -74,7 +83,8 @@ struct Cfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 1024 /*barriers*/;
     static_assert(ACC_BUFS * ACC_COLS + (TS ? A_SLOTS * A_SLOT_COLS : 0) <= TMEM_COLS, "tensor memory budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-    static_assert(STAGES > A_SLOTS, "the stage two units back must still be distinct");
+    static_assert(STAGES * STAGE_BYTES >= (TM + kMaxSplit) * TILE_N * 4, "split-K: ksplit slots of ceil(TM / ksplit) token rows");
+    static_assert(STAGES > A_SLOTS, "the stage A_SLOTS units back must still be distinct");
 };
 
 __device__ unsigned int g_status[4];
@@ -257,18 +267,43 @@ struct GemmParams {
     int32_t* acc;         // [M, N] or nullptr
     int M, N, K;
     int kblocks, n_tiles, m_tiles;
+    // Split-K (few tiles, many SMs): the channels of a tile are cut into ksplit ranges, one CTA each, and the
+    // ksplit CTAs of a tile form one thread-block cluster (cluster rank = range).  Rank o owns a 1/ksplit share
+    // of the tile's tokens: once every CTA of the cluster has its accumulator complete (first cluster barrier,
+    // after which nobody's pipeline stages are in use), each CTA stores its int32 partial sums for o's tokens
+    // into slot `own rank` of a buffer in o's shared memory (distributed shared memory, stores only); after the
+    // second barrier o adds the ksplit slots and writes those rows of Y.
+    int ksplit;
 };
 
-template <bool TS>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// Channel range, in pipeline units, of part `part` out of `ksplit` (balanced to within one unit).
+__device__ __forceinline__ int unit_begin(int part, int ksplit, int kunits) { return (int)((long long)part * kunits / ksplit); }
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address, in the cluster's shared window, of this CTA's shared-memory address `addr` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_s32(uint32_t cluster_addr, int v) {
+    asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
+template <bool TS, int TM>
+__global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
     gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                         const GemmParams p) {
-    using C = Cfg<TS>;
-    constexpr int STAGES = C::STAGES, KBU = C::KBU;
+    using C = Cfg<TS, TM>;
+    constexpr int STAGES = C::STAGES, KBU = C::KBU, TILE_M = C::TILE_M, ACC_COLS = C::ACC_COLS, A_SLOTS = C::A_SLOTS;
+    constexpr int EXPAND_GROUPS = C::EXPAND_GROUPS, EPI_SPLIT = C::EPI_SPLIT;
+    constexpr int B_TILE_BYTES = C::B_TILE_BYTES, EPI_COLS = C::EPI_COLS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ctrl = smem + STAGES * C::STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] acc_full[2] acc_empty[2]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] acc_full[2] acc_empty[2] epi
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 512);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 516);
 
@@ -279,6 +314,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
+        // start fetching the tensor-map descriptors now: the first tensor copy otherwise waits for them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
+        if (!TS) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, C::EMPTY_ARRIVALS);
@@ -304,26 +342,30 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     const uint32_t tmem_acc = tmem_base;
     const uint32_t tmem_a = tmem_base + ACC_BUFS * ACC_COLS;
     const int total_tiles = p.n_tiles * p.m_tiles;
+    const int total_items = total_tiles * p.ksplit;  // item = tile * ksplit + part; split: one item per CTA
     const int kunits = p.kblocks / KBU;  // the packed layouts pad K so that this is exact
+    int cluster_syncs = 0;               // cluster barriers this thread has passed (split-K)
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t it = 0, s = 0, ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+                const int tile = item / p.ksplit, part = item - tile * p.ksplit;
+                const int u_begin = unit_begin(part, p.ksplit, kunits), u_end = unit_begin(part + 1, p.ksplit, kunits);
                 const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
                 const uint8_t* wtile = p.wt + (size_t)(tile % p.n_tiles) * p.kblocks * W_PACKED_BYTES;
-                for (int u = 0; u < kunits; ++u, ++it) {
+                for (int u = u_begin; u < u_end; ++u, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
                     const uint32_t dst = smem_base + s * C::STAGE_BYTES, bar = bar_full + 8 * s;
                     mbar_expect_tx(bar, C::STAGE_BYTES);
-#pragma unroll
-                    for (int h = 0; h < KBU; ++h) tma_load_2d(dst + h * B_TILE_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
-                    if (TS) {
+                    if (TS)  // the weights first: they come from HBM, the activation tile mostly from L2
                         bulk_load(dst + KBU * B_TILE_BYTES, wtile + (size_t)u * KBU * W_PACKED_BYTES, KBU * W_PACKED_BYTES,
                                   bar);
-                    } else {
+#pragma unroll
+                    for (int h = 0; h < KBU; ++h) tma_load_2d(dst + h * B_TILE_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
+                    if (!TS) {
 #pragma unroll
                         for (int h = 0; h < KBU; ++h)
                             tma_load_2d(dst + KBU * B_TILE_BYTES + h * A_TILE_BYTES, &tm_w, (u * KBU + h) * BK, n0, bar);
@@ -352,13 +394,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         uint32_t it = 0, tcount = 0;
         uint32_t s = 0, ph = 0;  // stage ring position and phase, advanced without divisions
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++tcount) {
+            const int part = item % p.ksplit;
+            const int u_begin = unit_begin(part, p.ksplit, kunits), u_end = unit_begin(part + 1, p.ksplit, kunits);
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
             const uint32_t d_tmem = tmem_acc + ab * ACC_COLS;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8 * ab, pab ^ 1, abort_flag, 2, tcount));
             if (!ok) break;
             tc_fence_after();
-            for (int u = 0; u < kunits; ++u, ++it) {
+            for (int u = u_begin; u < u_end; ++u, ++it) {
                 const uint32_t slot = it % A_SLOTS, pslot = (it / A_SLOTS) & 1;
                 const uint32_t bar_in = TS ? bar_afull + 8 * slot : bar_full + 8 * s;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_in, TS ? pslot : ph, abort_flag, TS ? 4 : 3, it));
@@ -375,14 +419,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                             const uint32_t a_t = tmem_a + slot * C::A_SLOT_COLS + h * (BK / 4);
 #pragma unroll
                             for (int j = 0; j < BK / UMMA_K; ++j) {
-                                if (h == 0 && j == 0 && u == 0) mma_ts(d_tmem, a_t, b_desc, idesc, 0u);
+                                if (h == 0 && j == 0 && u == u_begin) mma_ts(d_tmem, a_t, b_desc, idesc, 0u);
                                 else mma_ts_acc(d_tmem, a_t + j * (UMMA_K / 4), b_lo + 2 * j, b_hi, idesc);
                             }
                         } else {
                             const uint64_t a_desc = smem_desc_sw128(b_addr + KBU * B_TILE_BYTES + h * A_TILE_BYTES);
 #pragma unroll
                             for (int j = 0; j < BK / UMMA_K; ++j)
-                                mma_ss(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (u > 0 || h > 0 || j > 0) ? 1u : 0u);
+                                mma_ss(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (u > u_begin || h > 0 || j > 0) ? 1u : 0u);
                         }
                     }
                     tc_commit(bar_empty + 8 * s);
@@ -398,13 +442,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         if (TS) {
             const int quad = warp & 3;            // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
             const int row = quad * 32 + lane;     // weight row inside the tile = TMEM lane
-            const uint32_t group = (uint32_t)(warp - 2) >> 2;  // takes the units with it % groups == group; owns slot `group`
-            const uint32_t a_dst = tmem_a + ((uint32_t)(quad * 32) << 16) + group * C::A_SLOT_COLS;
-            const long long total_units = (long long)kunits * ((total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x);
+            const uint32_t group = (uint32_t)(warp - 2) >> 2;  // takes the units with it % groups == group
+            const uint32_t a_lanes = tmem_a + ((uint32_t)(quad * 32) << 16);
+            long long total_units = 0;  // units of all items of this CTA
+            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+                const int part = item % p.ksplit;
+                total_units += unit_begin(part + 1, p.ksplit, kunits) - unit_begin(part, p.ksplit, kunits);
+            }
             bool ok = true;
             for (long long it64 = group; it64 < total_units && ok; it64 += EXPAND_GROUPS) {
                 const uint32_t it = (uint32_t)it64;
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1, slot = it % A_SLOTS;
+                const uint32_t a_dst = a_lanes + slot * C::A_SLOT_COLS;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag, 7, it));
                 if (!ok) break;
                 const uint4* src = reinterpret_cast<const uint4*>(smem + s * C::STAGE_BYTES + KBU * B_TILE_BYTES);
@@ -424,7 +473,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                 __syncwarp();  // every lane has consumed its packed words: the stage's weight bytes are free
                 if (lane == 0) mbar_arrive(bar_empty + 8 * s);
                 if (it >= (uint32_t)A_SLOTS) {
-                    // slot `group` was last read by the MMAs of unit it - A_SLOTS; their commit completes that stage's empty phase
+                    // the slot was last read by the MMAs of unit it - A_SLOTS; their commit completes that stage's empty phase
                     const uint32_t j = it - A_SLOTS, sj = j % STAGES, pj = (j / STAGES) & 1;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * sj, pj, abort_flag, 5, it));
                     if (!ok) break;
@@ -434,7 +483,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                 for (int h = 0; h < KBU; ++h) tmem_st32(a_dst + h * (BK / 4), v[h]);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
-                mbar_arrive(bar_afull + 8 * group);
+                mbar_arrive(bar_afull + 8 * slot);
             }
         }
     } else {
@@ -444,12 +493,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         const float alpha = *p.alpha;
         uint32_t tcount = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++tcount) {
+            const int tile = item / p.ksplit;
             const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, pab, abort_flag, 6, tcount));
             if (!ok) break;
             tc_fence_after();
+            if (p.ksplit > 1) {
+                cluster_sync_all();  // every CTA of the cluster is past its last MMA: stage memory is free everywhere
+                ++cluster_syncs;
+            }
             const int n = n0 + quad * 32 + lane;
             const bool n_ok = n < p.N;
 #pragma unroll 1
@@ -459,32 +513,77 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                 const int mrow = m0 + c0;
                 const int valid = p.M - mrow;  // tokens of this chunk that exist
                 const size_t o = (size_t)mrow * p.N + n;
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (!n_ok) continue;
+                if (p.ksplit > 1) {
+                    // token c of the tile belongs to rank c / per, row c % per; this CTA writes slot `part`
+                    const int tokens = min(TILE_M, p.M - m0), per = (tokens + p.ksplit - 1) / p.ksplit;
+                    const int part = item - tile * p.ksplit;
+                    int owner = c0 / per, row = c0 - owner * per;
+                    const uint32_t slot_addr = smem_base + (uint32_t)((part * per) * TILE_N + quad * 32 + lane) * 4u;
+                    uint32_t dst = map_to_rank(slot_addr, (uint32_t)min(owner, p.ksplit - 1));
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < valid) st_cluster_s32(dst + (uint32_t)(row * TILE_N) * 4u, (int)r[j]);
+                        if (++row == per) {
+                            row = 0;
+                            ++owner;
+                            dst = map_to_rank(slot_addr, (uint32_t)min(owner, p.ksplit - 1));
+                        }
+                    }
+                    continue;
+                }
                 float* yp = p.Y + o;
                 const float* sp = p.scale + mrow;
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (n_ok) {
-                    // y = fp32(acc) * (scale[m] * alpha): the prefactors of Eq. 2, 3 and 7
-                    if (valid >= 32) {
+                // y = fp32(acc) * (scale[m] * alpha): the prefactors of Eq. 2, 3 and 7
+                if (valid >= 32) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
-                            yp += p.N;
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < valid) yp[(size_t)j * p.N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                    for (int j = 0; j < 32; ++j) {
+                        *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                        yp += p.N;
                     }
-                    if (p.acc) {
-                        int32_t* ap = p.acc + o;
+                } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < valid) ap[(size_t)j * p.N] = (int)r[j];
-                    }
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) yp[(size_t)j * p.N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                }
+                if (p.acc) {
+                    int32_t* ap = p.acc + o;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) ap[(size_t)j * p.N] = (int)r[j];
                 }
             }
             tc_fence_before();
             mbar_arrive(bar_acc_empty + 8 * ab);
+        }
+    }
+    if (p.ksplit > 1) {
+        // Every thread of every CTA of the cluster passes exactly two cluster barriers, also after an abort.  The
+        // epilogue warps took the first one as soon as their accumulator was complete.
+        __syncwarp();
+        for (; cluster_syncs < 2; ++cluster_syncs) cluster_sync_all();
+        const int te = (int)threadIdx.x - 32 * (2 + 4 * EXPAND_GROUPS);  // index among the epilogue threads
+        if (te >= 0 && !*abort_flag) {
+            const int tile = (int)blockIdx.x / p.ksplit, rank = (int)blockIdx.x - tile * p.ksplit;
+            const int m0 = (tile / p.n_tiles) * TILE_M, nl = te & (TILE_N - 1), n = (tile % p.n_tiles) * TILE_N + nl;
+            const int tokens = min(TILE_M, p.M - m0);
+            const int per = (tokens + p.ksplit - 1) / p.ksplit;  // tokens owned by each rank
+            const int rows = min(per, tokens - rank * per);      // ... and by this one (may be <= 0)
+            const float alpha = *p.alpha;
+            const int* slots = reinterpret_cast<const int*>(smem);
+            if (n < p.N) {
+                for (int row = te >> 7; row < rows; row += 128 * EPI_SPLIT / TILE_N) {
+                    int sum = 0;
+#pragma unroll
+                    for (int q = 0; q < kMaxSplit; ++q)
+                        if (q < p.ksplit) sum += slots[(q * per + row) * TILE_N + nl];
+                    const int m = m0 + rank * per + row;
+                    const size_t e = (size_t)m * p.N + n;
+                    p.Y[e] = (float)sum * (__ldg(p.scale + m) * alpha);
+                    if (p.acc) p.acc[e] = sum;
+                }
+            }
         }
     }
     tc_fence_before();
@@ -534,23 +633,83 @@ int sm_count() {
     return c;
 }
 
-template <bool TS>
+// How a call is cut into work items.  With fewer tiles than SMs the channels of a tile are split over `ksplit`
+// CTAs (one cluster); the cost of a split, in pipeline units per CTA, is rounds * (units per item + a fixed
+// per-item charge for filling the pipeline and for the reduction through distributed shared memory).
+struct Plan {
+    int tile_m, n_tiles, m_tiles, ksplit;
+};
+
+Plan make_plan(const bitnet_a48_weight* w, int M, bool ts) {
+    Plan pl;
+    pl.tile_m = M <= TILE_M_SKINNY ? TILE_M_SKINNY : TILE_M_WIDE;
+    pl.n_tiles = (w->N + TILE_N - 1) / TILE_N;
+    pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
+    const int tiles = pl.n_tiles * pl.m_tiles, sms = sm_count();
+    const int kunits = w->Kp / BK / (ts ? 2 : 1);
+    constexpr int kItemCharge = 3;
+    pl.ksplit = 1;
+    long long best = (long long)((tiles + sms - 1) / sms) * (kunits + kItemCharge);
+    for (int ks = 2; ks <= kMaxSplit && ks <= kunits && tiles < sms; ++ks) {
+        const int slots = sms / ks * ks;  // whole clusters only
+        const long long rounds = ((long long)tiles * ks + slots - 1) / slots;
+        const long long cost = rounds * ((kunits + ks - 1) / ks + kItemCharge + 1);
+        if (cost * 10 < best * 9) {  // a split has to pay for itself by a clear margin
+            best = cost;
+            pl.ksplit = ks;
+        }
+    }
+    return pl;
+}
+
+template <bool TS, int TM>
 bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
-                         int32_t* acc, cudaStream_t st) {
-    static bool attr_set[64] = {};  // the attribute is per device
+                         int32_t* acc, Plan pl, cudaStream_t st) {
+    using C = Cfg<TS, TM>;
+    static bool attr_set[64] = {};        // the attribute is per device
+    static signed char cluster_ok[64][kMaxSplit + 1] = {};  // 0 unknown, 1 the device can host such a cluster, -1 it cannot
     int dev = 0;
     A48_CUDA_TRY(cudaGetDevice(&dev));
-    if (!attr_set[dev & 63]) {
-        A48_CUDA_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<TS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          Cfg<TS>::SMEM_BYTES));
-        attr_set[dev & 63] = true;
+    dev &= 63;
+    if (!attr_set[dev]) {
+        A48_CUDA_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<TS, TM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          C::SMEM_BYTES));
+        attr_set[dev] = true;
     }
     CUtensorMap tm_act, tm_w;
-    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TILE_M)) return BITNET_A48_ERR_CUDA;
+    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TM)) return BITNET_A48_ERR_CUDA;
     if (TS) {
         tm_w = tm_act;  // unused
     } else if (!make_map(&tm_w, w->i8, (uint64_t)w->Np, (uint64_t)w->Kp, (uint64_t)w->Kp, TILE_N)) {
         return BITNET_A48_ERR_CUDA;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(C::NUM_THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pl.ksplit > 1) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)pl.ksplit;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cfg.gridDim = dim3((unsigned)(pl.n_tiles * pl.m_tiles * pl.ksplit));
+        signed char& okc = cluster_ok[dev][pl.ksplit];
+        if (okc == 0) {
+            int clusters = 0;
+            okc = cudaOccupancyMaxActiveClusters(&clusters, gemm_tcgen05_kernel<TS, TM>, &cfg) == cudaSuccess &&
+                          clusters >= 1
+                      ? 1
+                      : -1;
+            if (okc < 0) (void)cudaGetLastError();
+        }
+        if (okc < 0) {  // whole tiles instead
+            pl.ksplit = 1;
+            cfg.attrs = nullptr;
+            cfg.numAttrs = 0;
+        }
     }
     GemmParams p;
     p.wt = w->gemm;
@@ -562,12 +721,14 @@ bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const 
     p.N = w->N;
     p.K = w->K;
     p.kblocks = w->Kp / BK;
-    p.n_tiles = (w->N + TILE_N - 1) / TILE_N;
-    p.m_tiles = (M + TILE_M - 1) / TILE_M;
-    const int total = p.n_tiles * p.m_tiles;
-    const int grid = total < sm_count() ? total : sm_count();
-    gemm_tcgen05_kernel<TS><<<grid, NUM_THREADS, Cfg<TS>::SMEM_BYTES, st>>>(tm_act, tm_w, p);
-    A48_CUDA_TRY(cudaGetLastError());
+    p.n_tiles = pl.n_tiles;
+    p.m_tiles = pl.m_tiles;
+    p.ksplit = pl.ksplit;
+    if (pl.ksplit == 1) {
+        const int total = p.n_tiles * p.m_tiles;
+        cfg.gridDim = dim3((unsigned)(total < sm_count() ? total : sm_count()));
+    }
+    A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TS, TM>, tm_act, tm_w, p));
     return BITNET_A48_OK;
 }
 
@@ -580,7 +741,12 @@ bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss) {
 
 bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                           float* Y, int32_t* acc, bool ss, cudaStream_t st) {
-    return ss ? launch<false>(w, codes, scale, M, Y, acc, st) : launch<true>(w, codes, scale, M, Y, acc, st);
+    const Plan pl = make_plan(w, M, !ss);
+    if (pl.tile_m == TILE_M_SKINNY)
+        return ss ? launch<false, TILE_M_SKINNY>(w, codes, scale, M, Y, acc, pl, st)
+                  : launch<true, TILE_M_SKINNY>(w, codes, scale, M, Y, acc, pl, st);
+    return ss ? launch<false, TILE_M_WIDE>(w, codes, scale, M, Y, acc, pl, st)
+              : launch<true, TILE_M_WIDE>(w, codes, scale, M, Y, acc, pl, st);
 }
 
 bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]) {

@@ -87,3 +87,30 @@ def test_gemm_full_size_sampled(a48, oracle, cuda_dev):
     codes_h, scale_h = codes.cpu().numpy(), scale.cpu().numpy().astype(np.float64)
     acc_c, _ = oracle.linear(codes_h, scale_h, t_ref[cols.cpu().numpy()], a_ref, nthreads=8, want_y=False)
     assert np.array_equal(acc[:, cols].cpu().numpy().astype(np.int64), acc_c)
+
+
+# Few tokens: the 64-token tile and the split of a tile's channels over the CTAs of a cluster.  (M, N, K) cover one and
+# several weight-row tiles, a ragged N tail, K = 3200 / 8640 (padded to whole pipeline units), M around the
+# 64-token boundary and a two-tile M of the wide kernel.
+SKINNY = [(9, 128, 512), (16, 384, 2048), (33, 200, 3200), (64, 1024, 8640), (65, 256, 2048), (100, 640, 4096),
+          (191, 130, 1536), (40, 3200, 3200)]
+
+
+@pytest.mark.parametrize("M,N,K", SKINNY)
+@pytest.mark.parametrize("variant", ["tmem", "smem_i8"])
+def test_gemm_few_tokens_split_k(a48, oracle, cuda_dev, M, N, K, variant):
+    W = synth.latent_weights(N, K, seed=N + K + 1)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_GEMM | a48.LAYOUT_I8)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    x = synth.student_t3(M, K, seed=M + 7)
+    codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+    c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS, nthreads=8)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    algo = _algos(a48)[variant]
+    for _ in range(2):
+        y, acc = a48.linear(w, codes, scale, a48.ACT_TOPK_INT8, algo, want_acc=True)
+        torch.cuda.synchronize()
+        assert a48.kernel_status() == [0, 0, 0, 0]
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
