@@ -252,6 +252,12 @@ bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* co
     if (count <= 4 && a48_decode_multi_workspace_bytes(count, weights, M) > 0)
         return a48_launch_decode_multi(count, weights, codes_dev, scale_dev, M, Y_dev, nullptr, workspace_dev,
                                        workspace_bytes, (cudaStream_t)stream);
+    {  // beyond the decode kernel's token count: one tensor-core launch over the tiles of all matrices
+        bool any_decode = false;
+        for (int j = 0; j < count; ++j) any_decode = any_decode || a48_decode_supported(weights[j], M);
+        if (!any_decode && a48_gemm_tcgen05_multi_supported(count, weights, M))
+            return a48_launch_gemm_tcgen05_multi(count, weights, codes_dev, scale_dev, M, Y_dev, (cudaStream_t)stream);
+    }
     for (int j = 0; j < count; ++j) {
         bitnet_a48_status s = bitnet_a48_linear(weights[j], codes_dev, scale_dev, M, kind, Y_dev[j], nullptr, workspace_dev,
                                                 workspace_bytes, stream);

@@ -259,14 +259,20 @@ __device__ __forceinline__ void expand_word(uint32_t p, uint32_t* out) {
     out[3] = prmt(kTable, r >> 16);
 }
 
+constexpr int MAX_MATS = 4;  // weight matrices (one K, one set of codes) that one launch can take
+
 struct GemmParams {
-    const uint8_t* wt;    // tile-major packed weights (TS)
+    // Matrix j of the launch owns the weight-row tiles tile_base[j] .. tile_base[j+1]-1 of every token tile.
+    const uint8_t* wt[MAX_MATS];   // tile-major packed weights (TS)
+    const float* alpha[MAX_MATS];  // device scalars
+    float* Y[MAX_MATS];            // [M, N_j]
+    int N[MAX_MATS];
+    int tile_base[MAX_MATS + 1];
+    int count;
     const float* scale;   // [M]
-    const float* alpha;   // device scalar
-    float* Y;             // [M, N]
-    int32_t* acc;         // [M, N] or nullptr
-    int M, N, K;
-    int kblocks, n_tiles, m_tiles;
+    int32_t* acc;         // [M, N_0] or nullptr (single-matrix launches only)
+    int M, K;
+    int kblocks, n_tiles /* all matrices together */, m_tiles;
     // Split-K (few tiles, many SMs): the channels of a tile are cut into ksplit ranges, one CTA each, and the
     // ksplit CTAs of a tile form one thread-block cluster (cluster rank = range).  Rank o owns a 1/ksplit share
     // of the tile's tokens: once every CTA of the cluster has its accumulator complete (first cluster barrier,
@@ -275,6 +281,13 @@ struct GemmParams {
     // second barrier o adds the ksplit slots and writes those rows of Y.
     int ksplit;
 };
+
+// Which matrix a weight-row tile (index over all matrices) belongs to.
+__device__ __forceinline__ int matrix_of(const GemmParams& p, int nt) {
+    int j = 0;
+    while (j + 1 < p.count && nt >= p.tile_base[j + 1]) ++j;
+    return j;
+}
 
 // Channel range, in pipeline units, of part `part` out of `ksplit` (balanced to within one unit).
 __device__ __forceinline__ int unit_begin(int part, int ksplit, int kunits) { return (int)((long long)part * kunits / ksplit); }
@@ -354,8 +367,9 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
             for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
                 const int tile = item / p.ksplit, part = item - tile * p.ksplit;
                 const int u_begin = unit_begin(part, p.ksplit, kunits), u_end = unit_begin(part + 1, p.ksplit, kunits);
-                const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
-                const uint8_t* wtile = p.wt + (size_t)(tile % p.n_tiles) * p.kblocks * W_PACKED_BYTES;
+                const int nt = tile % p.n_tiles, mj = matrix_of(p, nt), ntl = nt - p.tile_base[mj];
+                const int m0 = (tile / p.n_tiles) * TILE_M, n0 = ntl * TILE_N;
+                const uint8_t* wtile = p.wt[mj] + (size_t)ntl * p.kblocks * W_PACKED_BYTES;
                 for (int u = u_begin; u < u_end; ++u, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
                     const uint32_t dst = smem_base + s * C::STAGE_BYTES, bar = bar_full + 8 * s;
@@ -490,12 +504,14 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
         // ------------------------------------------------------------- epilogue
         const int quad = warp & 3;
         const int cbase = ((warp - (2 + 4 * EXPAND_GROUPS)) >> 2) * EPI_COLS;  // this warp's share of the token columns
-        const float alpha = *p.alpha;
         uint32_t tcount = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++tcount) {
             const int tile = item / p.ksplit;
-            const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (tile % p.n_tiles) * TILE_N;
+            const int nt = tile % p.n_tiles, mj = matrix_of(p, nt);
+            const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (nt - p.tile_base[mj]) * TILE_N;
+            const int N = p.N[mj];
+            const float alpha = __ldg(p.alpha[mj]);
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, pab, abort_flag, 6, tcount));
             if (!ok) break;
@@ -505,14 +521,14 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
                 ++cluster_syncs;
             }
             const int n = n0 + quad * 32 + lane;
-            const bool n_ok = n < p.N;
+            const bool n_ok = n < N;
 #pragma unroll 1
             for (int c0 = cbase; c0 < cbase + EPI_COLS; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + ab * ACC_COLS + c0, r);
                 const int mrow = m0 + c0;
                 const int valid = p.M - mrow;  // tokens of this chunk that exist
-                const size_t o = (size_t)mrow * p.N + n;
+                const size_t o = (size_t)mrow * N + n;
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (!n_ok) continue;
                 if (p.ksplit > 1) {
@@ -533,25 +549,25 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
                     }
                     continue;
                 }
-                float* yp = p.Y + o;
+                float* yp = p.Y[mj] + o;
                 const float* sp = p.scale + mrow;
                 // y = fp32(acc) * (scale[m] * alpha): the prefactors of Eq. 2, 3 and 7
                 if (valid >= 32) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
-                        yp += p.N;
+                        yp += N;
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (j < valid) yp[(size_t)j * p.N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                        if (j < valid) yp[(size_t)j * N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
                 }
                 if (p.acc) {
                     int32_t* ap = p.acc + o;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (j < valid) ap[(size_t)j * p.N] = (int)r[j];
+                        if (j < valid) ap[(size_t)j * N] = (int)r[j];
                 }
             }
             tc_fence_before();
@@ -566,21 +582,22 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
         const int te = (int)threadIdx.x - 32 * (2 + 4 * EXPAND_GROUPS);  // index among the epilogue threads
         if (te >= 0 && !*abort_flag) {
             const int tile = (int)blockIdx.x / p.ksplit, rank = (int)blockIdx.x - tile * p.ksplit;
-            const int m0 = (tile / p.n_tiles) * TILE_M, nl = te & (TILE_N - 1), n = (tile % p.n_tiles) * TILE_N + nl;
+            const int nt = tile % p.n_tiles, mj = matrix_of(p, nt), N = p.N[mj];
+            const int m0 = (tile / p.n_tiles) * TILE_M, nl = te & (TILE_N - 1), n = (nt - p.tile_base[mj]) * TILE_N + nl;
             const int tokens = min(TILE_M, p.M - m0);
             const int per = (tokens + p.ksplit - 1) / p.ksplit;  // tokens owned by each rank
             const int rows = min(per, tokens - rank * per);      // ... and by this one (may be <= 0)
-            const float alpha = *p.alpha;
+            const float alpha = __ldg(p.alpha[mj]);
             const int* slots = reinterpret_cast<const int*>(smem);
-            if (n < p.N) {
+            if (n < N) {
                 for (int row = te >> 7; row < rows; row += 128 * EPI_SPLIT / TILE_N) {
                     int sum = 0;
 #pragma unroll
                     for (int q = 0; q < kMaxSplit; ++q)
                         if (q < p.ksplit) sum += slots[(q * per + row) * TILE_N + nl];
                     const int m = m0 + rank * per + row;
-                    const size_t e = (size_t)m * p.N + n;
-                    p.Y[e] = (float)sum * (__ldg(p.scale + m) * alpha);
+                    const size_t e = (size_t)m * N + n;
+                    p.Y[mj][e] = (float)sum * (__ldg(p.scale + m) * alpha);
                     if (p.acc) p.acc[e] = sum;
                 }
             }
@@ -640,13 +657,14 @@ struct Plan {
     int tile_m, n_tiles, m_tiles, ksplit;
 };
 
-Plan make_plan(const bitnet_a48_weight* w, int M, bool ts) {
+Plan make_plan(int count, const bitnet_a48_weight* const* ws, int M, bool ts) {
     Plan pl;
     pl.tile_m = M <= TILE_M_SKINNY ? TILE_M_SKINNY : TILE_M_WIDE;
-    pl.n_tiles = (w->N + TILE_N - 1) / TILE_N;
+    pl.n_tiles = 0;
+    for (int j = 0; j < count; ++j) pl.n_tiles += (ws[j]->N + TILE_N - 1) / TILE_N;
     pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
     const int tiles = pl.n_tiles * pl.m_tiles, sms = sm_count();
-    const int kunits = w->Kp / BK / (ts ? 2 : 1);
+    const int kunits = ws[0]->Kp / BK / (ts ? 2 : 1);
     constexpr int kItemCharge = 3;
     pl.ksplit = 1;
     long long best = (long long)((tiles + sms - 1) / sms) * (kunits + kItemCharge);
@@ -663,8 +681,8 @@ Plan make_plan(const bitnet_a48_weight* w, int M, bool ts) {
 }
 
 template <bool TS, int TM>
-bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
-                         int32_t* acc, Plan pl, cudaStream_t st) {
+bitnet_a48_status launch(int count, const bitnet_a48_weight* const* ws, const int8_t* codes, const float* scale, int M,
+                         float* const* Y, int32_t* acc, Plan pl, cudaStream_t st) {
     using C = Cfg<TS, TM>;
     static bool attr_set[64] = {};        // the attribute is per device
     static signed char cluster_ok[64][kMaxSplit + 1] = {};  // 0 unknown, 1 the device can host such a cluster, -1 it cannot
@@ -676,6 +694,7 @@ bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const 
                                           C::SMEM_BYTES));
         attr_set[dev] = true;
     }
+    const bitnet_a48_weight* w = ws[0];
     CUtensorMap tm_act, tm_w;
     if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TM)) return BITNET_A48_ERR_CUDA;
     if (TS) {
@@ -711,14 +730,19 @@ bitnet_a48_status launch(const bitnet_a48_weight* w, const int8_t* codes, const 
             cfg.numAttrs = 0;
         }
     }
-    GemmParams p;
-    p.wt = w->gemm;
+    GemmParams p = {};
+    p.count = count;
+    p.tile_base[0] = 0;
+    for (int j = 0; j < count; ++j) {
+        p.wt[j] = ws[j]->gemm;
+        p.alpha[j] = ws[j]->alpha_dev;
+        p.Y[j] = Y[j];
+        p.N[j] = ws[j]->N;
+        p.tile_base[j + 1] = p.tile_base[j] + (ws[j]->N + TILE_N - 1) / TILE_N;
+    }
     p.scale = scale;
-    p.alpha = w->alpha_dev;
-    p.Y = Y;
     p.acc = acc;
     p.M = M;
-    p.N = w->N;
     p.K = w->K;
     p.kblocks = w->Kp / BK;
     p.n_tiles = pl.n_tiles;
@@ -741,12 +765,27 @@ bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss) {
 
 bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                           float* Y, int32_t* acc, bool ss, cudaStream_t st) {
-    const Plan pl = make_plan(w, M, !ss);
+    const Plan pl = make_plan(1, &w, M, !ss);
     if (pl.tile_m == TILE_M_SKINNY)
-        return ss ? launch<false, TILE_M_SKINNY>(w, codes, scale, M, Y, acc, pl, st)
-                  : launch<true, TILE_M_SKINNY>(w, codes, scale, M, Y, acc, pl, st);
-    return ss ? launch<false, TILE_M_WIDE>(w, codes, scale, M, Y, acc, pl, st)
-              : launch<true, TILE_M_WIDE>(w, codes, scale, M, Y, acc, pl, st);
+        return ss ? launch<false, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st)
+                  : launch<true, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st);
+    return ss ? launch<false, TILE_M_WIDE>(1, &w, codes, scale, M, &Y, acc, pl, st)
+              : launch<true, TILE_M_WIDE>(1, &w, codes, scale, M, &Y, acc, pl, st);
+}
+
+bool a48_gemm_tcgen05_multi_supported(int count, const bitnet_a48_weight* const* ws, int M) {
+    if (count < 1 || count > MAX_MATS) return false;
+    for (int j = 0; j < count; ++j)
+        if (!a48_gemm_tcgen05_supported(ws[j], M, false) || ws[j]->K != ws[0]->K) return false;
+    return true;
+}
+
+bitnet_a48_status a48_launch_gemm_tcgen05_multi(int count, const bitnet_a48_weight* const* ws, const int8_t* codes,
+                                                const float* scale, int M, float* const* Y, cudaStream_t st) {
+    if (!a48_gemm_tcgen05_multi_supported(count, ws, M)) return BITNET_A48_ERR_UNSUPPORTED;
+    const Plan pl = make_plan(count, ws, M, true);
+    return pl.tile_m == TILE_M_SKINNY ? launch<true, TILE_M_SKINNY>(count, ws, codes, scale, M, Y, nullptr, pl, st)
+                                      : launch<true, TILE_M_WIDE>(count, ws, codes, scale, M, Y, nullptr, pl, st);
 }
 
 bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]) {

@@ -114,3 +114,24 @@ def test_gemm_few_tokens_split_k(a48, oracle, cuda_dev, M, N, K, variant):
         assert a48.kernel_status() == [0, 0, 0, 0]
         assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
         assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+
+
+@pytest.mark.parametrize("Ns,K,M", [((512, 256), 1536, 12), ((3200, 3200, 3200), 3200, 64), ((130, 257, 64, 1000), 400, 33),
+                                    ((1024, 1024), 2048, 100), ((640, 384, 128), 512, 300)])
+def test_gemm_grouped_launch_matches_oracle(a48, oracle, cuda_dev, Ns, K, M):
+    # q/k/v-like and gate/up-like groups beyond the decode kernel's token count: one tensor-core launch walks the
+    # tiles of all matrices (with and without the cluster split); every output against the oracle
+    Ws = [synth.latent_weights(N, K, seed=3 * N + i) for i, N in enumerate(Ns)]
+    ws = [a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_GEMM) for W in Ws]
+    x = synth.gaussian_outlier_activations(M, K, seed=M)
+    codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+    c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS, nthreads=8)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    fused = a48.linear_multi(ws, codes, scale, a48.ACT_INT4)
+    torch.cuda.synchronize()
+    assert a48.kernel_status() == [0, 0, 0, 0]
+    for W, w, y in zip(Ws, ws, fused):
+        t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+        _, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+        assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+        assert torch.equal(y, a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05))
