@@ -273,6 +273,10 @@ struct GemmParams {
     int32_t* acc;         // [M, N_0] or nullptr (single-matrix launches only)
     int M, K;
     int kblocks, n_tiles /* all matrices together */, m_tiles;
+    // Rows of the activation tile that the tensor copy brings in (the box height of the tensor map): the tile
+    // height, or less when the call has fewer tokens.  The MMAs still read the whole tile; what the rows beyond
+    // hold ends up in accumulator columns of tokens that do not exist and is never stored.
+    int act_rows;
     // Split-K (few tiles, many SMs): the channels of a tile are cut into ksplit ranges, one CTA each, and the
     // ksplit CTAs of a tile form one thread-block cluster (cluster rank = range).  Rank o owns a 1/ksplit share
     // of the tile's tokens: once every CTA of the cluster has its accumulator complete (first cluster barrier,
@@ -280,7 +284,17 @@ struct GemmParams {
     // into slot `own rank` of a buffer in o's shared memory (distributed shared memory, stores only); after the
     // second barrier o adds the ksplit slots and writes those rows of Y.
     int ksplit;
+    // Divisions on the path to the first copy cost a single thread hundreds of clocks each, so the host hands
+    // over what they would compute: the unit range of every part, and multipliers that turn the divisions by
+    // ksplit and by n_tiles into a multiply-high (0 stands for a divisor of 1).
+    int ubegin[kMaxSplit + 1];
+    unsigned int ksplit_magic, n_tiles_magic;
 };
+
+// floor(n / d) for n * d < 2^32, with magic = floor(2^32 / d) + 1 (d > 1) or 0 (d == 1).
+__device__ __forceinline__ int fast_div(int n, unsigned int magic) {
+    return magic ? (int)__umulhi((unsigned int)n, magic) : n;
+}
 
 // Which matrix a weight-row tile (index over all matrices) belongs to.
 __device__ __forceinline__ int matrix_of(const GemmParams& p, int nt) {
@@ -288,9 +302,6 @@ __device__ __forceinline__ int matrix_of(const GemmParams& p, int nt) {
     while (j + 1 < p.count && nt >= p.tile_base[j + 1]) ++j;
     return j;
 }
-
-// Channel range, in pipeline units, of part `part` out of `ksplit` (balanced to within one unit).
-__device__ __forceinline__ int unit_begin(int part, int ksplit, int kunits) { return (int)((long long)part * kunits / ksplit); }
 
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -326,6 +337,10 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    // Touch the launch parameters now: their first (cold) reads then overlap the prologue instead of sitting
+    // in front of the producer's first copy.
+    asm volatile("" ::"r"(p.ksplit), "r"(p.n_tiles), "r"(p.m_tiles), "r"(p.kblocks), "r"(p.tile_base[1]), "r"(p.M),
+                 "r"(p.N[0]), "l"(p.wt[0]), "l"(p.scale), "l"(p.Y[0]));
     if (threadIdx.x == 0) {
         // start fetching the tensor-map descriptors now: the first tensor copy otherwise waits for them
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
@@ -356,44 +371,46 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
     const uint32_t tmem_a = tmem_base + ACC_BUFS * ACC_COLS;
     const int total_tiles = p.n_tiles * p.m_tiles;
     const int total_items = total_tiles * p.ksplit;  // item = tile * ksplit + part; split: one item per CTA
-    const int kunits = p.kblocks / KBU;  // the packed layouts pad K so that this is exact
     int cluster_syncs = 0;               // cluster barriers this thread has passed (split-K)
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            uint32_t it = 0, s = 0, ph = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-                const int tile = item / p.ksplit, part = item - tile * p.ksplit;
-                const int u_begin = unit_begin(part, p.ksplit, kunits), u_end = unit_begin(part + 1, p.ksplit, kunits);
-                const int nt = tile % p.n_tiles, mj = matrix_of(p, nt), ntl = nt - p.tile_base[mj];
-                const int m0 = (tile / p.n_tiles) * TILE_M, n0 = ntl * TILE_N;
-                const uint8_t* wtile = p.wt[mj] + (size_t)ntl * p.kblocks * W_PACKED_BYTES;
-                for (int u = u_begin; u < u_end; ++u, ++it) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it))) break;
-                    const uint32_t dst = smem_base + s * C::STAGE_BYTES, bar = bar_full + 8 * s;
-                    mbar_expect_tx(bar, C::STAGE_BYTES);
-                    if (TS)  // the weights first: they come from HBM, the activation tile mostly from L2
+        // The warp walks the loop in lockstep; per unit lane 0 posts the byte count and the weights' bulk copy,
+        // and lanes 1.. issue one tensor copy each (the same instruction, so they go out together).
+        uint32_t it = 0, s = 0, ph = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            const int tile = fast_div(item, p.ksplit_magic), part = item - tile * p.ksplit;
+            const int u_begin = p.ubegin[part], u_end = p.ubegin[part + 1];
+            const int mt = fast_div(tile, p.n_tiles_magic), nt = tile - mt * p.n_tiles;
+            const int mj = matrix_of(p, nt), ntl = nt - p.tile_base[mj];
+            const int m0 = mt * TILE_M, n0 = ntl * TILE_N;
+            const uint8_t* wtile = p.wt[mj] + (size_t)ntl * p.kblocks * W_PACKED_BYTES;
+            const int h = lane - 1;  // the 128-channel block this lane copies (activation tile; SS: then weights)
+            for (int u = u_begin; u < u_end; ++u, ++it) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 1, it));
+                if (!ok) break;
+                const uint32_t dst = smem_base + s * C::STAGE_BYTES, bar = bar_full + 8 * s;
+                if (lane == 0) {
+                    mbar_expect_tx(bar, (uint32_t)(KBU * (p.act_rows * BK + (TS ? W_PACKED_BYTES : A_TILE_BYTES))));
+                    if (TS)  // the weights come from HBM, the activation tile mostly from L2
                         bulk_load(dst + KBU * B_TILE_BYTES, wtile + (size_t)u * KBU * W_PACKED_BYTES, KBU * W_PACKED_BYTES,
                                   bar);
-#pragma unroll
-                    for (int h = 0; h < KBU; ++h) tma_load_2d(dst + h * B_TILE_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
-                    if (!TS) {
-#pragma unroll
-                        for (int h = 0; h < KBU; ++h)
-                            tma_load_2d(dst + KBU * B_TILE_BYTES + h * A_TILE_BYTES, &tm_w, (u * KBU + h) * BK, n0, bar);
-                    }
-                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
+                __syncwarp();
+                if (h >= 0 && h < KBU) tma_load_2d(dst + h * B_TILE_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
+                if (!TS && h >= KBU && h < 2 * KBU)
+                    tma_load_2d(dst + KBU * B_TILE_BYTES + (h - KBU) * A_TILE_BYTES, &tm_w, (u * KBU + h - KBU) * BK, n0, bar);
+                __syncwarp();
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
-            if (!ok) {
-                // aborting: let the copies already issued land before the CTA exits
-                for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
-                    const uint32_t j = it - back, sj = j % STAGES, pj = (j / STAGES) & 1;
-                    const unsigned long long t0 = clock64();
-                    while (!mbar_try(bar_full + 8 * sj, pj) && clock64() - t0 < kWaitClocks) {
-                    }
+        }
+        if (!ok && lane == 0) {
+            // aborting: let the copies already issued land before the CTA exits
+            for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
+                const uint32_t j = it - back, sj = j % STAGES, pj = (j / STAGES) & 1;
+                const unsigned long long t0 = clock64();
+                while (!mbar_try(bar_full + 8 * sj, pj) && clock64() - t0 < kWaitClocks) {
                 }
             }
         }
@@ -409,8 +426,8 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
         uint32_t s = 0, ph = 0;  // stage ring position and phase, advanced without divisions
         bool ok = true;
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++tcount) {
-            const int part = item % p.ksplit;
-            const int u_begin = unit_begin(part, p.ksplit, kunits), u_end = unit_begin(part + 1, p.ksplit, kunits);
+            const int part = item - fast_div(item, p.ksplit_magic) * p.ksplit;
+            const int u_begin = p.ubegin[part], u_end = p.ubegin[part + 1];
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
             const uint32_t d_tmem = tmem_acc + ab * ACC_COLS;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8 * ab, pab ^ 1, abort_flag, 2, tcount));
@@ -460,8 +477,8 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
             const uint32_t a_lanes = tmem_a + ((uint32_t)(quad * 32) << 16);
             long long total_units = 0;  // units of all items of this CTA
             for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
-                const int part = item % p.ksplit;
-                total_units += unit_begin(part + 1, p.ksplit, kunits) - unit_begin(part, p.ksplit, kunits);
+                const int part = item - fast_div(item, p.ksplit_magic) * p.ksplit;
+                total_units += p.ubegin[part + 1] - p.ubegin[part];
             }
             bool ok = true;
             for (long long it64 = group; it64 < total_units && ok; it64 += EXPAND_GROUPS) {
@@ -507,9 +524,9 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
         uint32_t tcount = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++tcount) {
-            const int tile = item / p.ksplit;
-            const int nt = tile % p.n_tiles, mj = matrix_of(p, nt);
-            const int m0 = (tile / p.n_tiles) * TILE_M, n0 = (nt - p.tile_base[mj]) * TILE_N;
+            const int tile = fast_div(item, p.ksplit_magic);
+            const int mt = fast_div(tile, p.n_tiles_magic), nt = tile - mt * p.n_tiles, mj = matrix_of(p, nt);
+            const int m0 = mt * TILE_M, n0 = (nt - p.tile_base[mj]) * TILE_N;
             const int N = p.N[mj];
             const float alpha = __ldg(p.alpha[mj]);
             const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
@@ -581,9 +598,9 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
         for (; cluster_syncs < 2; ++cluster_syncs) cluster_sync_all();
         const int te = (int)threadIdx.x - 32 * (2 + 4 * EXPAND_GROUPS);  // index among the epilogue threads
         if (te >= 0 && !*abort_flag) {
-            const int tile = (int)blockIdx.x / p.ksplit, rank = (int)blockIdx.x - tile * p.ksplit;
-            const int nt = tile % p.n_tiles, mj = matrix_of(p, nt), N = p.N[mj];
-            const int m0 = (tile / p.n_tiles) * TILE_M, nl = te & (TILE_N - 1), n = (nt - p.tile_base[mj]) * TILE_N + nl;
+            const int tile = fast_div((int)blockIdx.x, p.ksplit_magic), rank = (int)blockIdx.x - tile * p.ksplit;
+            const int mt = fast_div(tile, p.n_tiles_magic), nt = tile - mt * p.n_tiles, mj = matrix_of(p, nt), N = p.N[mj];
+            const int m0 = mt * TILE_M, nl = te & (TILE_N - 1), n = (nt - p.tile_base[mj]) * TILE_N + nl;
             const int tokens = min(TILE_M, p.M - m0);
             const int per = (tokens + p.ksplit - 1) / p.ksplit;  // tokens owned by each rank
             const int rows = min(per, tokens - rank * per);      // ... and by this one (may be <= 0)
@@ -696,7 +713,8 @@ bitnet_a48_status launch(int count, const bitnet_a48_weight* const* ws, const in
     }
     const bitnet_a48_weight* w = ws[0];
     CUtensorMap tm_act, tm_w;
-    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, TM)) return BITNET_A48_ERR_CUDA;
+    const int act_rows = M >= TM ? TM : (M + 15) / 16 * 16;
+    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, (uint32_t)act_rows)) return BITNET_A48_ERR_CUDA;
     if (TS) {
         tm_w = tm_act;  // unused
     } else if (!make_map(&tm_w, w->i8, (uint64_t)w->Np, (uint64_t)w->Kp, (uint64_t)w->Kp, TILE_N)) {
@@ -748,6 +766,17 @@ bitnet_a48_status launch(int count, const bitnet_a48_weight* const* ws, const in
     p.n_tiles = pl.n_tiles;
     p.m_tiles = pl.m_tiles;
     p.ksplit = pl.ksplit;
+    p.act_rows = act_rows;
+    {
+        const int kunits = p.kblocks / C::KBU;
+        for (int i = 0; i <= kMaxSplit; ++i) p.ubegin[i] = i <= pl.ksplit ? (int)((long long)i * kunits / pl.ksplit) : kunits;
+        auto magic = [](int d) { return d > 1 ? (unsigned int)((1ull << 32) / (unsigned)d) + 1u : 0u; };
+        p.ksplit_magic = magic(pl.ksplit);
+        p.n_tiles_magic = magic(pl.n_tiles);
+        // the multiply-high is exact while dividend * divisor < 2^32
+        if ((unsigned long long)pl.n_tiles * pl.m_tiles * pl.ksplit * (pl.n_tiles > pl.ksplit ? pl.n_tiles : pl.ksplit) >= (1ull << 32))
+            return BITNET_A48_ERR_SHAPE;
+    }
     if (pl.ksplit == 1) {
         const int total = p.n_tiles * p.m_tiles;
         cfg.gridDim = dim3((unsigned)(total < sm_count() ? total : sm_count()));
