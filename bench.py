@@ -413,83 +413,93 @@ def run_ours(args):
 
 
 def bench_decode(a48, synth, dev, stream, peaks, rank):
-    """Batch-1 BitLinear over all 7 x 32 matrices of the 7B shape, captured once in a CUDA graph."""
+    """BitLinear chain over all 7 x 32 matrices of the 7B shape, one CUDA graph per token count (1, 8, 32, 64)."""
     weights = []
     for layer_i in range(LAYERS):
         for i, (name, n, k, kind) in enumerate(PROJ):
             lat = synth.ternary_latents(n, k, seed=1000 + layer_i * 8 + i + 7000 * rank, device=dev)
-            weights.append((a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE | a48.LAYOUT_SPARSE), n, k, kind))
+            weights.append((a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE | a48.LAYOUT_SPARSE | a48.LAYOUT_GEMM), n, k, kind))
             del lat
-    x_h = synth.gaussian_outlier_activations(1, H, seed=50, device=dev)
-    s_h = synth.student_t3(1, H, seed=51, device=dev)
-    s_f = synth.student_t3(1, F, seed=52, device=dev)
-    c4, d4 = a48.quant_int4(x_h, EPS)
-    c8h, d8h, _ = a48.topk_quant_int8(s_h, H // 2, EPS)
-    c8f, d8f, _ = a48.topk_quant_int8(s_f, F // 2, EPS)
-    y = torch.empty(1, F, dtype=torch.float32, device=dev)
-    ws_need = max(a48.linear_workspace_bytes(w, 1) for w, *_ in weights)
-    ws = torch.zeros(max(ws_need, 16), dtype=torch.uint8, device=dev)
     packed_bytes = sum(w.packed_bytes for w, *_ in weights)
-    nz = {"int4": float((c4 != 0).float().mean()), "topk_h": float((c8h != 0).float().mean()),
-          "topk_f": float((c8f != 0).float().mean())}
-    needed_bytes = 0
-    for w, n, k, kind in weights:
-        frac = nz["int4"] if kind == "int4" else (nz["topk_h"] if k == H else nz["topk_f"])
-        needed_bytes += w.packed_bytes * frac
-
-    ys = [torch.empty(1, F, dtype=torch.float32, device=dev) for _ in range(3)]
-    ws_multi = max(a48.linear_multi_workspace_bytes([w for w, *_ in weights[0:3]], 1),
-                   a48.linear_multi_workspace_bytes([w for w, *_ in weights[4:6]], 1), ws_need, 16)
-    ws = torch.zeros(ws_multi, dtype=torch.uint8, device=dev)
     fused = not os.environ.get("A48_BENCH_DECODE_UNFUSED")
 
-    def chain():
-        # per layer: q,k,v share the attention input and gate,up the FFN input: one call each (one launch each)
-        for li in range(LAYERS):
-            (wq, *_), (wk, *_), (wv, *_), (wo, *_), (wg, *_), (wu, *_), (wd, *_) = weights[7 * li:7 * li + 7]
-            if fused:
-                a48.linear_multi([wq, wk, wv], c4, d4, a48.ACT_INT4, Ys=[t[:, :H] for t in ys], workspace=ws)
-            else:
-                for w_, t in zip((wq, wk, wv), ys):
-                    a48.linear(w_, c4, d4, a48.ACT_INT4, Y=t[:, :H], workspace=ws)
-            a48.linear(wo, c8h, d8h, a48.ACT_TOPK_INT8, Y=y[:, :H], workspace=ws)
-            if fused:
-                a48.linear_multi([wg, wu], c4, d4, a48.ACT_INT4, Ys=[ys[0], ys[1]], workspace=ws)
-            else:
-                a48.linear(wg, c4, d4, a48.ACT_INT4, Y=ys[0], workspace=ws)
-                a48.linear(wu, c4, d4, a48.ACT_INT4, Y=ys[1], workspace=ws)
-            a48.linear(wd, c8f, d8f, a48.ACT_TOPK_INT8, Y=y[:, :H], workspace=ws)
+    def time_chain(M):
+        x_h = synth.gaussian_outlier_activations(M, H, seed=50, device=dev)
+        s_h = synth.student_t3(M, H, seed=51, device=dev)
+        s_f = synth.student_t3(M, F, seed=52, device=dev)
+        c4, d4 = a48.quant_int4(x_h, EPS)
+        c8h, d8h, _ = a48.topk_quant_int8(s_h, H // 2, EPS)
+        c8f, d8f, _ = a48.topk_quant_int8(s_f, F // 2, EPS)
+        y = torch.empty(M, F, dtype=torch.float32, device=dev)
+        ys = [torch.empty(M, F, dtype=torch.float32, device=dev) for _ in range(3)]
+        yh = [torch.empty(M, H, dtype=torch.float32, device=dev) for _ in range(3)]
+        ws_need = max(a48.linear_workspace_bytes(w, M) for w, *_ in weights[:7])
+        ws_multi = max(a48.linear_multi_workspace_bytes([w for w, *_ in weights[0:3]], M),
+                       a48.linear_multi_workspace_bytes([w for w, *_ in weights[4:6]], M), ws_need, 16)
+        ws = torch.zeros(ws_multi, dtype=torch.uint8, device=dev)
+        # channels with a non-zero code in at least one of the M tokens: the weight bytes a call really needs
+        nz = {"int4": float((c4 != 0).any(0).float().mean()), "topk_h": float((c8h != 0).any(0).float().mean()),
+              "topk_f": float((c8f != 0).any(0).float().mean())}
+        needed_bytes = 0
+        for w, n, k, kind in weights:
+            needed_bytes += w.packed_bytes * (nz["int4"] if kind == "int4" else (nz["topk_h"] if k == H else nz["topk_f"]))
 
-    for _ in range(2):
-        chain()
-    torch.cuda.synchronize()
-    side = torch.cuda.Stream()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(side):
-        chain()
-        side.synchronize()
-        with torch.cuda.graph(graph, stream=side):
+        def chain():
+            # per layer: q,k,v share the attention input and gate,up the FFN input: one call each (one launch each)
+            for li in range(LAYERS):
+                (wq, *_), (wk, *_), (wv, *_), (wo, *_), (wg, *_), (wu, *_), (wd, *_) = weights[7 * li:7 * li + 7]
+                if fused:
+                    a48.linear_multi([wq, wk, wv], c4, d4, a48.ACT_INT4, Ys=yh, workspace=ws)
+                else:
+                    for w_, t in zip((wq, wk, wv), yh):
+                        a48.linear(w_, c4, d4, a48.ACT_INT4, Y=t, workspace=ws)
+                a48.linear(wo, c8h, d8h, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws)
+                if fused:
+                    a48.linear_multi([wg, wu], c4, d4, a48.ACT_INT4, Ys=[ys[0], ys[1]], workspace=ws)
+                else:
+                    a48.linear(wg, c4, d4, a48.ACT_INT4, Y=ys[0], workspace=ws)
+                    a48.linear(wu, c4, d4, a48.ACT_INT4, Y=ys[1], workspace=ws)
+                a48.linear(wd, c8f, d8f, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws)
+
+        for _ in range(2):
             chain()
-    torch.cuda.synchronize()
-    for _ in range(3):
-        graph.replay()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = 10
-    e0.record(stream)
-    for _ in range(reps):
-        graph.replay()
-    e1.record(stream)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
-    gbs_dense = packed_bytes / (ms * 1e-3) / 1e9
-    out = {"metric": "decode_weight_stream_gbs_7b_batch1", "value": gbs_dense, "unit": "GB/s",
-           "ms_per_token_all_bitlinears": ms, "packed_weight_bytes": packed_bytes, "matrices": len(weights),
-           "hbm_peak_gbs": peaks["hbm_gbs"], "frac_of_hbm_peak": gbs_dense / peaks["hbm_gbs"],
-           "algorithmic_gbs": needed_bytes / (ms * 1e-3) / 1e9, "nonzero_code_fraction": nz,
-           "tokens_per_s": 1e3 / ms, "launches_per_layer": 4 if fused else 7,
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            chain()
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                chain()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 10
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        del graph
+        return {"ms_all_bitlinears": ms, "weight_stream_gbs": packed_bytes / (ms * 1e-3) / 1e9,
+                "algorithmic_gbs": needed_bytes / (ms * 1e-3) / 1e9, "tokens_per_s": M * 1e3 / ms,
+                "dense_equivalent_tops": 2.0 * M * packed_bytes * 4 / (ms * 1e-3) / 1e12, "nonzero_channel_fraction": nz}
+
+    by_tokens = {str(M): time_chain(M) for M in (1, 8, 32, 64)}
+    one = by_tokens["1"]
+    out = {"metric": "decode_weight_stream_gbs_7b_batch1", "value": one["weight_stream_gbs"], "unit": "GB/s",
+           "ms_per_token_all_bitlinears": one["ms_all_bitlinears"], "packed_weight_bytes": packed_bytes,
+           "matrices": len(weights), "hbm_peak_gbs": peaks["hbm_gbs"],
+           "frac_of_hbm_peak": one["weight_stream_gbs"] / peaks["hbm_gbs"], "algorithmic_gbs": one["algorithmic_gbs"],
+           "nonzero_code_fraction": one["nonzero_channel_fraction"], "tokens_per_s": one["tokens_per_s"],
+           "launches_per_layer": 4 if fused else 7, "by_tokens": by_tokens,
            "note": "CUDA-graph chain over 224 distinct matrices (1.6 GB >> L2), q/k/v and gate/up each as one "
-           "bitnet_a48_linear_multi call; value counts every packed byte, algorithmic_gbs only channels with a non-zero code"}
+           "bitnet_a48_linear_multi call; value counts every packed byte, algorithmic_gbs only channels with a non-zero "
+           "code in some token; 1 and 8 tokens run the streaming decode kernel, 32 and 64 the tensor-core kernel "
+           "(64-token tile, cluster split-K)"}
     for w, *_ in weights:
         w.free()
     return out
