@@ -230,15 +230,37 @@ __global__ void __launch_bounds__(256) attn_tile_kernel(const float* __restrict_
     }
 }
 
-// Few queries per sequence (decode): one block per (query, head, batch); the 8
-// warps stride over the keys, each lane holding hd/32 (rounded up) columns.
+// Few queries per sequence (decode): the keys of one (query, head, batch) are split over the ATTN_SPLITS CTAs
+// of a thread-block cluster, so that a batch-1 step at a 2048-token context runs on 256 CTAs instead of 32 and
+// streams the fp32 cache at memory speed.  Inside a CTA the 8 warps stride over the keys, four keys per
+// iteration (their loads are in flight together), each lane holding hd/32 (rounded up) columns; online softmax
+// per warp, warps meet in shared memory.  The CTAs of a cluster then combine through distributed shared memory:
+// rank r reads every rank's (max, sum) and its own 1/ATTN_SPLITS share of the output columns.
+constexpr int ATTN_SPLITS = 8;
+
+__device__ __forceinline__ float ld_cluster_f32(const float* p, unsigned rank) {
+    float v;
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %1, %2;\n\tld.shared::cluster.f32 %0, [ra];\n\t}"
+        : "=f"(v)
+        : "r"((unsigned)__cvta_generic_to_shared(p)), "r"(rank));
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 template <int CPL>
 __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__ q, const float* __restrict__ kcache,
                                                        const float* __restrict__ vcache, int T, int nh, int hd,
                                                        int pos0, int cap, float scale, float* __restrict__ out) {
+    constexpr int COLS = 32 * CPL;
+    static_assert(COLS % ATTN_SPLITS == 0, "every rank finishes the same number of columns");
     __shared__ float sm_m[8], sm_l[8];
-    __shared__ float sm_o[8][32 * CPL];
-    const int t = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    __shared__ float sm_o[8][COLS];
+    __shared__ float cta_ml[2];  // this CTA's running max and sum, read by the peers
+    __shared__ float cta_o[COLS];
+    const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z / T, t = blockIdx.z % T;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t H = (size_t)nh * hd;
     const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
@@ -253,25 +275,44 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
     }
     float m = -INFINITY, l = 0.f;
     const int n_keys = pos0 + t + 1;
-    for (int j = warp; j < n_keys; j += 8) {
-        float dot = 0.f;
-        float vv[CPL];
+    const int per = (n_keys + ATTN_SPLITS - 1) / ATTN_SPLITS;
+    const int j_end = min(n_keys, (split + 1) * per);
+    for (int j = split * per + warp; j < j_end; j += 32) {
+        float kk[4][CPL], vv[4][CPL], dot[4];
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-            int col = lane + 32 * c;
-            float kv = col < hd ? kbase[(size_t)j * hd + col] : 0.f;
-            vv[c] = col < hd ? vbase[(size_t)j * hd + col] : 0.f;
-            dot += qreg[c] * kv;
+        for (int u = 0; u < 4; ++u) {
+            const int jj = j + 8 * u;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const int col = lane + 32 * c;
+                const bool ok = jj < j_end && col < hd;
+                kk[u][c] = ok ? __ldg(kbase + (size_t)jj * hd + col) : 0.f;
+                vv[u][c] = ok ? __ldg(vbase + (size_t)jj * hd + col) : 0.f;
+            }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-        float m_new = fmaxf(m, dot);
-        float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
-        float p = expf(dot - m_new);
-        l = l * corr + p;
+        for (int u = 0; u < 4; ++u) {
+            dot[u] = 0.f;
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) o[c] = o[c] * corr + p * vv[c];
-        m = m_new;
+            for (int c = 0; c < CPL; ++c) dot[u] += qreg[c] * kk[u][c];
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], off);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (j + 8 * u < j_end) {
+                const float m_new = fmaxf(m, dot[u]);
+                const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+                const float pr = expf(dot[u] - m_new);
+                l = l * corr + pr;
+#pragma unroll
+                for (int c = 0; c < CPL; ++c) o[c] = o[c] * corr + pr * vv[u][c];
+                m = m_new;
+            }
+        }
     }
     if (lane == 0) {
         sm_m[warp] = m;
@@ -294,12 +335,55 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
 #pragma unroll
             for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][lane + 32 * c] * f;
         }
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-            int col = lane + 32 * c;
-            if (col < hd) out[((size_t)b * T + t) * H + (size_t)h * hd + col] = acc[c] / ll;
+        if (lane == 0) {
+            cta_ml[0] = mm;
+            cta_ml[1] = ll;
         }
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) cta_o[lane + 32 * c] = acc[c];
     }
+    cluster_sync_all();  // every CTA's partial is in its shared memory
+    constexpr int CPR = COLS / ATTN_SPLITS;  // columns finished by each rank
+    if (threadIdx.x < CPR) {
+        const int col = split * CPR + (int)threadIdx.x;
+        float pm[ATTN_SPLITS], pl[ATTN_SPLITS], po[ATTN_SPLITS];
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) {
+            pm[r] = ld_cluster_f32(&cta_ml[0], (unsigned)r);
+            pl[r] = ld_cluster_f32(&cta_ml[1], (unsigned)r);
+            po[r] = ld_cluster_f32(&cta_o[col], (unsigned)r);
+        }
+        float mm = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) mm = fmaxf(mm, pm[r]);
+        float ll = 0.f, acc = 0.f;
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) {
+            const float f = pm[r] == -INFINITY ? 0.f : expf(pm[r] - mm);
+            ll += pl[r] * f;
+            acc += po[r] * f;
+        }
+        if (col < hd) out[((size_t)b * T + t) * H + (size_t)h * hd + col] = acc / ll;
+    }
+    cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
+}
+
+template <int CPL>
+cudaError_t launch_attn_row(const float* q, const float* kcache, const float* vcache, int B, int T, int nh, int hd,
+                            int pos0, int cap, float* out, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ATTN_SPLITS, (unsigned)nh, (unsigned)(B * T));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ATTN_SPLITS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attn_row_kernel<CPL>, q, kcache, vcache, T, nh, hd, pos0, cap,
+                              1.f / sqrtf((float)hd), out);
 }
 
 __global__ void add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ y, size_t n4) {
@@ -383,11 +467,9 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
                                                                           kcache, vcache);
     }
     if (T <= 8) {
-        dim3 grid(T, nh, B);
-        const float sc = 1.f / sqrtf((float)hd);
-        if (hd <= 64) attn_row_kernel<2><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
-        else if (hd <= 128) attn_row_kernel<4><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
-        else attn_row_kernel<8><<<grid, 256, 0, st>>>(q, kcache, vcache, T, nh, hd, pos0, cap, sc, att);
+        if (hd <= 64) A48_CUDA_TRY(launch_attn_row<2>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+        else if (hd <= 128) A48_CUDA_TRY(launch_attn_row<4>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+        else A48_CUDA_TRY(launch_attn_row<8>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     } else if (hd <= 64) {
         A48_TRY(launch_attn_tile<64>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     } else if (hd <= 128) {
