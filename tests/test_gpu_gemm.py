@@ -135,3 +135,40 @@ def test_gemm_grouped_launch_matches_oracle(a48, oracle, cuda_dev, Ns, K, M):
         _, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
         assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
         assert torch.equal(y, a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05))
+
+
+@pytest.mark.parametrize("M", [32, 64])
+def test_gemm_decode_batch_3b_layer(a48, oracle, cuda_dev, M):
+    # The 3B decode configuration at 32 and 64 tokens, in the launch form the benchmark's chain uses: q/k/v and
+    # gate/up as grouped launches, o and down as single (cluster split-K) launches; int32-exact against the oracle
+    H, F = 3200, 8640
+    def make(n, k, seed):
+        W = synth.ternary_latents(n, k, seed=seed)
+        return W, a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_GEMM)
+    x4 = synth.gaussian_outlier_activations(M, H, seed=5)
+    c4, d4 = a48.quant_int4(x4.to(cuda_dev), EPS)
+    c4_ref, d4_ref = oracle.quant_int4(x4.numpy(), EPS, nthreads=8)
+    assert np.array_equal(c4.cpu().numpy(), c4_ref)
+    for Ns, K, codes, scale, c_ref, d_ref, act in [((H, H, H), H, c4, d4, c4_ref, d4_ref, a48.ACT_INT4),
+                                                   ((F, F), H, c4, d4, c4_ref, d4_ref, a48.ACT_INT4)]:
+        pairs = [make(n, K, 70 + i) for i, n in enumerate(Ns)]
+        ys = a48.linear_multi([w for _, w in pairs], codes, scale, act)
+        torch.cuda.synchronize()
+        assert a48.kernel_status() == [0, 0, 0, 0]
+        for (W, w), y in zip(pairs, ys):
+            t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+            _, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+            assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+    for n, k in [(H, H), (H, F)]:
+        xs = synth.student_t3(M, k, seed=k)
+        c8, d8, _ = a48.topk_quant_int8(xs.to(cuda_dev), k // 2, EPS)
+        c8_ref, d8_ref, _ = oracle.topk_quant_int8(xs.numpy(), k // 2, EPS, nthreads=8)
+        assert np.array_equal(c8.cpu().numpy(), c8_ref)
+        W, w = make(n, k, 90 + n % 7)
+        y, acc = a48.linear(w, c8, d8, a48.ACT_TOPK_INT8, want_acc=True)
+        torch.cuda.synchronize()
+        assert a48.kernel_status() == [0, 0, 0, 0]
+        t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+        acc_ref, y_ref = oracle.linear(c8_ref, d8_ref, t_ref, alpha, nthreads=8)
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
