@@ -126,6 +126,17 @@ bitnet_a48_status bitnet_a48_topk_quant_int8(const float* X_dev, int M, int K, i
                                              int8_t* codes_dev, float* scale_dev, uint32_t* mask_bits_dev,
                                              void* stream);
 
+/* Compacted form of code rows for consumers that skip masked channels (Section 2.1: the masked entries of
+ * Eq. 1 contribute nothing to the contraction; a channel is skipped iff its code is 0, which also covers
+ * kept entries that quantise to 0).  For every row m of codes_dev [M, K] (int8, row-major): the channels
+ * with a non-zero code in ascending order, idx_dev [M, cap] (uint16 channel index) and val_dev [M, cap]
+ * (the code), and count_dev[m] = the number of non-zero codes of the row.  Only the first min(count, cap)
+ * entries of a row are written; count > cap tells the caller that the row did not fit (cap >= k always fits
+ * the output of bitnet_a48_topk_quant_int8).  All buffers caller-owned device memory, 16-byte aligned;
+ * K <= 65535; asynchronous on `stream`. */
+bitnet_a48_status bitnet_a48_compact_codes(const int8_t* codes_dev, int M, int K, int cap, uint16_t* idx_dev,
+                                           int8_t* val_dev, int32_t* count_dev, void* stream);
+
 /* FP4 (E2M1) MinMax quantiser, Eq. 8-9: per token, 2^b = 12/|x|max, step =
  * 2^(max(floor(log2|x·2^b|),1)-1), code = step·round(x·2^b/step) (an integer in
  * {0,±1,±2,±3,±4,±6,±8,±12}), scale[m] = |x|max/12.  Same shapes as quant_int4. */

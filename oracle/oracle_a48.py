@@ -104,6 +104,29 @@ def quant_fp4(X, nthreads=1):
     return g, d
 
 
+def compact_codes(codes):
+    """Section 2.1 / Eq. 1: per row the channels whose code is non-zero, ascending, with their codes.
+
+    Returns a list of (idx int64 array, val int8 array), one pair per row.  The definition written out."""
+    codes = np.ascontiguousarray(codes, dtype=np.int8)
+    out = []
+    for row in codes:
+        idx = np.flatnonzero(row != 0)
+        out.append((idx.astype(np.int64), row[idx].copy()))
+    return out
+
+
+def linear_from_lists(lists, scale, t, alpha):
+    """Eq. 1 evaluated over the compacted rows only: acc[m, n] = sum over listed channels of code * t[n, channel]."""
+    t = np.ascontiguousarray(t, dtype=np.int8).astype(np.int64)
+    scale = np.ascontiguousarray(scale, dtype=np.float64)
+    acc = np.zeros((len(lists), t.shape[0]), np.int64)
+    for m, (idx, val) in enumerate(lists):
+        for j, c in zip(idx.tolist(), val.tolist()):
+            acc[m] += int(c) * t[:, j]
+    return acc, acc.astype(np.float64) * scale[:, None] * float(alpha)
+
+
 def linear(codes, scale, t, alpha, nthreads=1, want_acc=True, want_y=True):
     """Eq. 1 / Eq. 6.  Returns (acc int64 [M,N] or None, y float64 [M,N] or None)."""
     codes = np.ascontiguousarray(codes, dtype=np.int8)

@@ -25,6 +25,7 @@ EXPORTS = [
     "bitnet_a48_status_string", "bitnet_a48_pack_ternary", "bitnet_a48_weight_unpack",
     "bitnet_a48_weight_unpack_layout", "bitnet_a48_weight_dims", "bitnet_a48_weight_packed_bytes",
     "bitnet_a48_weight_free", "bitnet_a48_quant_int4", "bitnet_a48_topk_quant_int8", "bitnet_a48_quant_fp4",
+    "bitnet_a48_compact_codes",
     "bitnet_a48_linear", "bitnet_a48_linear_ex", "bitnet_a48_linear_workspace_bytes",
     "bitnet_a48_bitlinear_host", "bitnet_a48_bitlinear_host_workspace_bytes", "bitnet_a48_block_create",
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
@@ -75,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_topk_quant_int8.argtypes = [c_void_p, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p,
                                                  c_void_p]
         L.bitnet_a48_quant_fp4.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p]
+        L.bitnet_a48_compact_codes.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.bitnet_a48_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                         c_size_t, c_void_p]
         L.bitnet_a48_linear_ex.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p,
@@ -195,6 +197,18 @@ def quant_fp4(X: torch.Tensor, codes=None, scale=None, stream=None):
     scale = scale if scale is not None else torch.empty(M, dtype=torch.float32, device=X.device)
     _check(lib().bitnet_a48_quant_fp4(_ptr(X), M, K, _ptr(codes), _ptr(scale), _stream(stream)), "quant_fp4")
     return codes, scale
+
+
+def compact_codes(codes: torch.Tensor, cap: int, stream=None):
+    """Non-zero codes of every row as (channel index uint16, code int8) lists [M, cap] plus counts [M] (int32)."""
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.is_contiguous() and codes.dim() == 2
+    M, K = codes.shape
+    idx = torch.zeros(M, cap, dtype=torch.uint16, device=codes.device)
+    val = torch.zeros(M, cap, dtype=torch.int8, device=codes.device)
+    count = torch.empty(M, dtype=torch.int32, device=codes.device)
+    _check(lib().bitnet_a48_compact_codes(_ptr(codes), M, K, cap, _ptr(idx), _ptr(val), _ptr(count), _stream(stream)),
+           "compact_codes")
+    return idx, val, count
 
 
 def linear_workspace_bytes(w: Weight, M: int) -> int:

@@ -164,6 +164,16 @@ bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t*
     return a48_launch_quant_fp4(X_dev, M, K, codes_dev, scale_dev, (cudaStream_t)stream);
 }
 
+bitnet_a48_status bitnet_a48_compact_codes(const int8_t* codes_dev, int M, int K, int cap, uint16_t* idx_dev,
+                                           int8_t* val_dev, int32_t* count_dev, void* stream) {
+    if (!codes_dev || !idx_dev || !val_dev || !count_dev) return BITNET_A48_ERR_INVALID_ARG;
+    if (M <= 0 || K <= 0 || K > 65535 || cap <= 0) return BITNET_A48_ERR_SHAPE;  // indices are 16-bit
+    if (!a48_aligned16(codes_dev) || !a48_aligned16(idx_dev) || !a48_aligned16(val_dev) || !a48_aligned16(count_dev))
+        return BITNET_A48_ERR_ALIGNMENT;
+    if (!have_device()) return BITNET_A48_ERR_CUDA;
+    return a48_launch_compact_codes(codes_dev, M, K, cap, idx_dev, val_dev, count_dev, (cudaStream_t)stream);
+}
+
 size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M) {
     if (!w || M <= 0) return 0;
     const size_t dense = a48_decode_workspace_bytes(w, M), sparse = a48_decode_sparse_workspace_bytes(w, M);

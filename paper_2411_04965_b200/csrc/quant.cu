@@ -465,6 +465,47 @@ __global__ void __launch_bounds__(kBlock) quant_fp4_generic_kernel(const float* 
     if (t == 0) scale[row] = (float)(amax / 12.0);
 }
 
+// ---------------------------------------------------------------------------- compacted form of a code row
+// The channels with a non-zero code, in ascending channel order, as (index, code) pairs: what a consumer of
+// Eq. 1 needs when it skips the masked channels.  One block per row; a thread owns four consecutive channels
+// per step, so thread order is channel order and an exclusive scan of the per-thread counts gives the places.
+__global__ void __launch_bounds__(kBlock) compact_codes_kernel(const int8_t* __restrict__ codes, int M, int K, int cap,
+                                                               uint16_t* __restrict__ idx, int8_t* __restrict__ val,
+                                                               int32_t* __restrict__ count) {
+    __shared__ unsigned red[kBlock / 32];
+    const int row = blockIdx.x, t = threadIdx.x;
+    const int8_t* cr = codes + (size_t)row * K;
+    const bool words = (K & 3) == 0;  // rows then start on a 4-byte boundary
+    unsigned running = 0;
+    for (int j0 = 0; j0 < K; j0 += kBlock * 4) {
+        const int j = j0 + 4 * t;
+        int c[4];
+        if (words && j + 3 < K) {
+            const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(cr + j));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) c[q] = (int)(int8_t)(w >> (8 * q));
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) c[q] = j + q < K ? (int)cr[j + q] : 0;
+        }
+        const unsigned cnt = (unsigned)(c[0] != 0) + (c[1] != 0) + (c[2] != 0) + (c[3] != 0);
+        unsigned total;
+        unsigned at = running + group_excl_scan<kBlock>(cnt, red, 0, total);
+        running += total;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (c[q] != 0) {
+                if (at < (unsigned)cap) {
+                    idx[(size_t)row * cap + at] = (uint16_t)(j + q);
+                    val[(size_t)row * cap + at] = (int8_t)c[q];
+                }
+                ++at;
+            }
+        }
+    }
+    if (t == 0) count[row] = (int32_t)running;
+}
+
 template <bool NORM>
 void launch_int4(const float* X, int M, int K, double eps, int8_t* codes, float* scale, const float* gain,
                  double norm_eps, cudaStream_t st) {
@@ -521,6 +562,13 @@ bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k
 
 bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st) {
     quant_fp4_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, codes, scale);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_launch_compact_codes(const int8_t* codes, int M, int K, int cap, uint16_t* idx, int8_t* val,
+                                           int32_t* count, cudaStream_t st) {
+    compact_codes_kernel<<<M, kBlock, 0, st>>>(codes, M, K, cap, idx, val, count);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }

@@ -122,3 +122,33 @@ def test_quantisers_at_benchmark_size_sampled(a48, oracle, cuda_dev, K, kind):
         assert bool((codes.abs().amax(1) == 127).all())
     assert np.array_equal(codes[rows].cpu().numpy(), q_ref)
     assert np.array_equal(scale[rows].cpu().numpy(), d_ref.astype(np.float32))
+
+
+@pytest.mark.parametrize("M,K,kfrac", [(1, 4096, 0.5), (3, 11008, 0.5), (8, 3200, 0.5), (5, 250, 0.3), (2, 65535, 0.1),
+                                       (4, 1027, 1.0)])
+def test_compact_codes_matches_oracle(a48, oracle, cuda_dev, M, K, kfrac):
+    # compacted (channel, code) lists of the top-K codes: same entries, same order, same counts as the oracle's
+    x = synth.student_t3(M, K, seed=K + M)
+    k = max(1, int(K * kfrac))
+    codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), k, EPS)
+    c_ref, _, _ = oracle.topk_quant_int8(x.numpy(), k, EPS)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    idx, val, count = a48.compact_codes(codes, cap=k)
+    torch.cuda.synchronize()
+    lists = oracle.compact_codes(c_ref)
+    idx_h, val_h, cnt_h = idx.cpu().numpy().astype(np.int64), val.cpu().numpy(), count.cpu().numpy()
+    for m, (i_ref, v_ref) in enumerate(lists):
+        assert cnt_h[m] == len(i_ref) <= k
+        assert np.array_equal(idx_h[m, :cnt_h[m]], i_ref) and np.array_equal(val_h[m, :cnt_h[m]], v_ref)
+        assert not idx_h[m, cnt_h[m]:].any() and not val_h[m, cnt_h[m]:].any()  # nothing written past the count
+
+
+def test_compact_codes_capacity_and_arguments(a48, cuda_dev):
+    codes = torch.zeros(2, 64, dtype=torch.int8, device=cuda_dev)
+    codes[0, ::2] = 7   # 32 non-zero codes, capacity 8: only the first 8 are written, the count says 32
+    idx, val, count = a48.compact_codes(codes, cap=8)
+    assert count.tolist() == [32, 0]
+    assert idx[0].tolist() == list(range(0, 16, 2)) and val[0].tolist() == [7] * 8
+    wide = torch.zeros(1, 65536, dtype=torch.int8, device=cuda_dev)  # indices would not fit 16 bits
+    with pytest.raises(RuntimeError):
+        a48.compact_codes(wide, cap=16)

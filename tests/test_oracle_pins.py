@@ -241,3 +241,26 @@ def test_fp4_grid(oracle):
     assert (np.diff(g[0][order].astype(int)) >= 0).all()
     gz, dz = oracle.quant_fp4(np.zeros((1, 8), np.float32))
     assert not gz.any() and dz[0] == 0.0
+
+
+def test_compacted_rows_reproduce_the_dense_contraction(oracle):
+    # Section 2.1: masked channels contribute nothing to Eq. 1, so the contraction over the listed channels
+    # alone equals the dense one; the list itself is pinned by hand on a small row and by its invariants.
+    row = np.array([[0, 5, 0, 0, -3, 0, 127, 0, -128, 0, 0, 1]], np.int8)
+    (idx, val), = oracle.compact_codes(row)
+    assert idx.tolist() == [1, 4, 6, 8, 11] and val.tolist() == [5, -3, 127, -128, 1]
+    rng = np.random.default_rng(5)
+    X = rng.standard_t(3, size=(6, 96)).astype(np.float32)
+    codes, d, mask = oracle.topk_quant_int8(X, 48, 1e-5)
+    lists = oracle.compact_codes(codes)
+    for m, (idx, val) in enumerate(lists):
+        assert np.all(np.diff(idx) > 0) and np.all(val != 0)           # ascending, no zero entries
+        assert len(idx) <= 48 and np.all(mask[m, idx] == 1)            # only kept channels, at most k of them
+        dense = np.zeros(96, np.int8)
+        dense[idx] = val
+        assert np.array_equal(dense, codes[m])                         # scatter gives the row back
+    W = rng.normal(0, 0.02, size=(10, 96)).astype(np.float32)
+    t, alpha = oracle.ternarise(W, 1e-5)
+    acc_dense, y_dense = oracle.linear(codes, d, t, alpha)
+    acc_list, y_list = oracle.linear_from_lists(lists, d, t, alpha)
+    assert np.array_equal(acc_dense, acc_list) and np.array_equal(y_dense, y_list)
