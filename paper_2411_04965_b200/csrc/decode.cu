@@ -575,7 +575,10 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     // Two CTAs must fit on an SM for a launch to request its weights while its predecessor still computes: with
     // many tokens the staged codes take room, so the pieces get shorter (more rounds of pieces) until they do.
     const size_t fixed_smem = (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
+    // (Only while the pieces stay whole tiles: pieces that share every tile pay more in fix-ups than the overlap
+    // gives back - 13.4 us instead of 9 us for 4096 x 11008 at four tokens.)
     while (fixed_smem <= 64 * 1024 && grid % sm_count() == 0 && grid < 2ll * sm_count() && p.units / grid > 32 &&
+           ntiles >= grid + sm_count() &&
            fixed_smem + (size_t)((p.units + grid - 1) / grid) * UNIT_BYTES > 112 * 1024)
         grid += sm_count();
     p.grid = (int)grid;

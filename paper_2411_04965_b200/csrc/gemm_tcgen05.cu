@@ -682,13 +682,15 @@ Plan make_plan(int count, const bitnet_a48_weight* const* ws, int M, bool ts) {
     pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
     const int tiles = pl.n_tiles * pl.m_tiles, sms = sm_count();
     const int kunits = ws[0]->Kp / BK / (ts ? 2 : 1);
-    constexpr int kItemCharge = 3;
+    // fixed cost of a wave of CTAs in units: launch, prologue, first copy, epilogue come to about 5 us, a unit to
+    // 0.33-0.47 us (measured); with 3 a split into two waves was chosen for 512 tokens x 4096 x 11008 and lost 2x
+    constexpr int kItemCharge = 10;
     pl.ksplit = 1;
     long long best = (long long)((tiles + sms - 1) / sms) * (kunits + kItemCharge);
     for (int ks = 2; ks <= kMaxSplit && ks <= kunits && tiles < sms; ++ks) {
         const int slots = sms / ks * ks;  // whole clusters only
         const long long rounds = ((long long)tiles * ks + slots - 1) / slots;
-        const long long cost = rounds * ((kunits + ks - 1) / ks + kItemCharge + 1);
+        const long long cost = rounds * ((kunits + ks - 1) / ks + kItemCharge + 2);
         if (cost * 10 < best * 9) {  // a split has to pay for itself by a clear margin
             best = cost;
             pl.ksplit = ks;
