@@ -34,10 +34,23 @@
 //
 // Warp roles (one persistent CTA per SM): warp 0 TMA producer, warp 1 MMA issuer
 // and TMEM owner, warps 2-9 weight expanders (TS only; two groups of four, group
-// g takes every second unit and owns slot g), warps 10-17 epilogue (two per
-// tensor-memory lane quadrant, each draining half of the accumulator columns).
-// Every mbarrier wait is bounded; a wait that gives up records a status word and
-// the CTA drains and exits without touching tensor memory again.
+// g takes every second unit, unit it goes to slot it % slots), warps 10-17
+// epilogue (two per tensor-memory lane quadrant, each draining half of the
+// accumulator columns).  Every mbarrier wait is bounded; a wait that gives up
+// records a status word and the CTA drains and exits without touching tensor
+// memory again.
+//
+// Three forms of the same kernel:
+//   - 192-token tiles (prefill): as described above.
+//   - 64-token tiles (at most 64 tokens in the call): MMA N = 64, eight pipeline
+//     stages, six slots for the expanded weights, activation box as high as the
+//     call has tokens.
+//   - split-K: with fewer tiles than SMs the channels of a tile are cut into up to
+//     eight ranges, one CTA each; the CTAs of a tile form a thread-block cluster
+//     and exchange their int32 partial sums through distributed shared memory
+//     (stores into the owner's shared memory between two cluster barriers).
+// One launch can walk the tiles of up to four weight matrices that share K and
+// the activation codes (q/k/v, gate/up).
 #include <cuda.h>
 
 #include "internal.h"
