@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libbitnet_a48.so")
 ACT_INT4, ACT_TOPK_INT8, ACT_FP4 = 0, 1, 2
 LAYOUT_GEMM, LAYOUT_DECODE, LAYOUT_SPARSE, LAYOUT_ALL, LAYOUT_I8 = 1, 2, 4, 7, 8
 ALGO_AUTO, ALGO_SIMPLE, ALGO_GEMM_TCGEN05, ALGO_DECODE, ALGO_DECODE_SPARSE, ALGO_GEMM_TCGEN05_I8 = 0, 1, 2, 3, 4, 5
+ALGO_GEMM_TCGEN05_PAIR = 6
 
 EXPORTS = [
     "bitnet_a48_status_string", "bitnet_a48_pack_ternary", "bitnet_a48_weight_unpack",

@@ -641,6 +641,286 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
     }
 }
 
+// ---- CTA-pair form (cta_group::2) ------------------------------------------------------------------------------
+// Two CTAs on neighbouring SMs (a cluster of two) work on one tile of 256 weight rows x 192 tokens.  Each CTA
+// expands and holds the 128 weight rows of its half in its own tensor memory and accumulates their 192 outputs
+// per token there; the token tile is split the other way: each CTA stages 96 of the 192 tokens in its shared
+// memory and the MMA (issued by the CTA of rank 0 for both) reads the two halves.  An activation byte thus feeds
+// 256 weight rows instead of 128: the traffic from L2 into an SM per MMA, which is what the single-CTA kernel's
+// stalls trace back to, is halved, and the ring of stages reaches twice as far ahead in time.
+// Protocol across the pair: the expanders of both CTAs arrive on the afull barriers of rank 0 (remote arrive for
+// rank 1) after they have seen their own stage land, so rank 0's issuer knows weights and tokens of both CTAs
+// are in place; one commit per stage is multicast to the empty barriers of both CTAs (stage and tensor-memory
+// slot free in both), one per tile to both acc_full barriers; the epilogue threads of both CTAs arrive on rank
+// 0's acc_empty.  No TMA multicast is used: every CTA copies its own half.
+template <int TOK_, int A_SLOTS_, int STAGES_>
+struct PairCfg {
+    static constexpr int TOK = TOK_, HALF = TOK / 2, KBU = 2;
+    static constexpr int B_HALF_BYTES = HALF * BK;
+    static constexpr int STAGE_BYTES = KBU * (B_HALF_BYTES + W_PACKED_BYTES);
+    static constexpr int STAGES = STAGES_;
+    static constexpr int A_SLOTS = A_SLOTS_, A_SLOT_COLS = KBU * BK / 4, ACC_COLS = TOK;
+    static constexpr int EXPAND_GROUPS = 2, EPI_SPLIT = 2;
+    static constexpr int EPI_FIRST = (TOK / 32 + 1) / 2 * 32;  // columns drained by the first epilogue warp of a quadrant
+    static constexpr int NUM_THREADS = 32 * (2 + 4 * EXPAND_GROUPS + 4 * EPI_SPLIT);
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 1024;
+    static_assert(HALF % 8 == 0 && TOK % 32 == 0, "swizzle rows and 32-column epilogue chunks");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(ACC_BUFS * ACC_COLS + A_SLOTS * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
+    static_assert(STAGES > A_SLOTS, "the stage A_SLOTS units back must still be distinct");
+};
+
+__device__ __forceinline__ void mbar_arrive_rank(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(rank)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrives on `bar` in both CTAs of the pair
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"((unsigned short)3)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc),
+        "r"(accumulate)
+        : "memory");
+}
+
+struct PairParams {
+    const uint8_t* wt;
+    const float* alpha;
+    const float* scale;
+    float* Y;
+    int32_t* acc;
+    int M, N, kblocks, n_pairs, m_tiles;
+    unsigned int n_pairs_magic;
+};
+
+template <class PC>
+__global__ void __launch_bounds__(PC::NUM_THREADS, 1)
+    gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const PairParams p) {
+    constexpr int TOK = PC::TOK, HALF = PC::HALF, KBU = PC::KBU, B_HALF_BYTES = PC::B_HALF_BYTES;
+    constexpr int STAGE_BYTES = PC::STAGE_BYTES, STAGES = PC::STAGES, A_SLOTS = PC::A_SLOTS, A_SLOT_COLS = PC::A_SLOT_COLS;
+    constexpr int ACC_COLS = PC::ACC_COLS, EXPAND_GROUPS = PC::EXPAND_GROUPS, EPI_SPLIT = PC::EPI_SPLIT;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* ctrl = smem + STAGES * STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);  // full[S] empty[S] afull[A] acc_full[2] acc_empty[2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 512);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 516);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
+    const uint32_t bar_afull = bar_empty + 8 * STAGES;
+    const uint32_t bar_acc_full = bar_afull + 8 * A_SLOTS, bar_acc_empty = bar_acc_full + 8 * ACC_BUFS;
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = (int)(blockIdx.x & 1u);       // rank in the pair; rank 0 issues the MMAs
+    const int pair = (int)(blockIdx.x >> 1), pairs = (int)(gridDim.x >> 1);
+
+    asm volatile("" ::"r"(p.n_pairs), "r"(p.m_tiles), "r"(p.kblocks), "r"(p.M), "r"(p.N), "l"(p.wt), "l"(p.scale), "l"(p.Y));
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 5);  // four expander warps of this CTA and the multicast commit
+        }
+        // afull and acc_empty are used in rank 0 only; one lane per warp arrives for its warp (a release at
+        // cluster scope by every thread cost ~1400 clocks per unit)
+        for (int s = 0; s < A_SLOTS; ++s) mbar_init(bar_afull + 8 * s, 2 * 4);  // one expander group of each CTA
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 2 * 4 * EPI_SPLIT);  // the epilogue warps of both CTAs
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers are initialised and its tensor memory is allocated
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_acc = tmem_base;
+    const uint32_t tmem_a = tmem_base + ACC_BUFS * ACC_COLS;
+    const int total_tiles = p.n_pairs * p.m_tiles;
+    const int kunits = p.kblocks / KBU;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------- TMA producer (both CTAs, own halves)
+        uint32_t it = 0, s = 0, ph = 0;
+        bool ok = true;
+        for (int tile = pair; tile < total_tiles && ok; tile += pairs) {
+            const int mt = fast_div(tile, p.n_pairs_magic), pn = tile - mt * p.n_pairs;
+            const int m0 = mt * TOK + rank * HALF;  // this CTA stages its half of the token tile
+            const uint8_t* wtile = p.wt + (size_t)(2 * pn + rank) * p.kblocks * W_PACKED_BYTES;
+            const int h = lane - 1;
+            for (int u = 0; u < kunits; ++u, ++it) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 11, it));
+                if (!ok) break;
+                const uint32_t dst = smem_base + s * STAGE_BYTES, bar = bar_full + 8 * s;
+                if (lane == 0) {
+                    mbar_expect_tx(bar, STAGE_BYTES);
+                    bulk_load(dst + KBU * B_HALF_BYTES, wtile + (size_t)u * KBU * W_PACKED_BYTES, KBU * W_PACKED_BYTES, bar);
+                }
+                __syncwarp();
+                if (h >= 0 && h < KBU) tma_load_2d(dst + h * B_HALF_BYTES, &tm_act, (u * KBU + h) * BK, m0, bar);
+                __syncwarp();
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+            }
+        }
+        if (!ok && lane == 0) {
+            for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
+                const uint32_t j = it - back, sj = j % STAGES, pj = (j / STAGES) & 1;
+                const unsigned long long t0 = clock64();
+                while (!mbar_try(bar_full + 8 * sj, pj) && clock64() - t0 < kWaitClocks) {
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------- MMA issuer (rank 0 only)
+        if (rank == 0) {
+            constexpr uint32_t idesc = idesc_i8(2 * TILE_N, TOK);
+            const bool leader = elect_one();
+            uint32_t it = 0, tcount = 0, s = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += pairs, ++tcount) {
+                const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
+                const uint32_t d_tmem = tmem_acc + ab * ACC_COLS;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8 * ab, pab ^ 1, abort_flag, 12, tcount));
+                if (!ok) break;
+                tc_fence_after();
+                for (int u = 0; u < kunits; ++u, ++it) {
+                    const uint32_t slot = it % A_SLOTS, pslot = (it / A_SLOTS) & 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * slot, pslot, abort_flag, 14, it));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (leader) {
+                        const uint32_t b_addr = smem_base + s * STAGE_BYTES;
+#pragma unroll
+                        for (int h = 0; h < KBU; ++h) {
+                            const uint64_t b_desc = smem_desc_sw128(b_addr + h * B_HALF_BYTES);
+                            const uint32_t a_t = tmem_a + slot * A_SLOT_COLS + h * (BK / 4);
+#pragma unroll
+                            for (int j = 0; j < BK / UMMA_K; ++j)
+                                mma_ts_pair(d_tmem, a_t + j * (UMMA_K / 4), b_desc + 2 * j, idesc, (u > 0 || h > 0 || j > 0) ? 1u : 0u);
+                        }
+                        tc_commit_pair(bar_empty + 8 * s);
+                    }
+                    __syncwarp();
+                    if (++s == (uint32_t)STAGES) s = 0;
+                }
+                if (ok && leader) tc_commit_pair(bar_acc_full + 8 * ab);
+                __syncwarp();
+            }
+        }
+    } else if (warp < 2 + 4 * EXPAND_GROUPS) {
+        // ------------------------------------------------------------- weight expanders (both CTAs)
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t group = (uint32_t)(warp - 2) >> 2;
+        const uint32_t a_lanes = tmem_a + ((uint32_t)(quad * 32) << 16);
+        const int my_tiles = (total_tiles - pair + pairs - 1) / pairs;
+        const long long total_units = (long long)kunits * (my_tiles > 0 ? my_tiles : 0);
+        bool ok = true;
+        for (long long it64 = group; it64 < total_units && ok; it64 += EXPAND_GROUPS) {
+            const uint32_t it = (uint32_t)it64;
+            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1, slot = it % A_SLOTS;
+            const uint32_t a_dst = a_lanes + slot * A_SLOT_COLS;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag, 17, it));
+            if (!ok) break;
+            const uint4* src = reinterpret_cast<const uint4*>(smem + s * STAGE_BYTES + KBU * B_HALF_BYTES);
+            uint32_t v[KBU][32];
+#pragma unroll
+            for (int h = 0; h < KBU; ++h) {
+                const uint4 lo = src[h * 256 + row], hi = src[h * 256 + 128 + row];
+                expand_word(lo.x, v[h] + 0);
+                expand_word(lo.y, v[h] + 4);
+                expand_word(lo.z, v[h] + 8);
+                expand_word(lo.w, v[h] + 12);
+                expand_word(hi.x, v[h] + 16);
+                expand_word(hi.y, v[h] + 20);
+                expand_word(hi.z, v[h] + 24);
+                expand_word(hi.w, v[h] + 28);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            if (it >= (uint32_t)A_SLOTS) {
+                const uint32_t j = it - A_SLOTS, sj = j % STAGES, pj = (j / STAGES) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * sj, pj, abort_flag, 15, it));
+                if (!ok) break;
+            }
+            tc_fence_after();
+#pragma unroll
+            for (int h = 0; h < KBU; ++h) tmem_st32(a_dst + h * (BK / 4), v[h]);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_rank(bar_afull + 8 * slot, 0u);  // this warp's rows are in tensor memory, the tokens have landed
+        }
+    } else {
+        // ------------------------------------------------------------- epilogue (both CTAs, own 128 rows)
+        const int quad = warp & 3;
+        const int half = (warp - (2 + 4 * EXPAND_GROUPS)) >> 2;
+        const int c_begin = half ? PC::EPI_FIRST : 0, c_end = half ? TOK : PC::EPI_FIRST;
+        const float alpha = __ldg(p.alpha);
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = pair; tile < total_tiles && ok; tile += pairs, ++tcount) {
+            const int mt = fast_div(tile, p.n_pairs_magic), pn = tile - mt * p.n_pairs;
+            const int m0 = mt * TOK, n = (2 * pn + rank) * TILE_N + quad * 32 + lane;
+            const uint32_t ab = tcount % ACC_BUFS, pab = (tcount / ACC_BUFS) & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, pab, abort_flag, 16, tcount));
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + ab * ACC_COLS + c0, r);
+                const int mrow = m0 + c0;
+                const int valid = p.M - mrow;
+                const size_t o = (size_t)mrow * p.N + n;
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                float* yp = p.Y + o;
+                const float* sp = p.scale + mrow;
+                if (valid >= 32) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                        yp += p.N;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) yp[(size_t)j * p.N] = (float)(int)r[j] * (__ldg(sp + j) * alpha);
+                }
+                if (p.acc) {
+                    int32_t* ap = p.acc + o;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) ap[(size_t)j * p.N] = (int)r[j];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_rank(bar_acc_empty + 8 * ab, 0u);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs are done with both tensor memories and with each other's barriers
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
 // ---- host side -----------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -800,7 +1080,67 @@ bitnet_a48_status launch(int count, const bitnet_a48_weight* const* ws, const in
     return BITNET_A48_OK;
 }
 
+template <class PC>
+bitnet_a48_status launch_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
+                              int32_t* acc, cudaStream_t st) {
+    static signed char ready[64] = {};  // per device: 0 unknown, 1 attribute set and a pair can be hosted, -1 not
+    int dev = 0;
+    A48_CUDA_TRY(cudaGetDevice(&dev));
+    dev &= 63;
+    CUtensorMap tm_act;
+    if (!make_map(&tm_act, codes, (uint64_t)M, (uint64_t)w->K, (uint64_t)w->K, PC::HALF)) return BITNET_A48_ERR_CUDA;
+    PairParams p;
+    p.wt = w->gemm;
+    p.alpha = w->alpha_dev;
+    p.scale = scale;
+    p.Y = Y;
+    p.acc = acc;
+    p.M = M;
+    p.N = w->N;
+    p.kblocks = w->Kp / BK;
+    p.n_pairs = w->N / (2 * TILE_N);
+    p.m_tiles = (M + PC::TOK - 1) / PC::TOK;
+    p.n_pairs_magic = p.n_pairs > 1 ? (unsigned int)((1ull << 32) / (unsigned)p.n_pairs) + 1u : 0u;
+    const long long total = (long long)p.n_pairs * p.m_tiles;
+    if (total * p.n_pairs >= (1ll << 32)) return BITNET_A48_ERR_SHAPE;
+    const int pairs_max = sm_count() / 2;
+    const int pairs = total < pairs_max ? (int)total : pairs_max;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(PC::NUM_THREADS);
+    cfg.dynamicSmemBytes = PC::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (ready[dev] == 0) {
+        A48_CUDA_TRY(cudaFuncSetAttribute(gemm_pair_kernel<PC>, cudaFuncAttributeMaxDynamicSharedMemorySize, PC::SMEM_BYTES));
+        int clusters = 0;
+        ready[dev] = cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel<PC>, &cfg) == cudaSuccess && clusters >= 1 ? 1 : -1;
+        if (ready[dev] < 0) (void)cudaGetLastError();
+    }
+    if (ready[dev] < 0) return BITNET_A48_ERR_UNSUPPORTED;
+    A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_pair_kernel<PC>, tm_act, p));
+    return BITNET_A48_OK;
+}
+
 }  // namespace
+
+bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M) {
+    return a48_gemm_tcgen05_supported(w, M, false) && w->N % (2 * TILE_N) == 0;
+}
+
+bitnet_a48_status a48_launch_gemm_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
+                                       float* Y, int32_t* acc, cudaStream_t st) {
+    if (!a48_gemm_pair_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
+    // 192 tokens, two weight slots, seven 32 KB stages: measured 4-8 % ahead of 160 tokens / three slots / eight
+    // stages and 15 % ahead of 128 / four / nine
+    return launch_pair<PairCfg<192, 2, 7>>(w, codes, scale, M, Y, acc, st);
+}
 
 bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss) {
     if (w->K % 16 != 0 || M < 1) return false;  // TMA needs a 16-byte row pitch

@@ -45,6 +45,44 @@ def test_gemm_tcgen05_matches_oracle(a48, oracle, cuda_dev, M, N, K, variant, ki
     assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
 
 
+# CTA-pair form (cta_group::2): 256 weight rows per two SMs; N must be a multiple of 256.  One pair tile, several
+# k-blocks, ragged M (second half of the token tile partly or wholly beyond M), several tiles per pair, K = 8640.
+PAIR_SHAPES = [(192, 256, 256), (100, 256, 1024), (97, 512, 384), (300, 768, 2048), (1100, 1536, 1536), (200, 256, 8640)]
+
+
+@pytest.mark.parametrize("M,N,K", PAIR_SHAPES)
+@pytest.mark.parametrize("kind", ["int4", "topk"])
+def test_gemm_pair_matches_oracle(a48, oracle, cuda_dev, M, N, K, kind):
+    W = synth.latent_weights(N, K, seed=N + K + 2)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_GEMM)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=M + 1)
+        codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+        c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS, nthreads=8)
+        act = a48.ACT_INT4
+    else:
+        x = synth.student_t3(M, K, seed=M + 1)
+        codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+        c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS, nthreads=8)
+        act = a48.ACT_TOPK_INT8
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    for _ in range(2):
+        y, acc = a48.linear(w, codes, scale, act, a48.ALGO_GEMM_TCGEN05_PAIR, want_acc=True)
+        torch.cuda.synchronize()
+        assert a48.kernel_status() == [0, 0, 0, 0]
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+
+
+def test_gemm_pair_rejects_other_row_counts(a48, cuda_dev):
+    w = a48.pack_ternary(synth.latent_weights(384, 256, seed=1).to(cuda_dev), EPS, a48.LAYOUT_GEMM)  # 384 = 1.5 x 256
+    codes = torch.zeros(64, 256, dtype=torch.int8, device=cuda_dev)
+    with pytest.raises(RuntimeError):
+        a48.linear(w, codes, torch.ones(64, device=cuda_dev), a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05_PAIR)
+
+
 def test_gemm_extreme_codes_do_not_overflow(a48, oracle, cuda_dev):
     # all codes +-127 against all-(+1) weights: |acc| = 127*K, the largest accumulator this path can see
     M, N, K = 256, 128, 11008
@@ -68,9 +106,13 @@ def test_gemm_full_size_sampled(a48, oracle, cuda_dev):
     t_dev, alpha = a48.weight_unpack(w)
     x = synth.gaussian_outlier_activations(M, K, seed=40, device=cuda_dev)
     codes, scale = a48.quant_int4(x, EPS)
-    y, acc = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05, want_acc=True)
+    # the library's own choice at this size, as in the benchmark: the CTA-pair form
+    y, acc = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_AUTO, want_acc=True)
+    y1, acc1 = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_GEMM_TCGEN05, want_acc=True)
     torch.cuda.synchronize()
     assert a48.kernel_status() == [0, 0, 0, 0]
+    assert torch.equal(acc, acc1) and torch.equal(y, y1)  # single-CTA form: the same bits
+    del y1, acc1
     g = torch.Generator().manual_seed(0)
     rows = torch.cat([torch.tensor([0, 255, 256, M - 1]), torch.randint(0, M, (20,), generator=g)]).to(cuda_dev)
     cols = torch.cat([torch.tensor([0, 127, 128, N - 1]), torch.randint(0, N, (20,), generator=g)]).to(cuda_dev)
