@@ -42,10 +42,10 @@ PROJ = (("q", H, H, "int4"), ("k", H, H, "int4"), ("v", H, H, "int4"), ("o", H, 
 STEP_OPS = sum(2 * M_PREFILL * n * k for _, n, k, _ in PROJ)
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum).
-# Capture: profiles/gemm_tcgen05_prefill_M4096_N11008_K4096.md (151.3 MB of DRAM traffic against 208.5 MB of
+# Capture: profiles/gemm_pair_prefill_M4096_N11008_K4096.md (150.9 MB of DRAM traffic against 208.5 MB of
 # algorithmic bytes at M=4096, part of the output still in L2 at kernel end), scaled to the mean algorithmic bytes
 # of the seven launches of a step at M=16384 (488 MB): traffic grows with M like the algorithmic bytes do.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 3.54e8
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 3.53e8
 
 
 def load_peaks():

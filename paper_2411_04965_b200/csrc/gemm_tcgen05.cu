@@ -40,7 +40,8 @@
 // records a status word and the CTA drains and exits without touching tensor
 // memory again.
 //
-// Three forms of the same kernel:
+// A fourth form, gemm_pair_kernel further down, puts one 256-row tile on a pair of CTAs (cta_group::2).
+// Three forms of this kernel:
 //   - 192-token tiles (prefill): as described above.
 //   - 64-token tiles (at most 64 tokens in the call): MMA N = 64, eight pipeline
 //     stages, six slots for the expanded weights, activation box as high as the
