@@ -65,7 +65,7 @@ typedef enum {
     BITNET_A48_ALGO_DECODE = 3,       /* M <= 8: streams every weight byte once */
     BITNET_A48_ALGO_DECODE_SPARSE = 4, /* M == 1: fetches only channels whose code is non-zero */
     BITNET_A48_ALGO_GEMM_TCGEN05_I8 = 5, /* comparison variant: int8 weight copy staged through shared memory */
-    BITNET_A48_ALGO_GEMM_TCGEN05_PAIR = 6 /* tcgen05 cta_group::2: two SMs per 256-row tile; N % 256 == 0 */
+    BITNET_A48_ALGO_GEMM_TCGEN05_PAIR = 6 /* tcgen05 cta_group::2: two SMs per tile of 256 weight rows */
 } bitnet_a48_algo;
 
 typedef struct bitnet_a48_weight bitnet_a48_weight; /* packed ternary matrix + alpha + N, K */

@@ -697,6 +697,8 @@ struct PairParams {
     float* Y;
     int32_t* acc;
     int M, N, kblocks, n_pairs, m_tiles;
+    int n_tiles128;  // 128-row weight tiles in the packed layout; an odd count leaves the last pair's second CTA
+                     // without rows of its own: it re-reads the last tile and stores nothing
     unsigned int n_pairs_magic;
 };
 
@@ -760,7 +762,7 @@ __global__ void __launch_bounds__(PC::NUM_THREADS, 1)
         for (int tile = pair; tile < total_tiles && ok; tile += pairs) {
             const int mt = fast_div(tile, p.n_pairs_magic), pn = tile - mt * p.n_pairs;
             const int m0 = mt * TOK + rank * HALF;  // this CTA stages its half of the token tile
-            const uint8_t* wtile = p.wt + (size_t)(2 * pn + rank) * p.kblocks * W_PACKED_BYTES;
+            const uint8_t* wtile = p.wt + (size_t)min(2 * pn + rank, p.n_tiles128 - 1) * p.kblocks * W_PACKED_BYTES;
             const int h = lane - 1;
             for (int u = 0; u < kunits; ++u, ++it) {
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, 11, it));
@@ -888,6 +890,7 @@ __global__ void __launch_bounds__(PC::NUM_THREADS, 1)
                 const int valid = p.M - mrow;
                 const size_t o = (size_t)mrow * p.N + n;
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (n >= p.N) continue;
                 float* yp = p.Y + o;
                 const float* sp = p.scale + mrow;
                 if (valid >= 32) {
@@ -1099,7 +1102,8 @@ bitnet_a48_status launch_pair(const bitnet_a48_weight* w, const int8_t* codes, c
     p.M = M;
     p.N = w->N;
     p.kblocks = w->Kp / BK;
-    p.n_pairs = w->N / (2 * TILE_N);
+    p.n_tiles128 = (w->N + TILE_N - 1) / TILE_N;
+    p.n_pairs = (p.n_tiles128 + 1) / 2;
     p.m_tiles = (M + PC::TOK - 1) / PC::TOK;
     p.n_pairs_magic = p.n_pairs > 1 ? (unsigned int)((1ull << 32) / (unsigned)p.n_pairs) + 1u : 0u;
     const long long total = (long long)p.n_pairs * p.m_tiles;
@@ -1131,9 +1135,7 @@ bitnet_a48_status launch_pair(const bitnet_a48_weight* w, const int8_t* codes, c
 
 }  // namespace
 
-bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M) {
-    return a48_gemm_tcgen05_supported(w, M, false) && w->N % (2 * TILE_N) == 0;
-}
+bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M) { return a48_gemm_tcgen05_supported(w, M, false); }
 
 bitnet_a48_status a48_launch_gemm_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                        float* Y, int32_t* acc, cudaStream_t st) {

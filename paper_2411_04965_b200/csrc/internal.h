@@ -72,7 +72,7 @@ bitnet_a48_status a48_launch_linear_simple(const bitnet_a48_weight* w, const int
 bool a48_gemm_tcgen05_supported(const bitnet_a48_weight* w, int M, bool ss);
 bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                           float* Y, int32_t* acc, bool ss, cudaStream_t st);
-// CTA-pair form (one tile of 256 weight rows per two SMs): N % 256 == 0.
+// CTA-pair form (one tile of 256 weight rows per two SMs).
 bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_gemm_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                        float* Y, int32_t* acc, cudaStream_t st);

@@ -110,7 +110,7 @@ def main():
             ms = _time(lambda: a48.topk_quant_int8(x, K // 2, EPS, codes, scale), args.reps, stream)
         out.update(ms=ms, gbs=(5.0 * M * K + 4 * M) / ms / 1e6)
     elif args.case == "gemm":
-        algo = args.algo or (a48.ALGO_GEMM_TCGEN05_PAIR if M >= 1024 and N % 256 == 0 else a48.ALGO_GEMM_TCGEN05)
+        algo = args.algo or (a48.ALGO_GEMM_TCGEN05_PAIR if M >= 1024 else a48.ALGO_GEMM_TCGEN05)
         layouts = a48.LAYOUT_GEMM | (a48.LAYOUT_I8 if algo == a48.ALGO_GEMM_TCGEN05_I8 else 0)
         w = a48.pack_ternary(synth.ternary_latents(N, K, seed=4, device=dev), EPS, layouts)
         _, codes, scale, act = _acts(args.kind, M, K, dev)
