@@ -319,7 +319,7 @@ __device__ __forceinline__ unsigned group_excl_scan(unsigned cnt, unsigned* red,
 }
 
 template <int TPR, int V>
-__global__ void __launch_bounds__(kBlock, V >= 12 ? 3 : (V >= 8 ? 4 : 6))
+__global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
     topk_quant_int8_kernel(const float* __restrict__ X, int M, int K, int k, double eps, int8_t* __restrict__ codes,
                            float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
