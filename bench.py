@@ -547,6 +547,25 @@ def bench_block(a48, synth, dev, stream, layer):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
         out[f"decode_b{Bd}"] = {"tokens_per_s": Bd / (ms * 1e-3), "ms": ms, "context": 2048}
+        # the same call captured once in a CUDA graph (the call is stream-ordered, so a caller can do this)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd, stream=side)
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd, stream=side)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_g = e0.elapsed_time(e1) / reps
+        out[f"decode_b{Bd}"].update({"ms_cuda_graph": ms_g, "tokens_per_s_cuda_graph": Bd / (ms_g * 1e-3)})
+        del graph
     blk.free()
     out["note"] = "one 7B-shape block (fp32 attention glue included); tokens/s per block, not per model"
     return out
