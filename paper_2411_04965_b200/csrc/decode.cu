@@ -37,8 +37,8 @@
 
 namespace {
 
-constexpr int WARPS = 8;
-constexpr int THREADS = 32 * WARPS;
+constexpr int WARPS_MANY = 8;   // warps per CTA of the mma.sync form (2..8 tokens)
+constexpr int WARPS_ONE = 12;   // ... of the one-token form
 constexpr int UNIT_BYTES = 512;   // 16 rows x 128 channels of 2-bit codes
 constexpr int TOK = 8;            // tokens per launch (one MMA column group)
 constexpr int MAX_SHARE = 288;    // units per CTA (144 KB of packed weights)
@@ -152,7 +152,11 @@ __device__ __forceinline__ int owner_of(const DecodeParams& p, int u) {
 }
 
 // Dynamic shared memory: wbuf [share][512] | act [M][act_row_bytes] | sacc [MAX_TILES][16][TOK] s32 | csum [TOK] s32
-__global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, int share_max) {
+// NW warps per CTA; ONE_TOKEN compiles the dp4a walk alone (M == 1: fewer registers, so twelve warps fit twice on
+// an SM and shorten the walk that has to follow the dependency wait), otherwise the mma.sync walk alone.
+template <int NW, bool ONE_TOKEN>
+__global__ void __launch_bounds__(32 * NW, ONE_TOKEN ? 2 : 1) decode_kernel(const DecodeParams p, int share_max) {
+    constexpr int WARPS = NW, THREADS = 32 * NW;
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* wbuf = smem;
     uint8_t* act = wbuf + (size_t)share_max * UNIT_BYTES;
@@ -179,7 +183,9 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     // depends on anything but the weights, so it runs before the wait for the kernel ahead of this one in the
     // stream (programmatic dependent launch): the weight stream of this call overlaps the tail of the previous one.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int cg = WARPS * ((p.kchunks + WARPS * MAX_GROUPS - 1) / (WARPS * MAX_GROUPS));
+    // (twelve warps: at most five groups, so that a group still gives every warp two units at K = 11008)
+    constexpr int GROUPS = ONE_TOKEN ? 5 : MAX_GROUPS;
+    const int cg = WARPS * ((p.kchunks + WARPS * GROUPS - 1) / (WARPS * GROUPS));
     const int ngroups = (p.kchunks + cg - 1) / cg;
     // Pieces of one to six whole tiles (the usual case at model shapes) run code compiled for their tile count,
     // with the per-tile addresses in registers: a copy or a fragment load then costs one multiply-add.
@@ -264,7 +270,7 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
     const int g = lane >> 2, tig = lane & 3;
     const bool tok_ok = g < p.M;  // B-fragment column g is token g; columns of missing tokens stay zero
     const uint8_t* arow = act + (size_t)(tok_ok ? g : 0) * p.act_row_bytes + tig * 4;
-    if (p.M == 1) {
+    if constexpr (ONE_TOKEN) {
         // One token: the MMA would spend seven of its eight columns on nothing, so the CUDA cores do it with dp4a.
         // A word masked with 0x03030303 << 2q is four u8 fields e * 4^q of one row and one 32-channel slice; the
         // sums of slice q carry the factor 4^q, which an exact shift removes at the end.  Rows g (words 0, 2) and
@@ -395,7 +401,8 @@ __global__ void __launch_bounds__(THREADS) decode_kernel(const DecodeParams p, i
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         if (lane == 0) atomicAdd(csum, xsum);
-    } else {
+    }
+    if constexpr (!ONE_TOKEN) {
     int xsum = 0;  // this lane's share of sum_k x[g][k]
     auto walk = [&](auto nt_c) {
     constexpr int NT = decltype(nt_c)::value;
@@ -593,17 +600,8 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     p.piece_r = (int)(items % grid);
     const size_t smem = (size_t)share_max * UNIT_BYTES + (size_t)M * p.act_row_bytes + (size_t)MAX_TILES * 16 * TOK * 4 + TOK * 4;
     if (smem > 227 * 1024 - 64) return BITNET_A48_ERR_UNSUPPORTED;
-    static size_t smem_set_dev[64] = {};  // the attribute is per device
-    int dev = 0;
-    A48_CUDA_TRY(cudaGetDevice(&dev));
-    size_t& smem_set = smem_set_dev[dev & 63];
-    if (smem > smem_set) {
-        A48_CUDA_TRY(cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        smem_set = smem;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -611,7 +609,30 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     attr[0].val.programmaticStreamSerializationAllowed = prefetch_ok ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel, p, share_max));
+    int dev = 0;
+    A48_CUDA_TRY(cudaGetDevice(&dev));
+    // one token: the dp4a form with twelve warps; more: the mma.sync form with eight (the attribute is per device)
+    if (M == 1) {
+        static size_t smem_set_dev[64] = {};
+        size_t& smem_set = smem_set_dev[dev & 63];
+        if (smem > smem_set) {
+            A48_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<WARPS_ONE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)smem));
+            smem_set = smem;
+        }
+        cfg.blockDim = dim3(32 * WARPS_ONE);
+        A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel<WARPS_ONE, true>, p, share_max));
+    } else {
+        static size_t smem_set_dev[64] = {};
+        size_t& smem_set = smem_set_dev[dev & 63];
+        if (smem > smem_set) {
+            A48_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<WARPS_MANY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)smem));
+            smem_set = smem;
+        }
+        cfg.blockDim = dim3(32 * WARPS_MANY);
+        A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel<WARPS_MANY, false>, p, share_max));
+    }
     for (int j = 0; j < count; ++j) wv[j]->decode_prefetch_ok = true;
     return BITNET_A48_OK;
 }
