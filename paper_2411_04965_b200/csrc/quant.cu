@@ -366,6 +366,24 @@ __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
     unsigned running = 0;
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
     const int mask_words = (K + 31) >> 5;
+    if (!ordered && !mask_bits) {
+        // The usual case (uniform over the row's threads): every entry equal to tau is kept, so the mask is one
+        // comparison, and no bitmap is wanted.  The clip of Eq. 3 is left out here: |127 x / (gamma + eps)| <= 127
+        // for every finite x of the row, so it cannot fire.
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int idx = i * TPR + t;
+            if (idx < nv) {
+                const int a = key(v[i].x) >= s.tau ? __double2int_rn(mult * (double)v[i].x) : 0;
+                const int b = key(v[i].y) >= s.tau ? __double2int_rn(mult * (double)v[i].y) : 0;
+                const int c = key(v[i].z) >= s.tau ? __double2int_rn(mult * (double)v[i].z) : 0;
+                const int d = key(v[i].w) >= s.tau ? __double2int_rn(mult * (double)v[i].w) : 0;
+                out[idx] = pack4(a, b, c, d);
+            }
+        }
+        if (t == 0) scale[row] = (float)(gamma / 127.0);
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         const int idx = i * TPR + t;
