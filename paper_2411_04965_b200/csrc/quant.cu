@@ -219,20 +219,23 @@ __device__ __forceinline__ Select radix_select(int k, unsigned* hist, unsigned* 
 // pass (the 8 exponent bits) runs over the registers as above; the elements of the chosen binade - about a third
 // of a row of real data - are then copied into shared memory, and the three remaining passes (8, 8 and 7 mantissa
 // bits) walk that list instead of testing every element of the row again.
-// hist: 256 bins; sel: 4 words; cand: room for every key of the row.
-template <class ForEachKey>
+// The first pass and the copy take the raw float bits: sign and exponent together index 512 bins (one shift per
+// element; the two halves are added when the bins are scanned), and the binade test is a mask and a compare.
+// hist: 512 bins; sel: 4 words; cand: room for every key of the row.
+template <class ForEachRaw>
 __device__ __forceinline__ Select radix_select_compact(int k, unsigned* hist, unsigned* sel, unsigned* cand, int t,
-                                                       ForEachKey for_each_key) {
+                                                       ForEachRaw for_each_raw) {
     unsigned prefix = 0, kr = (unsigned)k, eq_total = 0, n_cand = 0;
 #pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
         const int bits = pass == 3 ? 7 : 8;
         const int shift = pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0));
         hist[t] = 0;
+        if (pass == 0) hist[t + 256] = 0;
         if (pass == 0 && t == 0) sel[3] = 0;
         __syncthreads();
         if (pass == 0) {
-            for_each_key([&](unsigned u) { atomicAdd(&hist[u >> 23], 1u); });
+            for_each_raw([&](unsigned r) { atomicAdd(&hist[r >> 23], 1u); });
         } else {
             for (unsigned j = t; j < n_cand; j += kBlock) {
                 const unsigned u = cand[j];
@@ -246,6 +249,7 @@ __device__ __forceinline__ Select radix_select_compact(int k, unsigned* hist, un
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 h[i] = hist[255 - 8 * t - i];
+                if (pass == 0) h[i] += hist[511 - 8 * t - i];  // the same binade with the sign bit set
                 c += h[i];
             }
             unsigned incl = c;
@@ -274,11 +278,12 @@ __device__ __forceinline__ Select radix_select_compact(int k, unsigned* hist, un
         eq_total = sel[2];
         if (pass == 0) {
             // this thread's elements of the chosen binade go to a range of the list reserved with one atomic
+            const unsigned binade = prefix << 23;
             unsigned mine = 0;
-            for_each_key([&](unsigned u) { mine += (u >> 23) == prefix; });
+            for_each_raw([&](unsigned r) { mine += (r & 0x7f800000u) == binade; });
             unsigned pos = mine ? atomicAdd(&sel[3], mine) : 0u;
-            for_each_key([&](unsigned u) {
-                if ((u >> 23) == prefix) cand[pos++] = u;
+            for_each_raw([&](unsigned r) {
+                if ((r & 0x7f800000u) == binade) cand[pos++] = r & 0x7fffffffu;
             });
             __syncthreads();
             n_cand = sel[3];
@@ -324,7 +329,7 @@ __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
                            float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
     constexpr bool ONE_ROW = TPR == kBlock;  // the block owns one row: candidate list in dynamic shared memory
-    __shared__ unsigned hist[G][256];
+    __shared__ unsigned hist[ONE_ROW ? 512 : G * 256];
     __shared__ unsigned sel[G][4];
     __shared__ unsigned red[kBlock / 32];
     extern __shared__ unsigned cand[];  // K words when ONE_ROW
@@ -341,10 +346,11 @@ __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
     }
     auto key = [](float f) { return __float_as_uint(f) & 0x7fffffffu; };
 
-    unsigned gmax = 0;
+    float gm = 0.f;  // max |x| as a float maximum (one instruction per element); its bits are the largest key
 #pragma unroll
-    for (int i = 0; i < V; ++i) gmax = max(max(max(gmax, key(v[i].x)), max(key(v[i].y), key(v[i].z))), key(v[i].w));
-    gmax = group_max<TPR>(gmax, red, group);
+    for (int i = 0; i < V; ++i)
+        gm = fmaxf(fmaxf(fmaxf(gm, fabsf(v[i].x)), fmaxf(fabsf(v[i].y), fabsf(v[i].z))), fabsf(v[i].w));
+    unsigned gmax = group_max<TPR>(__float_as_uint(gm), red, group);
     const double gamma = (double)__uint_as_float(gmax);
     const double mult = 127.0 / (gamma + eps);
 
@@ -359,9 +365,20 @@ __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
             }
         }
     };
+    auto for_each_raw = [&](auto f) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            if (i * TPR + t < nv) {
+                f(__float_as_uint(v[i].x));
+                f(__float_as_uint(v[i].y));
+                f(__float_as_uint(v[i].z));
+                f(__float_as_uint(v[i].w));
+            }
+        }
+    };
     Select s;
-    if constexpr (ONE_ROW) s = radix_select_compact(k, hist[0], sel[0], cand, t, for_each_key);
-    else s = radix_select<TPR>(k, hist[group], sel[group], group, t, for_each_key);
+    if constexpr (ONE_ROW) s = radix_select_compact(k, hist, sel[0], cand, t, for_each_raw);
+    else s = radix_select<TPR>(k, hist + group * 256, sel[group], group, t, for_each_key);
     const bool ordered = s.eq_total != s.keep_eq;  // a tie straddles the k-th place: lowest indices win
     unsigned running = 0;
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
