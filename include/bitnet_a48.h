@@ -172,9 +172,10 @@ size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
 /* Several BitLinears on the SAME activation codes (Eq. 6: q, k and v share the attention input; gate and up
  * share the FFN input): Y_dev[j] = BitLinear(weights[j]) for j < count, all weights with the same K.
  * For M <= 8 and count <= 4 with the DECODE layout this is one launch that streams the matrices as one
- * sequence of tiles (a launch costs more than the HBM time of one 7B-shape matrix); for more tokens, count <= 4
- * and the GEMM layout it is one launch of the tensor-core kernel over the tiles of all matrices; otherwise it
- * is `count` calls of bitnet_a48_linear one after the other.  Results are identical to separate calls.
+ * sequence of tiles (a launch costs more than the HBM time of one 7B-shape matrix); for 9..1023 tokens,
+ * count <= 4 and the GEMM layout it is one launch of the tensor-core kernel over the tiles of all matrices;
+ * otherwise it is `count` calls of bitnet_a48_linear one after the other.  Results are identical to separate
+ * calls.
  * workspace_dev: bitnet_a48_linear_multi_workspace_bytes bytes, zero-filled before first use, left zero-filled
  * (same contract as bitnet_a48_linear). */
 bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* const weights[], const int8_t* codes_dev,

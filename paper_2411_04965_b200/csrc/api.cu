@@ -269,7 +269,8 @@ bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* co
     {  // beyond the decode kernel's token count: one tensor-core launch over the tiles of all matrices
         bool any_decode = false;
         for (int j = 0; j < count; ++j) any_decode = any_decode || a48_decode_supported(weights[j], M);
-        if (!any_decode && a48_gemm_tcgen05_multi_supported(count, weights, M))
+        // (from 1024 tokens on a launch per matrix on CTA pairs is faster than the grouped single-CTA launch)
+        if (!any_decode && M < 1024 && a48_gemm_tcgen05_multi_supported(count, weights, M))
             return a48_launch_gemm_tcgen05_multi(count, weights, codes_dev, scale_dev, M, Y_dev, (cudaStream_t)stream);
     }
     for (int j = 0; j < count; ++j) {
