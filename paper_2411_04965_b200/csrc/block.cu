@@ -487,8 +487,13 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         float* gu[2] = {gate, up};
         A48_TRY(bitnet_a48_linear_multi(2, blk->w + 4, codes, scale, M, BITNET_A48_ACT_INT4, gu, lin, lin_bytes, st));
     }
-    relu2glu_kernel<<<(unsigned)((nF4 + 255) / 256), 256, 0, st>>>(gate, up, nF4);
-    A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
+    if (a48_topk_quant_fast_shape(F)) {
+        // Eq. 5 inside the quantiser's load: the product up * ReLU(gate)^2 is never written
+        A48_TRY(a48_launch_topk_quant_int8_glu(gate, up, M, F, c.k_down, c.quant_eps, codes, scale, st));
+    } else {
+        relu2glu_kernel<<<(unsigned)((nF4 + 255) / 256), 256, 0, st>>>(gate, up, nF4);
+        A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
+    }
     A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));
     add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(hres, tmp, Y, nH4);
 #undef A48_TRY

@@ -59,6 +59,9 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
                                         const float* gain, float norm_eps, cudaStream_t st);
 bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
                                              float* scale, uint32_t* mask_bits, cudaStream_t st);
+bool a48_topk_quant_fast_shape(int K);
+bitnet_a48_status a48_launch_topk_quant_int8_glu(const float* gate, const float* up, int M, int K, int k, float eps,
+                                                 int8_t* codes, float* scale, cudaStream_t st);
 bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st);
 bitnet_a48_status a48_launch_compact_codes(const int8_t* codes, int M, int K, int cap, uint16_t* idx, int8_t* val,
                                            int32_t* count, cudaStream_t st);

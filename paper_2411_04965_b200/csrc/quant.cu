@@ -323,10 +323,12 @@ __device__ __forceinline__ unsigned group_excl_scan(unsigned cnt, unsigned* red,
     return base + incl - cnt;
 }
 
-template <int TPR, int V>
+// GLU: the row to quantise is up * ReLU(gate)^2 (Eq. 5), formed while loading: X is the gate projection and U the up
+// projection, and the product never goes to memory.
+template <int TPR, int V, bool GLU>
 __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
-    topk_quant_int8_kernel(const float* __restrict__ X, int M, int K, int k, double eps, int8_t* __restrict__ codes,
-                           float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
+    topk_quant_int8_kernel(const float* __restrict__ X, const float* __restrict__ U, int M, int K, int k, double eps,
+                           int8_t* __restrict__ codes, float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
     constexpr bool ONE_ROW = TPR == kBlock;  // the block owns one row: candidate list in dynamic shared memory
     __shared__ unsigned hist[ONE_ROW ? 512 : G * 256];
@@ -343,6 +345,11 @@ __global__ void __launch_bounds__(kBlock, V >= 8 ? 4 : 6)
     for (int i = 0; i < V; ++i) {
         int idx = i * TPR + t;
         v[i] = idx < nv ? __ldg(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (GLU && idx < nv) {
+            const float4 u = __ldg(reinterpret_cast<const float4*>(U + (size_t)row * K) + idx);
+            auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
+            v[i] = make_float4(f(v[i].x, u.x), f(v[i].y, u.y), f(v[i].z, u.z), f(v[i].w, u.w));
+        }
     }
     auto key = [](float f) { return __float_as_uint(f) & 0x7fffffffu; };
 
@@ -569,22 +576,20 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
     return BITNET_A48_OK;
 }
 
-bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
-                                             float* scale, uint32_t* mask_bits, cudaStream_t st) {
+template <bool GLU>
+bitnet_a48_status launch_topk(const float* X, const float* U, int M, int K, int k, double e, int8_t* codes, float* scale,
+                              uint32_t* mask_bits, cudaStream_t st) {
     const int nv = K / 4;
-    const bool fast = (K % 4 == 0) && nv <= 256 * 12;
-    const double e = (double)eps;
 #define A48_TK(TPR, V)                                                                                              \
     do {                                                                                                            \
         const size_t dyn = TPR == kBlock ? (size_t)K * sizeof(unsigned) : 0; /* candidate list of the one-row kernels */ \
         if (dyn > 40 * 1024)                                                                                        \
-            cudaFuncSetAttribute(topk_quant_int8_kernel<TPR, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); \
-        topk_quant_int8_kernel<TPR, V><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, dyn, st>>>(X, M, K, k, e,  \
-                                                                                                    codes, scale,   \
-                                                                                                    mask_bits);     \
+            cudaFuncSetAttribute(topk_quant_int8_kernel<TPR, V, GLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
+                                 64 * 1024);                                                                        \
+        topk_quant_int8_kernel<TPR, V, GLU><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, dyn, st>>>(         \
+            X, U, M, K, k, e, codes, scale, mask_bits);                                                             \
     } while (0)
-    if (!fast) topk_quant_int8_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, k, e, codes, scale, mask_bits);
-    else if (nv <= 32 * 4) A48_TK(32, 4);
+    if (nv <= 32 * 4) A48_TK(32, 4);
     else if (nv <= 64 * 4) A48_TK(64, 4);
     else if (nv <= 128 * 4) A48_TK(128, 4);
     else if (nv <= 256 * 4) A48_TK(256, 4);
@@ -593,6 +598,23 @@ bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k
 #undef A48_TK
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
+}
+
+bool a48_topk_quant_fast_shape(int K) { return (K % 4 == 0) && K / 4 <= 256 * 12; }
+
+bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
+                                             float* scale, uint32_t* mask_bits, cudaStream_t st) {
+    if (a48_topk_quant_fast_shape(K)) return launch_topk<false>(X, nullptr, M, K, k, (double)eps, codes, scale, mask_bits, st);
+    topk_quant_int8_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, k, (double)eps, codes, scale, mask_bits);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+// Top-K + INT8 of up * ReLU(gate)^2 (Eq. 5 fused into the quantiser's load); shapes of the register kernels only.
+bitnet_a48_status a48_launch_topk_quant_int8_glu(const float* gate, const float* up, int M, int K, int k, float eps,
+                                                 int8_t* codes, float* scale, cudaStream_t st) {
+    if (!a48_topk_quant_fast_shape(K)) return BITNET_A48_ERR_UNSUPPORTED;
+    return launch_topk<true>(gate, up, M, K, k, (double)eps, codes, scale, nullptr, st);
 }
 
 bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st) {
