@@ -480,9 +480,13 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     A48_TRY(a48_launch_topk_quant_int8(att, M, H, c.k_o, c.quant_eps, codes, scale, nullptr, st));
     A48_TRY(linear(3, BITNET_A48_ACT_TOPK_INT8, tmp));
     const size_t nH4 = (size_t)M * H / 4, nF4 = (size_t)M * F / 4;
-    add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
-    // feed-forward sub-layer
-    A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+    // feed-forward sub-layer: h = x + attention output, formed (and written for the last residual) in the quantiser's load
+    if (a48_topk_quant_fast_shape(H)) {
+        A48_TRY(a48_launch_quant_int4_add(X, tmp, hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+    } else {
+        add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
+        A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+    }
     {
         float* gu[2] = {gate, up};
         A48_TRY(bitnet_a48_linear_multi(2, blk->w + 4, codes, scale, M, BITNET_A48_ACT_INT4, gu, lin, lin_bytes, st));

@@ -60,6 +60,9 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
 bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
                                              float* scale, uint32_t* mask_bits, cudaStream_t st);
 bool a48_topk_quant_fast_shape(int K);
+bitnet_a48_status a48_launch_quant_int4_add(const float* X, const float* R, float* SUM, int M, int K, float eps,
+                                            int8_t* codes, float* scale, const float* gain, float norm_eps,
+                                            cudaStream_t st);
 bitnet_a48_status a48_launch_topk_quant_int8_glu(const float* gate, const float* up, int M, int K, int k, float eps,
                                                  int8_t* codes, float* scale, cudaStream_t st);
 bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st);

@@ -87,10 +87,12 @@ __device__ __forceinline__ void rmsnorm_inplace(float4 (&v)[V], int t, int nv, i
 }
 
 // ---------------------------------------------------------------------------- Eq. 7
-template <int TPR, int V, bool NORM>
+// ADD: the row is X + R (a residual connection), formed while loading and written to SUM for the later residual.
+template <int TPR, int V, bool NORM, bool ADD>
 __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restrict__ X, int M, int K, double eps,
                                                             int8_t* __restrict__ codes, float* __restrict__ scale,
-                                                            const float* __restrict__ gain, double norm_eps) {
+                                                            const float* __restrict__ gain, double norm_eps,
+                                                            const float* __restrict__ R, float* __restrict__ SUM) {
     constexpr int G = kBlock / TPR;
     __shared__ double red[kBlock / 32];
     const int group = threadIdx.x / TPR, t = threadIdx.x % TPR;
@@ -103,6 +105,11 @@ __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restr
     for (int i = 0; i < V; ++i) {
         int idx = i * TPR + t;
         v[i] = idx < nv ? __ldg(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ADD && idx < nv) {
+            const float4 r = __ldg(reinterpret_cast<const float4*>(R + (size_t)row * K) + idx);
+            v[i] = make_float4(v[i].x + r.x, v[i].y + r.y, v[i].z + r.z, v[i].w + r.w);
+            reinterpret_cast<float4*>(SUM + (size_t)row * K)[idx] = v[i];
+        }
     }
     if (NORM) rmsnorm_inplace<TPR, V>(v, t, nv, K, gain, norm_eps, red, group);
     double s = 0.0;
@@ -548,14 +555,14 @@ __global__ void __launch_bounds__(kBlock) compact_codes_kernel(const int8_t* __r
     if (t == 0) count[row] = (int32_t)running;
 }
 
-template <bool NORM>
+template <bool NORM, bool ADD = false>
 void launch_int4(const float* X, int M, int K, double eps, int8_t* codes, float* scale, const float* gain,
-                 double norm_eps, cudaStream_t st) {
+                 double norm_eps, cudaStream_t st, const float* R = nullptr, float* SUM = nullptr) {
     const int nv = K / 4;
     const bool fast = (K % 4 == 0) && nv <= 256 * 12;
-#define A48_Q4(TPR, V)                                                                                      \
-    quant_int4_kernel<TPR, V, NORM><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(X, M, K, eps, codes, \
-                                                                                               scale, gain, norm_eps)
+#define A48_Q4(TPR, V)                                                                                           \
+    quant_int4_kernel<TPR, V, NORM, ADD><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(         \
+        X, M, K, eps, codes, scale, gain, norm_eps, R, SUM)
     if (!fast) quant_int4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, eps, codes, scale, gain, norm_eps);
     else if (nv <= 32 * 4) A48_Q4(32, 4);
     else if (nv <= 64 * 4) A48_Q4(64, 4);
@@ -572,6 +579,17 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
                                         const float* gain, float norm_eps, cudaStream_t st) {
     if (gain) launch_int4<true>(X, M, K, (double)eps, codes, scale, gain, (double)norm_eps, st);
     else launch_int4<false>(X, M, K, (double)eps, codes, scale, nullptr, 0.0, st);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+// RMSNorm + INT4 of X + R with the sum written to SUM (the residual add fused into the quantiser's load); shapes of
+// the register kernels only.
+bitnet_a48_status a48_launch_quant_int4_add(const float* X, const float* R, float* SUM, int M, int K, float eps,
+                                            int8_t* codes, float* scale, const float* gain, float norm_eps,
+                                            cudaStream_t st) {
+    if (!((K % 4 == 0) && K / 4 <= 256 * 12) || !gain) return BITNET_A48_ERR_UNSUPPORTED;
+    launch_int4<true, true>(X, M, K, (double)eps, codes, scale, gain, (double)norm_eps, st, R, SUM);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }
