@@ -59,10 +59,11 @@ __global__ void rope_table_kernel(int pos0, int T, int half, double base, float2
 }
 
 // Rotates q in place on (i, i+hd/2) pairs, rotates k, and stores rotated k and v
-// into the cache rows [b][h][pos0+t][:].
+// into the cache rows [b][h][pos0+t][:].  table == nullptr (a few tokens): the angle is evaluated here, with the
+// expression of rope_table_kernel, instead of in a launch of its own.
 __global__ void rope_cache_kernel(float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
-                                  const float2* __restrict__ table, int B, int T, int nh, int hd, int pos0, int cap,
-                                  float* __restrict__ kcache, float* __restrict__ vcache) {
+                                  const float2* __restrict__ table, double base, int B, int T, int nh, int hd, int pos0,
+                                  int cap, float* __restrict__ kcache, float* __restrict__ vcache) {
     const int half = hd / 2;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     size_t total = (size_t)B * T * nh * half;
@@ -71,7 +72,15 @@ __global__ void rope_cache_kernel(float* __restrict__ q, const float* __restrict
     int h = (int)((idx / half) % nh);
     size_t m = idx / ((size_t)half * nh);
     int t = (int)(m % T), b = (int)(m / T);
-    float2 cs = table[t * half + i];
+    float2 cs;
+    if (table) {
+        cs = table[t * half + i];
+    } else {
+        double ang = (double)(pos0 + t) * pow(base, -(double)i / (double)half);
+        double sn, cn;
+        sincos(ang, &sn, &cn);
+        cs = make_float2((float)cn, (float)sn);
+    }
     size_t src = m * (size_t)nh * hd + (size_t)h * hd + i;
     float ql = q[src], qh = q[src + half];
     q[src] = ql * cs.x - qh * cs.y;
@@ -461,9 +470,11 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     }
     {
         int n = T * (hd / 2);
-        rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
+        const bool inline_angles = T <= 8;  // decode: every thread evaluates its own angle, one launch fewer
+        if (!inline_angles) rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
         size_t total = (size_t)M * nh * (hd / 2);
-        rope_cache_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(q, k, v, rope, B, T, nh, hd, pos0, cap,
+        rope_cache_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(q, k, v, inline_angles ? nullptr : rope,
+                                                                          (double)c.rope_base, B, T, nh, hd, pos0, cap,
                                                                           kcache, vcache);
     }
     if (T <= 8) {
