@@ -48,6 +48,27 @@ STEP_OPS = sum(2 * M_PREFILL * n * k for _, n, k, _ in PROJ)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 3.53e8
 
 
+def library_int8_tops(dev, stream):
+    """Dense int8 GEMM of the vendor library on this GPU, as a second reference beside the measured bf16 figure."""
+    try:
+        n = 8192
+        a = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=dev)
+        b = torch.randint(-1, 2, (n, n), dtype=torch.int8, device=dev).t()  # column-major second operand
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record(stream)
+        for _ in range(reps):
+            torch._int_mm(a, b)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return 2.0 * n ** 3 / (e0.elapsed_time(e1) / reps * 1e-3) / 1e12
+    except Exception:  # not every build has the int8 library path
+        return None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -337,6 +358,10 @@ def run_ours(args):
                 "avg_launch_ms": gemm_ms / len(gemm_events),
                 "peak_source": f"2 x {peak_kind} of {peaks['source']} peaks (no int8 peak is measured; nominal int8:bf16 = 2)",
                 "timed_region_ms": ms_total}
+    lib = library_int8_tops(dev, stream) if rank == 0 else None
+    if lib:
+        roofline["library_int8_tops"] = lib
+        roofline["library_int8_note"] = "torch._int_mm (vendor int8 GEMM) 8192^3, 20 calls, same GPU, outside the timed region"
 
     # ---- end to end with host buffers (pinned), copies inside the timed region
     e2e = None
