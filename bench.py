@@ -1,18 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the BitNet a4.8 BitLinear forward on B200.
 
-One step = the seven BitLinears of one 7B-shape transformer layer over 16384
+One pass = the seven BitLinears of one 7B-shape transformer layer over 16384
 tokens (prefill of 4096 tokens x batch 4): the per-token quantisers (INT4 for
 the q/k/v and gate/up inputs, top-K 50 % + INT8 for the o and down inputs)
-followed by the packed-ternary contractions and their rescale.  The headline
-value is dense-equivalent TOPS (2*M*N*K summed over the seven projections,
-divided by the step time, quantisers included).  The same JSON line also
-carries the batch-1 decode figure (GB/s of packed weight bytes streamed over
-every matrix of the 32-layer model), block tokens/s, the roofline of the
-dominant kernel, the end-to-end figure with host buffers, and the CPU oracle
-timed on a bounded sample.
+followed by the packed-ternary contractions and their rescale.  A counted step
+is `passes_per_step` such passes, chosen so that the timed region lasts at
+least a second whatever --steps says (the GPU then runs at the clock its power
+cap leaves, not at a cold burst).  The headline value is dense-equivalent TOPS
+(2*M*N*K summed over the seven projections, divided by the time of a pass,
+quantisers included).  The same JSON line also carries the roofline of every
+rated kernel, the end-to-end figure with host buffers, the CPU oracle timed on
+a bounded sample, and one leg per remaining benchmark configuration: the decode
+chains of the 7B and 3B shapes at 1/8/32/64 tokens, the 700M-shape prefill, the
+M = 1..16384 sweep of the isolated BitLinear, and block tokens/s.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--legs a,b,...]
 
 For N > 1 launch with torch.distributed.run; every rank runs an independent
 replica (tokens shard with no exchange), so scaling is weak.
@@ -41,11 +44,23 @@ PROJ = (("q", H, H, "int4"), ("k", H, H, "int4"), ("v", H, H, "int4"), ("o", H, 
         ("gate", F, H, "int4"), ("up", F, H, "int4"), ("down", H, F, "topk"))
 STEP_OPS = sum(2 * M_PREFILL * n * k for _, n, k, _ in PROJ)
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum).
-# Capture: profiles/gemm_pair_prefill_M4096_N11008_K4096.md (150.9 MB of DRAM traffic against 208.5 MB of
-# algorithmic bytes at M=4096, part of the output still in L2 at kernel end), scaled to the mean algorithmic bytes
-# of the seven launches of a step at M=16384 (488 MB): traffic grows with M like the algorithmic bytes do.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 3.53e8
+# DRAM bytes per launch of the prefill contraction (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
+# of the CTA-pair kernel at M = 4096, N = 11008, K = 4096: 150.9 MB against 208.5 MB of algorithmic bytes, part of
+# the output still in L2 when the kernel ends), scaled by the units processed: x (488 MB / 208.5 MB), the mean
+# algorithmic bytes M*K + N*K/4 + 4*M*N of the seven launches of a pass at M = 16384 over those of the captured case.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 150.9e6 * (488.0 / 208.5)
+NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part (2 x the 2.25 PFLOP/s dense bf16 figure)
+
+# the other shapes of the paper's model-configuration table used by the legs
+SHAPE_3B = dict(H=3200, F=8640, NH=32, LAYERS=26)
+SHAPE_700M = dict(H=1536, F=4096, NH=16, LAYERS=24)  # 16 heads as the benchmark configuration fixes (head dim 96)
+SHAPE_7B = dict(H=H, F=F, NH=NH, LAYERS=LAYERS)
+ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "cpu")
+
+
+def proj_list(Hs, Fs):
+    return (("q", Hs, Hs, "int4"), ("k", Hs, Hs, "int4"), ("v", Hs, Hs, "int4"), ("o", Hs, Hs, "topk"),
+            ("gate", Fs, Hs, "int4"), ("up", Fs, Hs, "int4"), ("down", Hs, Fs, "topk"))
 
 
 def library_int8_tops(dev, stream):
@@ -256,16 +271,80 @@ class Replicas:
 
 # --------------------------------------------------------------------------- our arm
 class Layer:
-    """Packed weights of one 7B-shape layer plus resident activation buffers."""
+    """Packed weights of one transformer layer of a given shape."""
 
-    def __init__(self, a48, dev, seed, layouts):
+    def __init__(self, a48, dev, seed, layouts, Hs=H, Fs=F):
         from paper_2411_04965_b200 import synth
         self.w = {}
-        for i, (name, n, k, _) in enumerate(PROJ):
+        for i, (name, n, k, _) in enumerate(proj_list(Hs, Fs)):
             lat = synth.ternary_latents(n, k, seed=seed * 16 + i, device=dev)
             self.w[name] = a48.pack_ternary(lat, EPS, layouts)
             del lat
         torch.cuda.synchronize()
+
+    def free(self):
+        for w in self.w.values():
+            w.free()
+
+
+class LayerStep:
+    """The seven BitLinears of one layer on resident buffers: 4 quantiser launches and 7 contractions per pass."""
+
+    KERNELS = ("int4_h", "q", "k", "v", "topk_h", "o", "int4_h2", "gate", "up", "topk_f", "down")
+
+    def __init__(self, a48, synth, dev, layer, M, Hs, Fs, seed):
+        self.a48, self.layer, self.M, self.H, self.F = a48, layer, M, Hs, Fs
+        self.x_h = synth.gaussian_outlier_activations(M, Hs, seed=seed, device=dev)
+        self.s_h = synth.student_t3(M, Hs, seed=seed + 1, device=dev)
+        self.s_f = synth.student_t3(M, Fs, seed=seed + 2, device=dev)
+        self.codes_h = torch.empty(M, Hs, dtype=torch.int8, device=dev)
+        self.codes_f = torch.empty(M, Fs, dtype=torch.int8, device=dev)
+        self.scale = torch.empty(M, dtype=torch.float32, device=dev)
+        self.y_h = torch.empty(M, Hs, dtype=torch.float32, device=dev)
+        self.y_f = torch.empty(M, Fs, dtype=torch.float32, device=dev)
+        ws_need = max([a48.linear_workspace_bytes(w, M) for w in layer.w.values()] + [16])
+        self.ws = torch.zeros(ws_need, dtype=torch.uint8, device=dev)
+        self.ops = sum(2 * M * n * k for _, n, k, _ in proj_list(Hs, Fs))
+
+    def run(self, stream, events=None):
+        """One pass.  events: a list that receives one CUDA event before every launch and one after the last."""
+        a48, w = self.a48, self.layer.w
+
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(stream)
+                events.append(e)
+
+        def lin(name, codes, kind, out):
+            mark()
+            a48.linear(w[name], codes, self.scale, kind, a48.ALGO_AUTO, Y=out, workspace=self.ws)
+
+        mark()
+        a48.quant_int4(self.x_h, EPS, self.codes_h, self.scale)
+        for name in ("q", "k", "v"):
+            lin(name, self.codes_h, a48.ACT_INT4, self.y_h)
+        mark()
+        a48.topk_quant_int8(self.s_h, self.H // 2, EPS, self.codes_h, self.scale)
+        lin("o", self.codes_h, a48.ACT_TOPK_INT8, self.y_h)
+        mark()
+        a48.quant_int4(self.x_h, EPS, self.codes_h, self.scale)
+        for name in ("gate", "up"):
+            lin(name, self.codes_h, a48.ACT_INT4, self.y_f)
+        mark()
+        a48.topk_quant_int8(self.s_f, self.F // 2, EPS, self.codes_f, self.scale)
+        lin("down", self.codes_f, a48.ACT_TOPK_INT8, self.y_h)
+        mark()
+        return len(self.KERNELS)  # kernel launches of this library per pass
+
+
+def per_kernel_ms(pass_events):
+    """Mean duration per kernel name over all passes: events sit before every launch and after the last."""
+    sums = {}
+    for ev in pass_events:
+        for name, a, b in zip(LayerStep.KERNELS, ev[:-1], ev[1:]):
+            sums.setdefault(name, []).append(a.elapsed_time(b))
+    return {k: sum(v) / len(v) for k, v in sums.items()}
 
 
 def run_ours(args):
@@ -285,6 +364,12 @@ def run_ours(args):
     peaks = load_peaks()
     M = M_PREFILL
     stream = torch.cuda.current_stream()
+    legs = set(ALL_LEGS if args.legs == "all" else [l for l in args.legs.split(",") if l])
+    unknown = legs - set(ALL_LEGS)
+    if unknown:
+        raise SystemExit(f"unknown legs {sorted(unknown)}; known: {ALL_LEGS}")
+    if world > 1:  # the legs are single-GPU figures; every rank of a multi-GPU run would only repeat them
+        legs &= {"e2e"}
 
     def barrier():
         reps.barrier()
@@ -292,127 +377,110 @@ def run_ours(args):
 
     max_over_ranks = reps.max_ms
 
-    # ---- resident inputs: larger than L2 (268 MB + 268 MB + 721 MB of fp32 activations per step)
+    # ---- resident inputs: larger than L2 (268 MB + 268 MB + 721 MB of fp32 activations per pass)
     layer = Layer(a48, dev, seed=4 + rank, layouts=a48.LAYOUT_ALL)
-    x_h = synth.gaussian_outlier_activations(M, H, seed=40 + rank, device=dev)
-    s_h = synth.student_t3(M, H, seed=41 + rank, device=dev)
-    s_f = synth.student_t3(M, F, seed=42 + rank, device=dev)
-    codes_h = torch.empty(M, H, dtype=torch.int8, device=dev)
-    codes_f = torch.empty(M, F, dtype=torch.int8, device=dev)
-    scale = torch.empty(M, dtype=torch.float32, device=dev)
-    y_h = torch.empty(M, H, dtype=torch.float32, device=dev)
-    y_f = torch.empty(M, F, dtype=torch.float32, device=dev)
-    gemm_events = []
-
-    def gemm(name, codes, kind, out, record):
-        if record:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-        a48.linear(layer.w[name], codes, scale, kind, a48.ALGO_AUTO, Y=out)
-        if record:
-            e1.record(stream)
-            gemm_events.append((name, e0, e1))
-
-    def step(record=False):
-        a48.quant_int4(x_h, EPS, codes_h, scale)
-        for name in ("q", "k", "v"):
-            gemm(name, codes_h, a48.ACT_INT4, y_h, record)
-        a48.topk_quant_int8(s_h, H // 2, EPS, codes_h, scale)
-        gemm("o", codes_h, a48.ACT_TOPK_INT8, y_h, record)
-        a48.quant_int4(x_h, EPS, codes_h, scale)
-        for name in ("gate", "up"):
-            gemm(name, codes_h, a48.ACT_INT4, y_f, record)
-        a48.topk_quant_int8(s_f, F // 2, EPS, codes_f, scale)
-        gemm("down", codes_f, a48.ACT_TOPK_INT8, y_h, record)
-        return 11  # kernel launches of this library per step
+    work = LayerStep(a48, synth, dev, layer, M, H, F, seed=40 + rank)
 
     sampler = ClockSampler(dev)
     sampler.start()
-    for _ in range(args.warmup):
-        step()
-    barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    work.run(stream)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(max(args.warmup, 3)):
+        work.run(stream)
+    e1.record(stream)
+    barrier()
+    est_ms = max_over_ranks(e0.elapsed_time(e1) / max(args.warmup, 3))
+    # a counted step repeats the pass so that steps x passes x pass time >= the wanted length of the timed region
+    passes = max(1, int(-(-args.min_region_ms // (args.steps * est_ms))))
+    pass_events = []
     barrier()
     t_begin = time.time()
     e0.record(stream)
     launches = 0
     for _ in range(args.steps):
-        launches += step(record=True)
+        for _ in range(passes):
+            ev = []
+            launches += work.run(stream, ev)
+            pass_events.append(ev)
     e1.record(stream)
     barrier()
     t_end = time.time()
     clocks = sampler.stop(t_begin, t_end)
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     ms_per_step = ms_total / args.steps
-    tops = reps.job_value(STEP_OPS, ms_per_step) / 1e12
+    ms_per_pass = ms_per_step / passes
+    tops = reps.job_value(STEP_OPS, ms_per_pass) / 1e12
+    n_burst = min(20, len(pass_events))
+    burst_ms = pass_events[0][0].elapsed_time(pass_events[n_burst - 1][-1]) / n_burst
+    n_tail = max(1, len(pass_events) // 2)
+    tail_ms = pass_events[-n_tail][0].elapsed_time(pass_events[-1][-1]) / n_tail
 
-    gemm_ms = sum(a.elapsed_time(b) for _, a, b in gemm_events)
-    gemm_ops = sum(2 * M * n * k for name, _, _ in gemm_events for pn, n, k, _ in PROJ if pn == name)
+    kms = per_kernel_ms(pass_events)
+    gemm_names = ("q", "k", "v", "o", "gate", "up", "down")
+    gemm_ms = sum(kms[n] for n in gemm_names)
+    gemm_ops = sum(2 * M * n * k for pn, n, k, _ in PROJ if pn in gemm_names)
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
-    # nominal int8:bf16 ratio of 2 on the measured bf16 figure: sustained for a region of a second or more, else burst
+    # second denominator: nominal int8:bf16 ratio of 2 on the measured bf16 figure (sustained for a region >= 1 s)
     peak_kind = "bf16_tflops_sustained" if ms_total >= 1000.0 else "bf16_tflops"
-    int8_peak = 2.0 * peaks[peak_kind]
-    roofline = {"bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
-                "frac": achieved / int8_peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                "kernel": "BitLinear contraction (prefill)", "launches": len(gemm_events),
-                "avg_launch_ms": gemm_ms / len(gemm_events),
-                "peak_source": f"2 x {peak_kind} of {peaks['source']} peaks (no int8 peak is measured; nominal int8:bf16 = 2)",
+    measured_x2 = 2.0 * peaks[peak_kind]
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": NOMINAL_INT8_TOPS, "unit": "TOPS",
+                "frac": achieved / NOMINAL_INT8_TOPS, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "kernel": "BitLinear contraction (prefill, tcgen05 kind::i8 on CTA pairs)",
+                "launches": 7 * len(pass_events), "avg_launch_ms": gemm_ms / 7,
+                "peak_source": "nominal dense int8 tensor peak of the part (no int8 peak is measured on this pool)",
+                "peak_measured_x2": measured_x2, "frac_of_measured": achieved / measured_x2,
+                "peak_measured_source": f"2 x {peak_kind} of {peaks['source']} peaks (nominal int8:bf16 = 2)",
                 "timed_region_ms": ms_total}
     lib = library_int8_tops(dev, stream) if rank == 0 else None
     if lib:
         roofline["library_int8_tops"] = lib
         roofline["library_int8_note"] = "torch._int_mm (vendor int8 GEMM) 8192^3, 20 calls, same GPU, outside the timed region"
 
+    def hbm_entry(kernel, names, K):
+        ms = sum(kms[n] for n in names) / len(names)
+        bytes_ = 5.0 * M * K + 4.0 * M  # fp32 in, int8 out, one fp32 scale per token
+        gbs = bytes_ / (ms * 1e-3) / 1e9
+        return {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "traffic": None, "avg_launch_ms": ms,
+                "launches": len(names) * len(pass_events), "algorithmic_bytes_per_launch": bytes_,
+                "peak_source": f"hbm_gbs of {peaks['source']} peaks"}
+
+    rooflines = [dict(roofline),
+                 hbm_entry("top-K + INT8 quantiser, 16384 x 11008 (Eq. 1, 3)", ("topk_f",), F),
+                 hbm_entry("top-K + INT8 quantiser, 16384 x 4096 (Eq. 1, 3)", ("topk_h",), H),
+                 hbm_entry("INT4 quantiser, 16384 x 4096 (Eq. 7)", ("int4_h", "int4_h2"), H)]
+
     # ---- end to end with host buffers (pinned), copies inside the timed region
-    e2e = None
-    if not args.skip_e2e:
-        xh_host = x_h.cpu().pin_memory()
-        sh_host = s_h.cpu().pin_memory()
-        sf_host = s_f.cpu().pin_memory()
-        calls = (("q", xh_host, a48.ACT_INT4, 0), ("k", xh_host, a48.ACT_INT4, 0), ("v", xh_host, a48.ACT_INT4, 0),
-                 ("o", sh_host, a48.ACT_TOPK_INT8, H // 2), ("gate", xh_host, a48.ACT_INT4, 0),
-                 ("up", xh_host, a48.ACT_INT4, 0), ("down", sf_host, a48.ACT_TOPK_INT8, F // 2))
-        outs = {name: torch.empty(M, layer.w[name].N, dtype=torch.float32).pin_memory() for name, *_ in calls}
-        ws_bytes = max(a48.bitlinear_host_workspace_bytes(layer.w[n], M) for n, *_ in PROJ)
-        # three streams, each with its own workspace: the upload of one call, the kernels of another and the
-        # download of a third run at the same time (every call still uploads its input and downloads its output)
-        e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
-        wss = [torch.zeros(ws_bytes, dtype=torch.uint8, device=dev) for _ in e2e_streams]
+    e2e = bench_e2e(a48, dev, layer, work, reps, barrier, args) if "e2e" in legs else None
+    del work
+    torch.cuda.empty_cache()
 
-        def step_host():
-            for i, (name, xin, kind, k) in enumerate(calls):
-                j = i % len(e2e_streams)
-                a48.bitlinear_host_async(layer.w[name], xin, outs[name], kind, k, EPS, wss[j], stream=e2e_streams[j])
-            for st_ in e2e_streams:
-                st_.synchronize()
-
-        step_host()
-        barrier()
-        n_e2e = max(1, min(args.steps, 3))
-        t0 = time.perf_counter()
-        for _ in range(n_e2e):
-            step_host()
-        barrier()
-        dt = max_over_ranks((time.perf_counter() - t0) * 1e3) / n_e2e
-        h2d = 6 * M * H * 4 + M * F * 4
-        d2h = 5 * M * H * 4 + 2 * M * F * 4
-        e2e = {"value": STEP_OPS * world / (dt * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "ms_per_step": dt, "steps": n_e2e,
-               "api": "bitnet_a48_bitlinear_host_async on 3 streams, pinned host buffers, stream sync per step"}
-        del xh_host, sh_host, sf_host, outs, wss
-
-    # ---- batch-1 decode over every matrix of the model (distinct buffers >> L2)
-    decode = None
-    if not args.skip_decode:
-        decode = bench_decode(a48, synth, dev, stream, peaks, rank)
-
-    # ---- block forward tokens/s
-    block = None
-    if not args.skip_block:
+    decode = decode3b = prefill700m = sweep = block = None
+    if "decode7b" in legs:
+        decode = bench_decode(a48, synth, dev, stream, peaks, rank, SHAPE_7B, "7b")
+        one = decode["by_tokens"]["1"]
+        rooflines.append({"kernel": "decode BitLinear chain, 7B shape, 1 token (224 matrices, CUDA graph)", "bound": "hbm",
+                          "achieved": one["algorithmic_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": one["algorithmic_gbs"] / peaks["hbm_gbs"], "traffic": None,
+                          "dense_gbs": one["weight_stream_gbs"],
+                          "dense_frac": one["weight_stream_gbs"] / peaks["hbm_gbs"],
+                          "note": "rated on algorithmic bytes (weight rows of channels with a non-zero code); "
+                                  "dense_gbs counts every packed byte the kernel streams",
+                          "peak_source": f"hbm_gbs of {peaks['source']} peaks"})
+    if "decode3b" in legs:
+        decode3b = bench_decode(a48, synth, dev, stream, peaks, rank, SHAPE_3B, "3b")
+        decode3b["block"] = bench_block_decode(a48, synth, dev, stream, SHAPE_3B, (1, 8, 32, 64))
+    if "prefill700m" in legs:
+        prefill700m = bench_prefill_700m(a48, synth, dev, stream)
+    if "sweep" in legs:
+        sweep = bench_sweep(a48, synth, dev, stream)
+    if "block" in legs:
         block = bench_block(a48, synth, dev, stream, layer)
 
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.skip_cpu:
+    if rank == 0 and world == 1 and "cpu" in legs:
         from oracle import oracle_a48 as oracle
         oracle.build()
         cores = len(os.sched_getaffinity(0))
@@ -424,40 +492,108 @@ def run_ours(args):
     if rank == 0:
         line = {
             "metric": "bitlinear_prefill_tops_7b", "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8 x int2 -> int32 (scales fp64/fp32)", "data": "synthetic",
             "config": {"workload": "7B-shape layer (hidden 4096, GLU 11008): 7 BitLinears incl. quantisers, "
                                    "prefill 4096 tokens x batch 4 = 16384 tokens",
-                       "l2": "inputs larger than L2 (1.26 GB of fp32 activations + 1.3 GB of outputs per step)",
+                       "passes_per_step": passes, "ms_per_pass": ms_per_pass,
+                       "l2": "inputs larger than L2 (1.26 GB of fp32 activations + 1.3 GB of outputs per pass)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e,
-            "cpu_baseline": cpu_baseline, "decode": decode, "block": block,
+            "sustained": {"ms_per_pass": tail_ms, "tops": STEP_OPS / (tail_ms * 1e-3) / 1e12,
+                          "window": f"last {n_tail} passes of the timed region"},
+            "first_burst": {"ms_per_pass": burst_ms, "tops": STEP_OPS / (burst_ms * 1e-3) / 1e12,
+                            "window": f"first {n_burst} passes of the timed region"},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "rooflines": rooflines, "e2e": e2e,
+            "cpu_baseline": cpu_baseline, "decode": decode, "decode_3b": decode3b, "prefill_700m": prefill700m,
+            "sweep": sweep, "block": block,
         }
         print(json.dumps(line))
     reps.close()
 
 
-def bench_decode(a48, synth, dev, stream, peaks, rank):
-    """BitLinear chain over all 7 x 32 matrices of the 7B shape, one CUDA graph per token count (1, 8, 32, 64)."""
+def bench_e2e(a48, dev, layer, work, reps, barrier, args):
+    """The same pass through the host-buffer entry point: every call uploads its input and downloads its output."""
+    M = work.M
+    xh_host = work.x_h.cpu().pin_memory()
+    sh_host = work.s_h.cpu().pin_memory()
+    sf_host = work.s_f.cpu().pin_memory()
+    calls = (("q", xh_host, a48.ACT_INT4, 0), ("k", xh_host, a48.ACT_INT4, 0), ("v", xh_host, a48.ACT_INT4, 0),
+             ("o", sh_host, a48.ACT_TOPK_INT8, H // 2), ("gate", xh_host, a48.ACT_INT4, 0),
+             ("up", xh_host, a48.ACT_INT4, 0), ("down", sf_host, a48.ACT_TOPK_INT8, F // 2))
+    outs = {name: torch.empty(M, layer.w[name].N, dtype=torch.float32).pin_memory() for name, *_ in calls}
+    ws_bytes = max(a48.bitlinear_host_workspace_bytes(layer.w[n], M) for n, *_ in PROJ)
+    # three streams, each with its own workspace: the upload of one call, the kernels of another and the
+    # download of a third run at the same time (every call still uploads its input and downloads its output)
+    e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
+    wss = [torch.zeros(ws_bytes, dtype=torch.uint8, device=dev) for _ in e2e_streams]
+
+    def step_host():
+        for i, (name, xin, kind, k) in enumerate(calls):
+            j = i % len(e2e_streams)
+            a48.bitlinear_host_async(layer.w[name], xin, outs[name], kind, k, EPS, wss[j], stream=e2e_streams[j])
+        for st_ in e2e_streams:
+            st_.synchronize()
+
+    step_host()
+    barrier()
+    n_e2e = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        step_host()
+    barrier()
+    dt = reps.max_ms((time.perf_counter() - t0) * 1e3) / n_e2e
+    h2d = 6 * M * H * 4 + M * F * 4
+    d2h = 5 * M * H * 4 + 2 * M * F * 4
+    return {"value": STEP_OPS * reps.world / (dt * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": dt, "steps": n_e2e,
+            "api": "bitnet_a48_bitlinear_host_async on 3 streams, pinned host buffers, stream sync per step"}
+
+
+def graph_time_ms(fn, stream, reps, warm=3):
+    """Captures fn() once in a CUDA graph on a side stream and returns the mean replay time."""
+    fn()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            fn(side)
+    torch.cuda.synchronize()
+    for _ in range(warm):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    del graph
+    return ms
+
+
+def bench_decode(a48, synth, dev, stream, peaks, rank, shape, tag):
+    """BitLinear chain over all 7 x LAYERS matrices of a model shape, one CUDA graph per token count (1, 8, 32, 64)."""
+    Hs, Fs, layers = shape["H"], shape["F"], shape["LAYERS"]
+    projs = proj_list(Hs, Fs)
     weights = []
-    for layer_i in range(LAYERS):
-        for i, (name, n, k, kind) in enumerate(PROJ):
+    for layer_i in range(layers):
+        for i, (name, n, k, kind) in enumerate(projs):
             lat = synth.ternary_latents(n, k, seed=1000 + layer_i * 8 + i + 7000 * rank, device=dev)
-            weights.append((a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE | a48.LAYOUT_SPARSE | a48.LAYOUT_GEMM), n, k, kind))
+            weights.append((a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE | a48.LAYOUT_GEMM), n, k, kind))
             del lat
     packed_bytes = sum(w.packed_bytes for w, *_ in weights)
-    fused = not os.environ.get("A48_BENCH_DECODE_UNFUSED")
 
     def time_chain(M):
-        x_h = synth.gaussian_outlier_activations(M, H, seed=50, device=dev)
-        s_h = synth.student_t3(M, H, seed=51, device=dev)
-        s_f = synth.student_t3(M, F, seed=52, device=dev)
+        x_h = synth.gaussian_outlier_activations(M, Hs, seed=50, device=dev)
+        s_h = synth.student_t3(M, Hs, seed=51, device=dev)
+        s_f = synth.student_t3(M, Fs, seed=52, device=dev)
         c4, d4 = a48.quant_int4(x_h, EPS)
-        c8h, d8h, _ = a48.topk_quant_int8(s_h, H // 2, EPS)
-        c8f, d8f, _ = a48.topk_quant_int8(s_f, F // 2, EPS)
-        y = torch.empty(M, F, dtype=torch.float32, device=dev)
-        ys = [torch.empty(M, F, dtype=torch.float32, device=dev) for _ in range(3)]
-        yh = [torch.empty(M, H, dtype=torch.float32, device=dev) for _ in range(3)]
+        c8h, d8h, _ = a48.topk_quant_int8(s_h, Hs // 2, EPS)
+        c8f, d8f, _ = a48.topk_quant_int8(s_f, Fs // 2, EPS)
+        ys = [torch.empty(M, Fs, dtype=torch.float32, device=dev) for _ in range(2)]
+        yh = [torch.empty(M, Hs, dtype=torch.float32, device=dev) for _ in range(3)]
         ws_need = max(a48.linear_workspace_bytes(w, M) for w, *_ in weights[:7])
         ws_multi = max(a48.linear_multi_workspace_bytes([w for w, *_ in weights[0:3]], M),
                        a48.linear_multi_workspace_bytes([w for w, *_ in weights[4:6]], M), ws_need, 16)
@@ -467,76 +603,150 @@ def bench_decode(a48, synth, dev, stream, peaks, rank):
               "topk_f": float((c8f != 0).any(0).float().mean())}
         needed_bytes = 0
         for w, n, k, kind in weights:
-            needed_bytes += w.packed_bytes * (nz["int4"] if kind == "int4" else (nz["topk_h"] if k == H else nz["topk_f"]))
+            needed_bytes += w.packed_bytes * (nz["int4"] if kind == "int4" else (nz["topk_h"] if k == Hs else nz["topk_f"]))
 
-        def chain():
+        def chain(st=None):
             # per layer: q,k,v share the attention input and gate,up the FFN input: one call each (one launch each)
-            for li in range(LAYERS):
+            for li in range(layers):
                 (wq, *_), (wk, *_), (wv, *_), (wo, *_), (wg, *_), (wu, *_), (wd, *_) = weights[7 * li:7 * li + 7]
-                if fused:
-                    a48.linear_multi([wq, wk, wv], c4, d4, a48.ACT_INT4, Ys=yh, workspace=ws)
-                else:
-                    for w_, t in zip((wq, wk, wv), yh):
-                        a48.linear(w_, c4, d4, a48.ACT_INT4, Y=t, workspace=ws)
-                a48.linear(wo, c8h, d8h, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws)
-                if fused:
-                    a48.linear_multi([wg, wu], c4, d4, a48.ACT_INT4, Ys=[ys[0], ys[1]], workspace=ws)
-                else:
-                    a48.linear(wg, c4, d4, a48.ACT_INT4, Y=ys[0], workspace=ws)
-                    a48.linear(wu, c4, d4, a48.ACT_INT4, Y=ys[1], workspace=ws)
-                a48.linear(wd, c8f, d8f, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws)
+                a48.linear_multi([wq, wk, wv], c4, d4, a48.ACT_INT4, Ys=yh, workspace=ws, stream=st)
+                a48.linear(wo, c8h, d8h, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws, stream=st)
+                a48.linear_multi([wg, wu], c4, d4, a48.ACT_INT4, Ys=ys, workspace=ws, stream=st)
+                a48.linear(wd, c8f, d8f, a48.ACT_TOPK_INT8, Y=yh[0], workspace=ws, stream=st)
 
-        for _ in range(2):
-            chain()
-        torch.cuda.synchronize()
-        side = torch.cuda.Stream()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            chain()
-            side.synchronize()
-            with torch.cuda.graph(graph, stream=side):
-                chain()
-        torch.cuda.synchronize()
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 10
-        e0.record(stream)
-        for _ in range(reps):
-            graph.replay()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / reps
-        del graph
+        chain()
+        ms = graph_time_ms(chain, stream, reps=10)
         return {"ms_all_bitlinears": ms, "weight_stream_gbs": packed_bytes / (ms * 1e-3) / 1e9,
                 "algorithmic_gbs": needed_bytes / (ms * 1e-3) / 1e9, "tokens_per_s": M * 1e3 / ms,
                 "dense_equivalent_tops": 2.0 * M * packed_bytes * 4 / (ms * 1e-3) / 1e12, "nonzero_channel_fraction": nz}
 
     by_tokens = {str(M): time_chain(M) for M in (1, 8, 32, 64)}
     one = by_tokens["1"]
-    out = {"metric": "decode_weight_stream_gbs_7b_batch1", "value": one["weight_stream_gbs"], "unit": "GB/s",
+    out = {"metric": f"decode_weight_stream_gbs_{tag}_batch1", "value": one["weight_stream_gbs"], "unit": "GB/s",
            "ms_per_token_all_bitlinears": one["ms_all_bitlinears"], "packed_weight_bytes": packed_bytes,
            "matrices": len(weights), "hbm_peak_gbs": peaks["hbm_gbs"],
            "frac_of_hbm_peak": one["weight_stream_gbs"] / peaks["hbm_gbs"], "algorithmic_gbs": one["algorithmic_gbs"],
+           "algorithmic_frac_of_hbm_peak": one["algorithmic_gbs"] / peaks["hbm_gbs"],
            "nonzero_code_fraction": one["nonzero_channel_fraction"], "tokens_per_s": one["tokens_per_s"],
-           "launches_per_layer": 4 if fused else 7, "by_tokens": by_tokens,
-           "note": "CUDA-graph chain over 224 distinct matrices (1.6 GB >> L2), q/k/v and gate/up each as one "
-           "bitnet_a48_linear_multi call; value counts every packed byte, algorithmic_gbs only channels with a non-zero "
-           "code in some token; 1 and 8 tokens run the streaming decode kernel, 32 and 64 the tensor-core kernel "
-           "(64-token tile, cluster split-K)"}
+           "launches_per_layer": 4, "by_tokens": by_tokens,
+           "note": f"CUDA-graph chain over {len(weights)} distinct matrices ({packed_bytes / 1e9:.2f} GB >> L2), q/k/v and "
+           "gate/up each as one bitnet_a48_linear_multi call; value counts every packed byte, algorithmic_gbs only "
+           "channels with a non-zero code in some token; 1 and 8 tokens run the streaming decode kernel, 32 and 64 the "
+           "tensor-core kernel (64-token tile, cluster split-K)"}
     for w, *_ in weights:
         w.free()
     return out
 
 
+def bench_block_decode(a48, synth, dev, stream, shape, batches, ctx=2048, layer=None):
+    """One block forward per new token against a context of `ctx` cached positions, per batch size."""
+    Hs, Fs, nh = shape["H"], shape["F"], shape["NH"]
+    own = layer is None
+    if own:
+        layer = Layer(a48, dev, seed=77, layouts=a48.LAYOUT_ALL, Hs=Hs, Fs=Fs)
+    g1 = synth.norm_gains(Hs, 60, device=dev)
+    g2 = synth.norm_gains(Hs, 61, device=dev)
+    cap = ctx + 8
+    blk = a48.Block(layer.w, g1, g2, n_heads=nh, k_o=Hs // 2, k_down=Fs // 2, ctx_cap=cap)
+    out = {}
+    for Bd in batches:
+        xd = synth.gaussian_outlier_activations(Bd, Hs, seed=63, device=dev)
+        kcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=64, device=dev)
+        vcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=65, device=dev)
+        yd = torch.empty_like(xd)
+        wsd = torch.empty(blk.workspace_bytes(Bd, 1), dtype=torch.uint8, device=dev)
+
+        def call(st=None):
+            blk.forward(xd, Bd, 1, ctx, kcd, vcd, Y=yd, workspace=wsd, stream=st)
+
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record(stream)
+        for _ in range(reps):
+            call()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        ms_g = graph_time_ms(call, stream, reps=reps)  # the call is stream-ordered, so a caller can capture it
+        out[f"b{Bd}"] = {"tokens_per_s": Bd / (ms * 1e-3), "ms": ms, "context": ctx, "ms_cuda_graph": ms_g,
+                         "tokens_per_s_cuda_graph": Bd / (ms_g * 1e-3)}
+        del kcd, vcd
+    blk.free()
+    if own:
+        layer.free()
+    return out
+
+
+def bench_prefill_700m(a48, synth, dev, stream):
+    """700M shape: the seven BitLinears of a layer and the whole block on a 2048-token prefill at batch 1."""
+    Hs, Fs, nh, layers = SHAPE_700M["H"], SHAPE_700M["F"], SHAPE_700M["NH"], SHAPE_700M["LAYERS"]
+    T = 2048
+    layer = Layer(a48, dev, seed=88, layouts=a48.LAYOUT_ALL, Hs=Hs, Fs=Fs)
+    work = LayerStep(a48, synth, dev, layer, T, Hs, Fs, seed=90)
+    ms = graph_time_ms(lambda st=None: work.run(st if st is not None else stream), stream, reps=50)
+    out = {"bitlinears_ms_per_layer": ms, "bitlinears_tops": work.ops / (ms * 1e-3) / 1e12,
+           "bitlinears_tokens_per_s_model": T / (ms * 1e-3 * layers)}
+    g1 = synth.norm_gains(Hs, 60, device=dev)
+    g2 = synth.norm_gains(Hs, 61, device=dev)
+    blk = a48.Block(layer.w, g1, g2, n_heads=nh, k_o=Hs // 2, k_down=Fs // 2, ctx_cap=0)
+    x = synth.gaussian_outlier_activations(T, Hs, seed=62, device=dev)
+    y = torch.empty_like(x)
+    ws = torch.empty(blk.workspace_bytes(1, T), dtype=torch.uint8, device=dev)
+    ms_b = graph_time_ms(lambda st=None: blk.forward(x, 1, T, 0, None, None, Y=y, workspace=ws, stream=st), stream, reps=20)
+    out.update({"block_ms": ms_b, "block_tokens_per_s": T / (ms_b * 1e-3),
+                "model_tokens_per_s": T / (ms_b * 1e-3 * layers),
+                "note": "hidden 1536, GLU 4096, 16 heads of 96, 2048 tokens, batch 1; per-layer figures, the model figure "
+                        "divides by 24 layers (no embedding or head)"})
+    blk.free()
+    layer.free()
+    return out
+
+
+def bench_sweep(a48, synth, dev, stream, copies=12, reps=5):
+    """Isolated BitLinear (the library's own choice of kernel) for M = 1, 2, 4, .., 16384 on the two 7B feed-forward
+    shapes with INT4 and top-K codes: one CUDA graph per point over `copies` distinct matrices, so that neither the
+    host's launch cost nor L2 residency of the weights enters the figure."""
+    points = []
+    for N, K in ((F, H), (H, F)):
+        ws = [a48.pack_ternary(synth.ternary_latents(N, K, seed=100 + i, device=dev), EPS,
+                               a48.LAYOUT_DECODE | a48.LAYOUT_GEMM) for i in range(copies)]
+        for kind in ("int4", "topk"):
+            for e in range(15):
+                M = 1 << e
+                if kind == "int4":
+                    codes, scale = a48.quant_int4(synth.gaussian_outlier_activations(M, K, seed=11, device=dev), EPS)
+                    act = a48.ACT_INT4
+                else:
+                    codes, scale, _ = a48.topk_quant_int8(synth.student_t3(M, K, seed=12, device=dev), K // 2, EPS)
+                    act = a48.ACT_TOPK_INT8
+                y = torch.empty(M, N, dtype=torch.float32, device=dev)
+                wsp = torch.zeros(max(a48.linear_workspace_bytes(ws[0], M), 16), dtype=torch.uint8, device=dev)
+                use = ws if M <= 1024 else ws[:2]  # large M: the activations alone exceed L2
+
+                def run(st=None):
+                    for w in use:
+                        a48.linear(w, codes, scale, act, Y=y, workspace=wsp, stream=st)
+
+                ms = graph_time_ms(run, stream, reps=reps, warm=1) / len(use)
+                points.append({"N": N, "K": K, "kind": kind, "M": M, "us": ms * 1e3,
+                               "dense_tops": 2.0 * M * N * K / ms / 1e9, "weight_gbs": ws[0].packed_bytes / ms / 1e6})
+                del y, codes
+        for w in ws:
+            w.free()
+    return {"points": points,
+            "note": "bitnet_a48_linear alone (codes resident), time per call; dense_tops = 2*M*N*K / time, weight_gbs = "
+                    "packed weight bytes / time"}
+
+
 def bench_block(a48, synth, dev, stream, layer):
-    """Block forward tokens/s at the 7B shape: prefill 4096 x 4 and batch-1 decode at context 2048."""
+    """Block forward tokens/s at the 7B shape: prefill 4096 x 4 and decode at context 2048."""
     g1 = synth.norm_gains(H, 60, device=dev)
     g2 = synth.norm_gains(H, 61, device=dev)
     out = {}
     blk = a48.Block(layer.w, g1, g2, n_heads=NH, k_o=H // 2, k_down=F // 2, ctx_cap=4096)
-    # prefill
     B, T = 4, 4096
     x = synth.gaussian_outlier_activations(B * T, H, seed=62, device=dev)
     ws = torch.empty(blk.workspace_bytes(B, T), dtype=torch.uint8, device=dev)
@@ -554,44 +764,11 @@ def bench_block(a48, synth, dev, stream, layer):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / reps
     out["prefill"] = {"tokens_per_s": B * T / (ms * 1e-3), "ms": ms, "B": B, "T": T}
-    # decode: one token per sequence against a 2048-token context
-    for Bd in (1, 8):
-        xd = synth.gaussian_outlier_activations(Bd, H, seed=63, device=dev)
-        kcd = synth.kv_cache(Bd, NH, 4096, H // NH, seed=64, device=dev)
-        vcd = synth.kv_cache(Bd, NH, 4096, H // NH, seed=65, device=dev)
-        yd = torch.empty_like(xd)
-        wsd = torch.empty(blk.workspace_bytes(Bd, 1), dtype=torch.uint8, device=dev)
-        for _ in range(3):
-            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd)
-        torch.cuda.synchronize()
-        reps = 20
-        e0.record(stream)
-        for _ in range(reps):
-            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / reps
-        out[f"decode_b{Bd}"] = {"tokens_per_s": Bd / (ms * 1e-3), "ms": ms, "context": 2048}
-        # the same call captured once in a CUDA graph (the call is stream-ordered, so a caller can do this)
-        side = torch.cuda.Stream()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd, stream=side)
-            side.synchronize()
-            with torch.cuda.graph(graph, stream=side):
-                blk.forward(xd, Bd, 1, 2048, kcd, vcd, Y=yd, workspace=wsd, stream=side)
-        torch.cuda.synchronize()
-        graph.replay()
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(reps):
-            graph.replay()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms_g = e0.elapsed_time(e1) / reps
-        out[f"decode_b{Bd}"].update({"ms_cuda_graph": ms_g, "tokens_per_s_cuda_graph": Bd / (ms_g * 1e-3)})
-        del graph
     blk.free()
+    del x, y, ws, kc, vc
+    torch.cuda.empty_cache()
+    dec = bench_block_decode(a48, synth, dev, stream, SHAPE_7B, (1, 8), layer=layer)
+    out["decode_b1"], out["decode_b8"] = dec["b1"], dec["b8"]
     out["note"] = "one 7B-shape block (fp32 attention glue included); tokens/s per block, not per model"
     return out
 
@@ -599,13 +776,13 @@ def bench_block(a48, synth, dev, stream, layer):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--skip-e2e", action="store_true")
-    ap.add_argument("--skip-decode", action="store_true")
-    ap.add_argument("--skip-block", action="store_true")
-    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--legs", default="all",
+                    help="comma-separated extra legs beside the main step (" + ",".join(ALL_LEGS) + "), 'all' or ''")
+    ap.add_argument("--min-region-ms", type=float, default=1000.0,
+                    help="the timed region lasts at least this long: a counted step repeats the pass as often as needed")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

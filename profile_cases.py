@@ -1,17 +1,14 @@
 """Small single-kernel cases for profiler captures (ncu) and quick timing.
 
-    python -m paper_2411_04965_b200.profile_cases gemm   --M 8192 --N 11008 --K 4096 --kind int4 --reps 3
-    python -m paper_2411_04965_b200.profile_cases quant  --M 16384 --K 4096 --kind topk --reps 3
-    python -m paper_2411_04965_b200.profile_cases decode --M 1 --N 11008 --K 4096 --kind topk --copies 32 --reps 3
-    python -m paper_2411_04965_b200.profile_cases sweep  --copies 12 --reps 5
+    python profile_cases.py gemm   --M 8192 --N 11008 --K 4096 --kind int4 --reps 3
+    python profile_cases.py quant  --M 16384 --K 4096 --kind topk --reps 3
+    python profile_cases.py decode --M 1 --N 11008 --K 4096 --kind topk --copies 32 --reps 3
 
 Each case builds seeded synthetic inputs (the same recipes the benchmark uses),
 runs the kernel `reps` times after one warm-up call and prints the mean time
 from CUDA events on the launching stream.  `decode` cycles over `copies`
 distinct weight matrices so that the weight bytes come from HBM, not L2.
-`sweep` times `linear` (the library's own choice of kernel) for M = 1, 2, 4, ..., 16384 on the two 7B
-feed-forward shapes with INT4 and top-K codes: one CUDA graph per point over `copies` distinct matrices, so
-that neither the host's launch cost nor L2 residency of the weights enters the figure.
+(The sweep over the token count is a leg of the benchmark: `python bench.py --legs sweep`.)
 """
 from __future__ import annotations
 
@@ -20,9 +17,9 @@ import json
 
 import torch
 
-from . import binding as a48
-from . import build as a48_build
-from . import synth
+from paper_2411_04965_b200 import binding as a48
+from paper_2411_04965_b200 import build as a48_build
+from paper_2411_04965_b200 import synth
 
 EPS = 1e-5
 
@@ -49,41 +46,9 @@ def _acts(kind, M, K, dev, k_frac=0.5):
     return x, codes, scale, a48.ACT_TOPK_INT8
 
 
-def sweep(args, dev, stream):
-    for N, K in ((11008, 4096), (4096, 11008)):
-        ws = [a48.pack_ternary(synth.ternary_latents(N, K, seed=100 + i, device=dev), EPS,
-                               a48.LAYOUT_DECODE | a48.LAYOUT_GEMM) for i in range(args.copies)]
-        for kind in ("int4", "topk"):
-            for e in range(15):
-                M = 1 << e
-                _, codes, scale, act = _acts(kind, M, K, dev)
-                y = torch.empty(M, N, dtype=torch.float32, device=dev)
-                wsp = torch.zeros(max(a48.linear_workspace_bytes(ws[0], M), 16), dtype=torch.uint8, device=dev)
-                copies = ws if M <= 1024 else ws[:2]  # large M: the activations alone exceed L2
-
-                def run():
-                    for w in copies:
-                        a48.linear(w, codes, scale, act, Y=y, workspace=wsp)
-
-                run()
-                torch.cuda.synchronize()
-                graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
-                with torch.cuda.stream(side):
-                    with torch.cuda.graph(graph, stream=side):
-                        run()
-                torch.cuda.synchronize()
-                ms = _time(graph.replay, args.reps, stream) / len(copies)
-                print(json.dumps({"case": "sweep", "N": N, "K": K, "kind": kind, "M": M, "us": ms * 1e3,
-                                  "dense_tops": 2.0 * M * N * K / ms / 1e9,
-                                  "weight_gbs": ws[0].packed_bytes / ms / 1e6}), flush=True)
-                del graph
-        for w in ws:
-            w.free()
-
-
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "quant", "decode", "sweep"])
+    ap.add_argument("case", choices=["gemm", "quant", "decode"])
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=11008)
     ap.add_argument("--K", type=int, default=4096)
@@ -96,8 +61,6 @@ def main():
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     stream = torch.cuda.current_stream()
-    if args.case == "sweep":
-        return sweep(args, dev, stream)
     M, N, K = args.M, args.N, args.K
     out = {"case": args.case, "M": M, "N": N, "K": K, "kind": args.kind}
     if args.case == "quant":

@@ -65,3 +65,24 @@ def test_host_buffer_entry_points_match_the_device_path(a48, cuda_dev, M):
     a48.bitlinear_host_async(w, xp, y2, a48.ACT_TOPK_INT8, K // 2, EPS, ws, stream=side)
     side.synchronize()
     assert torch.equal(y2, expected)
+
+
+# Eq. 8-9: the FP4 quantiser's codes are integers on the doubled E2M1 grid {0, ±1, ±2, ±3, ±4, ±6, ±8, ±12}, so they
+# go through the same int8 contraction exactly.  Every kernel the dispatcher can pick is covered: decode (M <= 8),
+# the tensor-core forms (64-token tile, 192-token tile, CTA pairs from 1024 tokens on) and the simple kernel.
+@pytest.mark.parametrize("M,N,K", [(1, 512, 1024), (7, 384, 512), (40, 640, 768), (300, 384, 512), (1100, 512, 256),
+                                   (33, 130, 250)])
+def test_fp4_codes_through_the_contraction(a48, oracle, cuda_dev, M, N, K):
+    W = synth.latent_weights(N, K, seed=N + K + 1)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_ALL)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    x = synth.gaussian_outlier_activations(M, K, seed=M + 2)
+    codes, scale = a48.quant_fp4(x.to(cuda_dev))
+    g_ref, d_ref = oracle.quant_fp4(x.numpy(), nthreads=8)
+    assert np.array_equal(codes.cpu().numpy(), g_ref)
+    acc_ref, y_ref = oracle.linear(g_ref, d_ref, t_ref, alpha, nthreads=8)
+    y, acc = a48.linear(w, codes, scale, a48.ACT_FP4, a48.ALGO_AUTO, want_acc=True)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert max_rel_err(y.cpu().numpy(), y_ref) <= REL_TOL
+    y2, acc2 = a48.linear(w, codes, scale, a48.ACT_FP4, a48.ALGO_SIMPLE, want_acc=True)
+    assert torch.equal(acc, acc2)
