@@ -7,9 +7,11 @@
 //   pass 0  histogram of the 8 exponent bits (raw bits index 512 bins, the sign halves are folded in the scan);
 //           real rows hit a handful of bins, and increments of one bin from one warp are merged by the hardware;
 //   pass 1  histogram of the next 8 mantissa bits of the entries in the chosen binade;
-//   finish  the chosen sub-bin holds a few dozen entries at most on real data: they are copied to a short list
-//           and one warp ranks them against each other (exact, ties counted).  A sub-bin with more entries than
-//           the list holds (many equal values, e.g. zeros after ReLU^2) takes two more histogram passes instead.
+//   codes   every entry at or above the chosen sub-bin's lower bound gets its code; the few entries inside the
+//           sub-bin (a few dozen at most on real data) are listed on the way, one warp then ranks them against
+//           each other by (|x| descending, index ascending) and clears the codes of those that lose.  A sub-bin
+//           with more entries than the list holds (many equal values, e.g. zeros after ReLU^2) takes two more
+//           histogram passes instead, which give the exact key of the k-th entry.
 // The codes are then rounded in float32 with a proof of exactness per entry: x*s is evaluated with the float
 // neighbours s_lo < s < s_hi of the float64 scale s = 127/(gamma+eps), each as one fused multiply-add onto
 // 1.5*2^23, which rounds the exact product to the nearest integer (ties to even).  Rounding is monotone, so when
@@ -31,7 +33,6 @@ struct Select {
 
 // Warp 0 of the group scans 256 (or, FOLD, 2 x 256) bins from the top digit down and finds the bin that holds the
 // kr-th entry: sel[0] = digit, sel[1] = rank inside that bin (1-based from its top), sel[2] = its count.
-// `pad` entries are taken off bin 0 first (zero-filled register slots beyond the row).
 template <bool FOLD>
 __device__ __forceinline__ void scan_bins(const unsigned* hist, unsigned kr, unsigned* sel, int lane) {
     // lane l owns bins 255-8l-7 .. 255-8l; lanes ascend as digits descend
@@ -63,6 +64,67 @@ __device__ __forceinline__ void scan_bins(const unsigned* hist, unsigned kr, uns
     }
 }
 
+// The cold form of the last pass for one row (a bitmap is wanted, or more equal values straddle the k-th place than
+// the ranking list holds): the row is read again (it is in L2), a group-wide scan per 4*TPR entries numbers the
+// entries equal to tau so that the lowest indices win, float64 rounding throughout.  Not unrolled: it is rarely run
+// and must not crowd the instruction cache of the common path.
+template <int TPR, bool GLU>
+__device__ __noinline__ void cold_final(const float* __restrict__ xrow, const float* __restrict__ urow, int K, unsigned tau,
+                                        unsigned keep_eq, bool ordered, double mult, int8_t* __restrict__ crow,
+                                        uint32_t* __restrict__ mrow, unsigned* red, int group, int t) {
+    const int nv = K >> 2, mask_words = (K + 31) >> 5;
+    auto key = [](float f) { return __float_as_uint(f) & 0x7fffffffu; };
+    unsigned running = 0;
+#pragma unroll 1
+    for (int i0 = 0; i0 < nv; i0 += TPR) {
+        const int idx = i0 + t;
+        const bool valid = idx < nv;
+        float4 x = valid ? __ldg(reinterpret_cast<const float4*>(xrow) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (GLU && valid) {
+            const float4 u = __ldg(reinterpret_cast<const float4*>(urow) + idx);
+            auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
+            x = make_float4(f(x.x, u.x), f(x.y, u.y), f(x.z, u.z), f(x.w, u.w));
+        }
+        const unsigned u0 = key(x.x), u1 = key(x.y), u2 = key(x.z), u3 = key(x.w);
+        const bool e0 = valid && u0 == tau, e1 = valid && u1 == tau, e2 = valid && u2 == tau, e3 = valid && u3 == tau;
+        bool k0 = valid && u0 > tau, k1 = valid && u1 > tau, k2 = valid && u2 > tau, k3 = valid && u3 > tau;
+        if (!ordered) {
+            k0 |= e0; k1 |= e1; k2 |= e2; k3 |= e3;
+        } else {
+            unsigned cnt = (unsigned)e0 + e1 + e2 + e3, total;
+            unsigned base = running + group_excl_scan<TPR>(cnt, red, group, total);
+            running += total;
+            k0 |= e0 && base < keep_eq; base += e0;
+            k1 |= e1 && base < keep_eq; base += e1;
+            k2 |= e2 && base < keep_eq; base += e2;
+            k3 |= e3 && base < keep_eq;
+        }
+        if (valid) {
+            int a = k0 ? clampi(__double2int_rn(mult * (double)x.x), -128, 127) : 0;
+            int b = k1 ? clampi(__double2int_rn(mult * (double)x.y), -128, 127) : 0;
+            int c = k2 ? clampi(__double2int_rn(mult * (double)x.z), -128, 127) : 0;
+            int d = k3 ? clampi(__double2int_rn(mult * (double)x.w), -128, 127) : 0;
+            reinterpret_cast<uint32_t*>(crow)[idx] = pack4(a, b, c, d);
+        }
+        if (mrow) {  // uniform across the group
+            unsigned nib = ((unsigned)k0 | (unsigned)k1 << 1 | (unsigned)k2 << 2 | (unsigned)k3 << 3) << (4 * (t & 7));
+            nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
+            nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
+            nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
+            int word = idx >> 3;
+            if ((t & 7) == 0 && word < mask_words) mrow[word] = nib;
+        }
+    }
+}
+
+__device__ __forceinline__ void red_shared_inc(unsigned addr) {
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+// increments the word at addr when z == 0 (one predicated instruction instead of a branch around it)
+__device__ __forceinline__ void red_shared_inc_if_zero(unsigned addr, unsigned z) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %1, 0;\n\t@p red.shared.add.u32 [%0], 1;\n\t}" ::"r"(addr), "r"(z) : "memory");
+}
+
 // GLU: the row to quantise is up * ReLU(gate)^2 (Eq. 5), formed while loading: X is the gate projection and U the up
 // projection, and the product never goes to memory.
 // EXACT: V == ceil(K/4 / TPR), so only the last of a thread's V vectors can lie beyond the row.
@@ -71,9 +133,10 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     topk_quant_int8_kernel(const float* __restrict__ X, const float* __restrict__ U, int M, int K, int k, double eps,
                            int8_t* __restrict__ codes, float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
-    __shared__ unsigned hist0[G][512];
-    __shared__ unsigned hist1[G][256];
-    __shared__ unsigned cand[G][kCand];
+    __shared__ __align__(2048) unsigned hist0[G][512];  // aligned so that a bin's address is base | offset
+    __shared__ __align__(1024) unsigned hist1[G][256];
+    __shared__ unsigned cand_key[G][kCand];
+    __shared__ unsigned cand_idx[G][kCand];
     __shared__ unsigned sel[G][4];
     __shared__ unsigned red[kBlock / 32];
     const int group = threadIdx.x / TPR, t = threadIdx.x % TPR;
@@ -98,6 +161,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     unsigned* h0 = hist0[group];
     unsigned* h1 = hist1[group];
     unsigned* sl = sel[group];
+    const unsigned h0_addr = (unsigned)__cvta_generic_to_shared(h0), h1_addr = (unsigned)__cvta_generic_to_shared(h1);
     for (int b = t; b < 512; b += TPR) h0[b] = 0;
     for (int b = t; b < 256; b += TPR) h1[b] = 0;
     if (t == 0) sl[3] = 0;
@@ -123,54 +187,28 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
         }
     };
 
-    // ---- pass 0: exponent
-    for_each_raw([&](unsigned r) { atomicAdd(&h0[r >> 23], 1u); });
+    // ---- pass 0: exponent (sign and exponent index 512 bins; the scan folds the two halves)
+    for_each_raw([&](unsigned r) { red_shared_inc(h0_addr | ((r >> 21) & 0x7fcu)); });
     group_sync<TPR>(group);
     if (t < 32) scan_bins<true>(h0, (unsigned)k, sl, t);
     group_sync<TPR>(group);
     const unsigned binade = sl[0] << 23;
     // ---- pass 1: the next 8 mantissa bits of the entries in that binade
-    for_each_raw([&](unsigned r) {
-        if ((r & 0x7f800000u) == binade) atomicAdd(&h1[(r >> 15) & 255u], 1u);
-    });
+    for_each_raw([&](unsigned r) { red_shared_inc_if_zero(h1_addr | ((r >> 13) & 0x3fcu), (r ^ binade) & 0x7f800000u); });
     const unsigned kr1 = sl[1];
     group_sync<TPR>(group);
     if (t < 32) scan_bins<false>(h1, kr1, sl, t);
     group_sync<TPR>(group);
     unsigned prefix = (binade >> 15) | sl[0];  // the 16 leading bits of the key
     unsigned kr = sl[1], eq_total = sl[2];
-    Select s;
-    if (eq_total <= (unsigned)kCand) {
-        // ---- finish: the entries of the chosen sub-bin rank each other
-        for_each_raw([&](unsigned r) {
-            if (((r >> 15) & 0xffffu) == prefix) cand[group][atomicAdd(&sl[3], 1u)] = r & 0x7fffffffu;
-        });
-        group_sync<TPR>(group);
-        if (t < 32) {
-            const unsigned n = eq_total;
-#pragma unroll
-            for (int half = 0; half < kCand / 32; ++half) {
-                const int mine = t + 32 * half;
-                if (mine < (int)n) {
-                    const unsigned c = cand[group][mine];
-                    unsigned greater = 0, equal = 0;
-                    for (unsigned j = 0; j < n; ++j) {
-                        const unsigned o = cand[group][j];
-                        greater += o > c;
-                        equal += o == c;
-                    }
-                    if (greater < kr && kr <= greater + equal) {  // every lane that holds tau writes the same words
-                        sl[0] = c;
-                        sl[1] = kr - greater;
-                        sl[2] = equal;
-                    }
-                }
-            }
-        }
-        group_sync<TPR>(group);
-        s = Select{sl[0], sl[1], sl[2]};
-    } else {
-        // ---- many entries share the 16 leading bits (equal values): two more histogram passes (8 and 7 bits)
+    // Entries at or above lo are kept for now; the few below hi (the chosen sub-bin) are listed while the codes are
+    // written, ranked afterwards, and the losers' codes are cleared.
+    float lo_f = __uint_as_float(prefix << 15), hi_f = __uint_as_float((prefix << 15) + 0x8000u);
+    bool listed = true;
+    if (eq_total > (unsigned)kCand || mask_bits) {
+        // ---- many entries share the 16 leading bits (equal values, e.g. zeros): two more histogram passes (8 and 7
+        // bits) give the exact key of the k-th entry
+        listed = false;
 #pragma unroll 1
         for (int pass = 2; pass < 4; ++pass) {
             const int bits = pass == 3 ? 7 : 8, shift = pass == 2 ? 7 : 0;
@@ -178,7 +216,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
             group_sync<TPR>(group);
             for_each_raw([&](unsigned r) {
                 const unsigned u = r & 0x7fffffffu;
-                if ((u >> (shift + bits)) == prefix) atomicAdd(&h1[(u >> shift) & ((1u << bits) - 1u)], 1u);
+                red_shared_inc_if_zero(h1_addr + 4u * ((u >> shift) & ((1u << bits) - 1u)), (u >> (shift + bits)) ^ prefix);
             });
             group_sync<TPR>(group);
             if (t < 32) scan_bins<false>(h1, kr, sl, t);
@@ -188,77 +226,73 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
             eq_total = sl[2];
             group_sync<TPR>(group);  // sel is rewritten by the next scan only after every thread has read it
         }
-        s = Select{prefix, kr, eq_total};
+        // prefix is now the key tau; kr of the eq_total entries equal to it are kept.  Which ones matters only when
+        // not all are, a bitmap is wanted or tau != 0 (a kept zero and a dropped zero both have code 0).
+        const bool ordered = eq_total != kr;
+        if (mask_bits || (ordered && prefix != 0u)) {
+            if (t == 0) scale[row] = (float)(gamma / 127.0);
+            const int mask_words = (K + 31) >> 5;
+            cold_final<TPR, GLU>(X + (size_t)row * K, GLU ? U + (size_t)row * K : nullptr, K, prefix, kr, ordered, mult,
+                                 codes + (size_t)row * K, mask_bits ? mask_bits + (size_t)row * mask_words : nullptr, red,
+                                 group, t);
+            return;
+        }
+        lo_f = __uint_as_float(prefix);
+        hi_f = 0.f;  // nothing is listed
     }
 
-    const bool ordered = s.eq_total != s.keep_eq;  // a tie straddles the k-th place: lowest indices win
+    // ---- codes.  The clip of Eq. 3 is left out: |127 x / (gamma + eps)| <= 127 for every finite x of the row.
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
     if (t == 0) scale[row] = (float)(gamma / 127.0);
-    // (a tie at zero needs no order when only codes are wanted: a kept zero and a dropped zero both have code 0)
-    if ((!ordered || s.tau == 0u) && !mask_bits) {
-        // The usual case (uniform over the row's threads): every entry equal to tau is kept, so the mask is one
-        // comparison, and no bitmap is wanted.  The clip of Eq. 3 is left out here: |127 x / (gamma + eps)| <= 127
-        // for every finite x of the row, so it cannot fire.
-        const float tau_f = __uint_as_float(s.tau);
-        const float s_mid = (float)mult;
-        const float s_hi = __uint_as_float(__float_as_uint(s_mid) + 1u), s_lo = __uint_as_float(__float_as_uint(s_mid) - 1u);
-        constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: floats there are the integers, its low bits the code
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-            if (!inside(i)) continue;
-            const float x[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-            unsigned hi[4], differ = 0;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                hi[q] = __float_as_uint(__fmaf_rn(x[q], s_hi, kMagic));
-                differ |= hi[q] ^ __float_as_uint(__fmaf_rn(x[q], s_lo, kMagic));
-            }
-            if (differ) {  // some product is within ~1e-5 of a rounding tie: float64 decides, as the definition does
-#pragma unroll
-                for (int q = 0; q < 4; ++q) hi[q] = (unsigned)__double2int_rn(mult * (double)x[q]);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) hi[q] = fabsf(x[q]) >= tau_f ? hi[q] : 0u;
-            out[i * TPR + t] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
-        }
-        return;
-    }
-    auto key = [](float f) { return __float_as_uint(f) & 0x7fffffffu; };
-    const int mask_words = (K + 31) >> 5;
-    unsigned running = 0;
+    const float s_mid = (float)mult;
+    const float s_hi = __uint_as_float(__float_as_uint(s_mid) + 1u), s_lo = __uint_as_float(__float_as_uint(s_mid) - 1u);
+    constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: floats there are the integers, the low byte is the code
 #pragma unroll
     for (int i = 0; i < V; ++i) {
-        const int idx = i * TPR + t;
-        const bool valid = idx < nv;
-        const unsigned u0 = key(v[i].x), u1 = key(v[i].y), u2 = key(v[i].z), u3 = key(v[i].w);
-        const bool e0 = valid && u0 == s.tau, e1 = valid && u1 == s.tau, e2 = valid && u2 == s.tau,
-                   e3 = valid && u3 == s.tau;
-        bool k0 = valid && u0 > s.tau, k1 = valid && u1 > s.tau, k2 = valid && u2 > s.tau, k3 = valid && u3 > s.tau;
-        if (!ordered) {
-            k0 |= e0; k1 |= e1; k2 |= e2; k3 |= e3;
-        } else {
-            unsigned cnt = (unsigned)e0 + e1 + e2 + e3, total;
-            unsigned base = running + group_excl_scan<TPR>(cnt, red, group, total);
-            running += total;
-            k0 |= e0 && base < s.keep_eq; base += e0;
-            k1 |= e1 && base < s.keep_eq; base += e1;
-            k2 |= e2 && base < s.keep_eq; base += e2;
-            k3 |= e3 && base < s.keep_eq;
+        if (!inside(i)) continue;
+        const float x[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+        unsigned hi[4], differ = 0;
+        bool keep[4], any_listed = false;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            hi[q] = __float_as_uint(__fmaf_rn(x[q], s_hi, kMagic));
+            differ |= hi[q] ^ __float_as_uint(__fmaf_rn(x[q], s_lo, kMagic));
+            keep[q] = fabsf(x[q]) >= lo_f;
+            any_listed |= keep[q] && fabsf(x[q]) < hi_f;
         }
-        if (valid) {
-            int a = k0 ? clampi(__double2int_rn(mult * (double)v[i].x), -128, 127) : 0;
-            int b = k1 ? clampi(__double2int_rn(mult * (double)v[i].y), -128, 127) : 0;
-            int c = k2 ? clampi(__double2int_rn(mult * (double)v[i].z), -128, 127) : 0;
-            int d = k3 ? clampi(__double2int_rn(mult * (double)v[i].w), -128, 127) : 0;
-            out[idx] = pack4(a, b, c, d);
+        if (differ != 0u || any_listed) {  // rare
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                // a product within ~1e-5 of a rounding tie: float64 decides, as the definition does
+                if (differ) hi[q] = (unsigned)__double2int_rn(mult * (double)x[q]);
+                if (keep[q] && fabsf(x[q]) < hi_f) {
+                    const unsigned at = atomicAdd(&sl[3], 1u);
+                    cand_key[group][at] = __float_as_uint(x[q]) & 0x7fffffffu;
+                    cand_idx[group][at] = (unsigned)((i * TPR + t) * 4 + q);
+                }
+            }
         }
-        if (mask_bits) {  // uniform across the group
-            unsigned nib = ((unsigned)k0 | (unsigned)k1 << 1 | (unsigned)k2 << 2 | (unsigned)k3 << 3) << (4 * (t & 7));
-            nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
-            nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
-            nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
-            int word = idx >> 3;
-            if ((t & 7) == 0 && word < mask_words) mask_bits[(size_t)row * mask_words + word] = nib;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) hi[q] = keep[q] ? hi[q] : 0u;
+        out[i * TPR + t] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
+    }
+    if (!listed) return;  // (uniform over the group)
+    // ---- the listed entries rank each other by (|x| descending, index ascending); those ranked kr or later lose
+    group_sync<TPR>(group);
+    if (t < 32) {
+        const unsigned n = sl[3];
+#pragma unroll
+        for (int half = 0; half < kCand / 32; ++half) {
+            const unsigned mine = t + 32 * half;
+            if (mine < n) {
+                const unsigned ck = cand_key[group][mine], ci = cand_idx[group][mine];
+                unsigned ahead = 0;
+                for (unsigned j = 0; j < n; ++j) {
+                    const unsigned ok = cand_key[group][j], oi = cand_idx[group][j];
+                    ahead += (ok > ck) || (ok == ck && oi < ci);
+                }
+                if (ahead >= kr) codes[(size_t)row * K + ci] = 0;
+            }
         }
     }
 }
