@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
                            int8_t* __restrict__ codes, float* __restrict__ scale, uint32_t* __restrict__ mask_bits) {
     constexpr int G = kBlock / TPR;
     __shared__ __align__(2048) unsigned hist0[G][512];  // aligned so that a bin's address is base | offset
-    __shared__ __align__(1024) unsigned hist1[G][256];
+    __shared__ __align__(16) unsigned hist1[G][260];  // 256 bins and one (index 256) for entries outside the binade
     __shared__ unsigned cand_key[G][kCand];
     __shared__ unsigned cand_idx[G][kCand];
     __shared__ unsigned sel[G][4];
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     unsigned* sl = sel[group];
     const unsigned h0_addr = (unsigned)__cvta_generic_to_shared(h0), h1_addr = (unsigned)__cvta_generic_to_shared(h1);
     for (int b = t; b < 512; b += TPR) h0[b] = 0;
-    for (int b = t; b < 256; b += TPR) h1[b] = 0;
+    for (int b = t; b < 257; b += TPR) h1[b] = 0;
     if (t == 0) sl[3] = 0;
 
     float gm = 0.f;  // max |x| as a float maximum (one instruction per element); its bits are the largest key
@@ -194,7 +194,10 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     group_sync<TPR>(group);
     const unsigned binade = sl[0] << 23;
     // ---- pass 1: the next 8 mantissa bits of the entries in that binade
-    for_each_raw([&](unsigned r) { red_shared_inc_if_zero(h1_addr | ((r >> 13) & 0x3fcu), (r ^ binade) & 0x7f800000u); });
+    // (no test per entry: with the sign shifted out, the distance to the binade's lower end is below 2^24 inside
+    // the binade, and wraps to a large number below it; everything else lands in the spare bin)
+    const unsigned binade2 = binade << 1;
+    for_each_raw([&](unsigned r) { red_shared_inc(h1_addr + 4u * min(((r << 1) - binade2) >> 16, 256u)); });
     const unsigned kr1 = sl[1];
     group_sync<TPR>(group);
     if (t < 32) scan_bins<false>(h1, kr1, sl, t);
@@ -251,30 +254,30 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     for (int i = 0; i < V; ++i) {
         if (!inside(i)) continue;
         const float x[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-        unsigned hi[4], differ = 0;
-        bool keep[4], any_listed = false;
+        unsigned code[4], differ = 0;
+        float lowest_kept = INFINITY;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            hi[q] = __float_as_uint(__fmaf_rn(x[q], s_hi, kMagic));
-            differ |= hi[q] ^ __float_as_uint(__fmaf_rn(x[q], s_lo, kMagic));
-            keep[q] = fabsf(x[q]) >= lo_f;
-            any_listed |= keep[q] && fabsf(x[q]) < hi_f;
+            const unsigned hi = __float_as_uint(__fmaf_rn(x[q], s_hi, kMagic));
+            differ |= hi ^ __float_as_uint(__fmaf_rn(x[q], s_lo, kMagic));
+            const bool keep = fabsf(x[q]) >= lo_f;
+            code[q] = keep ? hi : 0u;
+            lowest_kept = fminf(lowest_kept, keep ? fabsf(x[q]) : INFINITY);
         }
-        if (differ != 0u || any_listed) {  // rare
+        if ((differ != 0u) | (lowest_kept < hi_f)) {  // rare
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
+                const bool keep = fabsf(x[q]) >= lo_f;
                 // a product within ~1e-5 of a rounding tie: float64 decides, as the definition does
-                if (differ) hi[q] = (unsigned)__double2int_rn(mult * (double)x[q]);
-                if (keep[q] && fabsf(x[q]) < hi_f) {
+                if (differ) code[q] = keep ? (unsigned)__double2int_rn(mult * (double)x[q]) : 0u;
+                if (keep && fabsf(x[q]) < hi_f) {
                     const unsigned at = atomicAdd(&sl[3], 1u);
                     cand_key[group][at] = __float_as_uint(x[q]) & 0x7fffffffu;
                     cand_idx[group][at] = (unsigned)((i * TPR + t) * 4 + q);
                 }
             }
         }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) hi[q] = keep[q] ? hi[q] : 0u;
-        out[i * TPR + t] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
+        out[i * TPR + t] = __byte_perm(__byte_perm(code[0], code[1], 0x0040), __byte_perm(code[2], code[3], 0x0040), 0x5410);
     }
     if (!listed) return;  // (uniform over the group)
     // ---- the listed entries rank each other by (|x| descending, index ascending); those ranked kr or later lose
