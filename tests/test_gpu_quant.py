@@ -54,6 +54,36 @@ def test_topk_quant_int8_matches_oracle(a48, oracle, cuda_dev, M, K, kfrac):
     assert_codes_match(codes.cpu().numpy(), c_ref, x.numpy(), 127.0 / (gamma + EPS), "int8")
     assert np.array_equal(scale.cpu().numpy(), d_ref.astype(np.float32))
     assert np.array_equal(codes.cpu().numpy() != 0, (c_ref != 0))
+    # the same call without the bitmap takes the kernel that keeps the row in registers: identical codes and scales
+    codes2, scale2, _ = a48.topk_quant_int8(x.to(cuda_dev), k, EPS)
+    assert torch.equal(codes2, codes) and torch.equal(scale2, scale)
+
+
+@pytest.mark.parametrize("K", [512, 1536, 3200, 4096, 8640, 11008])
+def test_topk_rows_that_leave_the_common_path(a48, oracle, cuda_dev, K):
+    # Rows built to miss the interpolated window or to overflow the ranking list of the register kernel, next to
+    # ordinary ones: two far-apart clusters (the k-th entry sits at a cluster's edge), one value repeated over most
+    # of the row (more ties than the list holds), values that differ in the last bits only, tiny magnitudes
+    # (denormals), huge ones, and mostly-zero rows whose k-th entry is zero or the smallest non-zero one.
+    g = torch.Generator().manual_seed(K)
+    rows = []
+    r = torch.randn(K, generator=g)
+    rows.append(torch.where(torch.arange(K) % 2 == 0, r * 1e-3, 1.0 + 1e-4 * r))          # two clusters, k = K/2 at the gap
+    rows.append(torch.where(torch.arange(K) % 3 == 0, r, torch.full((K,), 0.75)))           # two thirds equal 0.75
+    rows.append(1.0 + torch.randint(0, 50, (K,), generator=g).float() * 2.0 ** -23)         # last-bit differences, many ties
+    rows.append(r * 1e-41)                                                                  # denormals only
+    rows.append(r * 1e37)                                                                   # near the top of the range
+    z = torch.relu(torch.randn(K, generator=g)) ** 2
+    rows.append(z)                                                                          # about half zeros
+    rows.append(torch.where(torch.rand(K, generator=g) < 0.9, torch.zeros(K), z + 0.1))     # 90 % zeros
+    rows.append(torch.sign(r) * torch.exp(8.0 * torch.randn(K, generator=g)))               # log-normal over many binades
+    rows.append(synth.student_t3(1, K, seed=K)[0])
+    x = torch.stack(rows).float().contiguous()
+    for k in (K // 2, K // 8, K - 3, 1):
+        codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), k, EPS)
+        c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), k, EPS, nthreads=4)
+        assert np.array_equal(codes.cpu().numpy(), c_ref), f"k={k}: rows {np.unique(np.argwhere(codes.cpu().numpy() != c_ref)[:, 0])}"
+        assert np.array_equal(scale.cpu().numpy(), d_ref.astype(np.float32))
 
 
 def test_topk_without_mask_output(a48, oracle, cuda_dev):
