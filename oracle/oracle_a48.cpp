@@ -19,8 +19,15 @@
 //   * FP4 (Eq. 8-9): a single floor of log2|x| + b with real-valued b; the
 //     doubled floor printed in the paper is read as a typesetting slip.
 //     PARITY UNPINNED beyond grid membership.
+//   * Low-bit attention (Section 3): "unsigned integers using the absmax function" is read as Eq. 3 with b bits in
+//     place of 8: per head vector (one token, one head) gamma = max|x|, L = 2^(b-1) - 1,
+//     q = RoundClip(L/(gamma+eps) * x, -(L+1), L), value gamma/L * q; the unsigned integer that is stored is
+//     q + L + 1.  The paper prints no zero-point and no formula: PARITY UNPINNED beyond the code range, the error
+//     bound gamma/(2L) and the nearest-level property.  The bos token is the one at position 0 of a sequence.
+//   * FP4 variant of the block (Section 2.3): FP4 for the inputs of q/k/v, of the attention output projection
+//     (dense, no top-K) and of gate/up; the input of the down projection stays top-K + INT8.
 //
-// Build: g++ -O2 -std=c++17 -shared -fPIC -pthread oracle_a48.cpp -o liboracle_a48.so
+// Build: g++ -O2 -std=c++17 -shared -fPIC -pthread -ffp-contract=off oracle_a48.cpp -o liboracle_a48.so
 
 #include <algorithm>
 #include <cmath>
@@ -138,6 +145,17 @@ void quant_fp4_row(const float* x, int64_t K, int8_t* g, double* d) {
     *d = amax / 12.0;
 }
 
+// O7.  Low-bit attention (Section 3): absmax quantisation of one head vector to `bits` bits, Eq. 3 with
+//      L = 2^(bits-1) - 1 in place of 127.  q[i] in [-(L+1), L] (the clip at -(L+1) cannot fire); *d = gamma / L.
+void quant_head_row(const double* x, int64_t n, int bits, double eps, int8_t* q, double* d) {
+    const long L = (1L << (bits - 1)) - 1;
+    double gamma = 0.0;
+    for (int64_t i = 0; i < n; ++i) gamma = std::max(gamma, std::fabs(x[i]));
+    const double s = (double)L / (gamma + eps);
+    for (int64_t i = 0; i < n; ++i) q[i] = (int8_t)round_clip(s * x[i], -(L + 1), L);
+    *d = gamma / (double)L;
+}
+
 }  // namespace
 
 extern "C" {
@@ -148,7 +166,20 @@ struct oracle_a48_block_params {
     int64_t B, T, pos0, ctx_cap;
     int64_t k_o, k_down;  // top-k counts for the o_proj and down_proj inputs
     double norm_eps, quant_eps, rope_base;
+    int64_t act_fp4;          // Section 2.3: FP4 inputs everywhere but the down projection
+    int64_t q_bits, kv_bits;  // Section 3 low-bit attention: 0 = off; q_bits 4; kv_bits 4 or 3 (position 0 keeps 4)
 };
+
+// O7 on M head vectors of length n given as fp32 (widened exactly); codes int8, scales gamma/L as float64.
+int oracle_a48_quant_heads(const float* X, int64_t M, int64_t n, int bits, double eps, int8_t* q, double* d) {
+    if (!X || !q || !d || M <= 0 || n <= 0 || bits < 2 || bits > 8) return 1;
+    std::vector<double> row(n);
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t i = 0; i < n; ++i) row[i] = (double)X[m * n + i];
+        quant_head_row(row.data(), n, bits, eps, q + m * n, d + m);
+    }
+    return 0;
+}
 
 int oracle_a48_ternarise(const float* W, int64_t N, int64_t K, double eps, int8_t* t, double* alpha) {
     if (!W || !t || !alpha || N <= 0 || K <= 0) return 1;
@@ -234,11 +265,13 @@ int oracle_a48_block_forward(const oracle_a48_block_params* p, const float* X, c
             for (int64_t j = 0; j < H; ++j) y[m * H + j] = (float)(x[m * H + j] * r * (double)g[j]);
         }
     };
+    // dense-input BitLinear: Eq. 6-7, or Eq. 8-9 in the floating-point variant
     auto bitlinear_int4 = [&](const std::vector<float>& a, const Lin& l, int64_t N, int64_t K,
                               std::vector<double>& y) {
         std::vector<int8_t> q(M * K);
         std::vector<double> d(M);
-        oracle_a48_quant_int4(a.data(), M, K, p->quant_eps, q.data(), d.data(), nthreads);
+        if (p->act_fp4) oracle_a48_quant_fp4(a.data(), M, K, q.data(), d.data(), nthreads);
+        else oracle_a48_quant_int4(a.data(), M, K, p->quant_eps, q.data(), d.data(), nthreads);
         y.assign(M * N, 0.0);
         oracle_a48_linear(q.data(), d.data(), M, l.t.data(), l.alpha, N, K, nullptr, y.data(), nthreads);
     };
@@ -279,6 +312,25 @@ int oracle_a48_block_forward(const oracle_a48_block_params* p, const float* X, c
     };
     rope(q);
     rope(k);
+    // Section 3, low-bit attention: post-RoPE absmax quantisation of every head vector; attention then runs on the
+    // dequantised values.  With 3-bit keys/values the heads of position 0 (bos) keep 4 bits.
+    auto quant_heads = [&](std::vector<double>& z, int bits, bool bos_rule) {
+        std::vector<int8_t> codes(hd);
+        for (int64_t b = 0; b < B; ++b)
+            for (int64_t t = 0; t < T; ++t)
+                for (int64_t h = 0; h < nh; ++h) {
+                    double* r = &z[(b * T + t) * H + h * hd];
+                    const int use = (bos_rule && bits == 3 && pos0 + t == 0) ? 4 : bits;
+                    double d;
+                    quant_head_row(r, hd, use, p->quant_eps, codes.data(), &d);
+                    for (int64_t i = 0; i < hd; ++i) r[i] = d * (double)codes[i];
+                }
+    };
+    if (p->q_bits) quant_heads(q, (int)p->q_bits, false);
+    if (p->kv_bits) {
+        quant_heads(k, (int)p->kv_bits, true);
+        quant_heads(v, (int)p->kv_bits, true);
+    }
     if (k_new && v_new)
         for (int64_t b = 0; b < B; ++b)
             for (int64_t h = 0; h < nh; ++h)
@@ -328,7 +380,8 @@ int oracle_a48_block_forward(const oracle_a48_block_params* p, const float* X, c
     });
 
     std::vector<double> o;
-    bitlinear_topk(att, lo, H, H, p->k_o, o);
+    if (p->act_fp4) bitlinear_int4(att, lo, H, H, o);  // Section 2.3: FP4, dense
+    else bitlinear_topk(att, lo, H, H, p->k_o, o);
     std::vector<double> hres(M * H);
     for (int64_t i = 0; i < M * H; ++i) hres[i] = x[i] + o[i];
 
@@ -347,6 +400,40 @@ int oracle_a48_block_forward(const oracle_a48_block_params* p, const float* X, c
     std::vector<double> down;
     bitlinear_topk(inter, ld, H, F, p->k_down, down);
     for (int64_t i = 0; i < M * H; ++i) out[i] = hres[i] + down[i];
+    return 0;
+}
+
+// O8.  Gate-first evaluation of the feed-forward sub-layer (Section 2.1, paragraph after Eq. 5): the gate projection
+// first, then the up projection only for the output channels n with ReLU²(gate[n]) != 0, then Eq. 5, top-k + INT8
+// and the down projection.  X is the (already normalised) input [M, H]; weights are ternary codes with their
+// alphas.  y [M, H] float64; active [M, F] (may be NULL) receives 1 where the up projection was evaluated.
+int oracle_a48_ffn_gate_first(const float* X, int64_t M, int64_t H, int64_t F, const int8_t* tg, double ag,
+                              const int8_t* tu, double au, const int8_t* td, double ad, int64_t k_down, double eps,
+                              double* y, uint8_t* active) {
+    if (!X || !tg || !tu || !td || !y || M <= 0 || H <= 0 || F <= 0 || k_down < 1 || k_down > F) return 1;
+    std::vector<int8_t> q(H), c(F);
+    std::vector<float> inter(F);
+    for (int64_t m = 0; m < M; ++m) {
+        double d, d8;
+        quant_int4_row(X + m * H, H, eps, q.data(), &d);
+        for (int64_t n = 0; n < F; ++n) {
+            int64_t a = 0;
+            for (int64_t j = 0; j < H; ++j) a += (int64_t)q[j] * (int64_t)tg[n * H + j];
+            const double gate = ((double)a * d) * ag;
+            const double r = gate > 0.0 ? gate : 0.0;
+            const bool on = r * r != 0.0;
+            if (active) active[m * F + n] = on ? 1 : 0;
+            double up = 0.0;
+            if (on) {  // only these rows of W_up are touched
+                int64_t u = 0;
+                for (int64_t j = 0; j < H; ++j) u += (int64_t)q[j] * (int64_t)tu[n * H + j];
+                up = ((double)u * d) * au;
+            }
+            inter[n] = (float)(up * (r * r));
+        }
+        topk_quant_int8_row(inter.data(), F, k_down, eps, c.data(), &d8, nullptr);
+        linear_rows(c.data(), &d8, 0, 1, td, ad, H, F, nullptr, y + m * H);
+    }
     return 0;
 }
 

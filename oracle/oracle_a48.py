@@ -27,6 +27,7 @@ class BlockParams(ctypes.Structure):
         ("B", _i64), ("T", _i64), ("pos0", _i64), ("ctx_cap", _i64),
         ("k_o", _i64), ("k_down", _i64),
         ("norm_eps", _f64), ("quant_eps", _f64), ("rope_base", _f64),
+        ("act_fp4", _i64), ("q_bits", _i64), ("kv_bits", _i64),
     ]
 
 
@@ -144,11 +145,46 @@ def linear(codes, scale, t, alpha, nthreads=1, want_acc=True, want_y=True):
     return acc, y
 
 
+def quant_heads(X, bits, eps=1e-5):
+    """Section 3, low-bit attention: absmax quantisation of head vectors (rows of X) to `bits` bits.
+
+    Returns (codes int8 [M, n] in [-(L+1), L] with L = 2^(bits-1) - 1, scale float64 [M] = gamma / L); the stored
+    unsigned integer is code + L + 1."""
+    X = _f32(X)
+    M, n = X.shape
+    q = np.empty((M, n), np.int8)
+    d = np.empty(M, np.float64)
+    rc = _load().oracle_a48_quant_heads(_p(X, ctypes.c_float), _i64(M), _i64(n), ctypes.c_int(bits), _f64(eps),
+                                        _p(q, ctypes.c_int8), _p(d, _f64))
+    assert rc == 0, rc
+    return q, d
+
+
+def ffn_gate_first(X, tg, ag, tu, au, td, ad, k_down, eps=1e-5):
+    """Section 2.1 (after Eq. 5): gate projection first, up projection only where ReLU²(gate) != 0.
+
+    X fp32 [M, H]; tg, tu int8 [F, H]; td int8 [H, F].  Returns (y float64 [M, H], active uint8 [M, F])."""
+    X = _f32(X)
+    M, H = X.shape
+    F = tg.shape[0]
+    tg, tu, td = (np.ascontiguousarray(t, dtype=np.int8) for t in (tg, tu, td))
+    y = np.empty((M, H), np.float64)
+    active = np.empty((M, F), np.uint8)
+    rc = _load().oracle_a48_ffn_gate_first(_p(X, ctypes.c_float), _i64(M), _i64(H), _i64(F), _p(tg, ctypes.c_int8),
+                                           _f64(ag), _p(tu, ctypes.c_int8), _f64(au), _p(td, ctypes.c_int8), _f64(ad),
+                                           _i64(k_down), _f64(eps), _p(y, _f64), _p(active, ctypes.c_uint8))
+    assert rc == 0, rc
+    return y, active
+
+
 def block_forward(X, weights, g1, g2, *, n_heads, B, T, pos0=0, ctx_cap=0, kcache=None, vcache=None,
-                  k_o, k_down, norm_eps=1e-5, quant_eps=1e-5, rope_base=10000.0, nthreads=1):
+                  k_o, k_down, norm_eps=1e-5, quant_eps=1e-5, rope_base=10000.0, nthreads=1, act_fp4=False,
+                  q_bits=0, kv_bits=0):
     """One transformer block.  ``weights`` = dict with fp32 latents q,k,v,o [H,H], gate,up [F,H], down [H,F].
 
     Returns (out float64 [B*T,H], k_new, v_new float64 [B,n_heads,T,head_dim]).
+    act_fp4: the floating-point variant of Section 2.3.  q_bits / kv_bits: low-bit attention of Section 3 (k_new and
+    v_new are then the dequantised heads; kcache / vcache hold dequantised values as well).
     """
     X = _f32(X)
     M, H = X.shape
@@ -158,7 +194,8 @@ def block_forward(X, weights, g1, g2, *, n_heads, B, T, pos0=0, ctx_cap=0, kcach
     g1 = _f32(g1)
     g2 = _f32(g2)
     hd = H // n_heads
-    p = BlockParams(H, n_heads, hd, F, B, T, pos0, ctx_cap, k_o, k_down, norm_eps, quant_eps, rope_base)
+    p = BlockParams(H, n_heads, hd, F, B, T, pos0, ctx_cap, k_o, k_down, norm_eps, quant_eps, rope_base,
+                    int(act_fp4), q_bits, kv_bits)
     out = np.empty((M, H), np.float64)
     k_new = np.empty((B, n_heads, T, hd), np.float64)
     v_new = np.empty((B, n_heads, T, hd), np.float64)
