@@ -233,6 +233,14 @@ typedef struct {
     int k_o, k_down;   /* top-k counts for the o_proj and down_proj inputs */
     int ctx_cap;       /* positions each KV-cache row can hold */
     float norm_eps, quant_eps, rope_base;
+    /* Floating-point variant (Section 2.3, sentence before Eq. 8): non-zero = the inputs of q/k/v, of the attention
+     * output projection (then without top-K) and of gate/up are quantised to FP4 (Eq. 8-9); the down projection's
+     * input stays top-K + INT8.  0 = the integer model. */
+    int act_fp4;
+    /* Low-bit attention (Section 3, low-bit attention paragraph): post-RoPE absmax quantisation per head vector.
+     * q_bits: 0 (fp32 queries) or 4.  kv_bits: 0 (fp32 cache), 4 or 3; with 3 the position-0 (bos) heads keep 4 bits.
+     * With kv_bits != 0 the caches passed to bitnet_a48_block_forward are packed (bitnet_a48_kv_cache_bytes). */
+    int q_bits, kv_bits;
 } bitnet_a48_block_config;
 
 /* weights: q, k, v, o [hidden,hidden], gate, up [ffn,hidden], down [hidden,ffn] in this order.

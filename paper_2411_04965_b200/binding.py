@@ -44,7 +44,8 @@ class A48Error(RuntimeError):
 
 class BlockConfig(ctypes.Structure):
     _fields_ = [("hidden", c_int), ("n_heads", c_int), ("ffn", c_int), ("k_o", c_int), ("k_down", c_int),
-                ("ctx_cap", c_int), ("norm_eps", c_float), ("quant_eps", c_float), ("rope_base", c_float)]
+                ("ctx_cap", c_int), ("norm_eps", c_float), ("quant_eps", c_float), ("rope_base", c_float),
+                ("act_fp4", c_int), ("q_bits", c_int), ("kv_bits", c_int)]
 
 
 _lib = None
@@ -295,10 +296,11 @@ class Block:
 
     def __init__(self, weights: dict, g_attn: torch.Tensor, g_ffn: torch.Tensor, *, n_heads: int, k_o: int,
                  k_down: int, ctx_cap: int = 0, norm_eps: float = 1e-5, quant_eps: float = 1e-5,
-                 rope_base: float = 10000.0):
+                 rope_base: float = 10000.0, act_fp4: bool = False, q_bits: int = 0, kv_bits: int = 0):
         self.weights, self.g_attn, self.g_ffn = weights, g_attn, g_ffn
         H, F = weights["q"].N, weights["gate"].N
-        self.cfg = BlockConfig(H, n_heads, F, k_o, k_down, ctx_cap, norm_eps, quant_eps, rope_base)
+        self.cfg = BlockConfig(H, n_heads, F, k_o, k_down, ctx_cap, norm_eps, quant_eps, rope_base, int(act_fp4),
+                               q_bits, kv_bits)
         arr = (c_void_p * 7)(*[c_void_p(weights[n].handle) for n in self.ORDER])
         out = c_void_p(0)
         _check(lib().bitnet_a48_block_create(byref(self.cfg), arr, _ptr(g_attn), _ptr(g_ffn), byref(out)),

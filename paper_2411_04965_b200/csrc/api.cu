@@ -161,7 +161,7 @@ bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t*
                                        void* stream) {
     bitnet_a48_status s = check_act_args(X_dev, M, K, codes_dev, scale_dev);
     if (s != BITNET_A48_OK) return s;
-    return a48_launch_quant_fp4(X_dev, M, K, codes_dev, scale_dev, (cudaStream_t)stream);
+    return a48_launch_quant_fp4(X_dev, M, K, codes_dev, scale_dev, nullptr, 0.f, (cudaStream_t)stream);
 }
 
 bitnet_a48_status bitnet_a48_compact_codes(const int8_t* codes_dev, int M, int K, int cap, uint16_t* idx_dev,

@@ -462,11 +462,14 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     };
     // the decode kernel wants its scratch zero on entry and leaves it zero
     if (o.total > o.lin) A48_CUDA_TRY(cudaMemsetAsync(lin, 0, o.total - o.lin, st));
-    // attention sub-layer
-    A48_TRY(a48_launch_quant_int4(X, M, H, c.quant_eps, codes, scale, blk->g_attn, c.norm_eps, st));
+    // attention sub-layer (Eq. 6-7; FP4 variant: Eq. 8-9 in the same places)
+    const bool fp4 = c.act_fp4 != 0;
+    const bitnet_a48_act dense_kind = fp4 ? BITNET_A48_ACT_FP4 : BITNET_A48_ACT_INT4;
+    if (fp4) A48_TRY(a48_launch_quant_fp4(X, M, H, codes, scale, blk->g_attn, c.norm_eps, st));
+    else A48_TRY(a48_launch_quant_int4(X, M, H, c.quant_eps, codes, scale, blk->g_attn, c.norm_eps, st));
     {
         float* qkv[3] = {q, k, v};
-        A48_TRY(bitnet_a48_linear_multi(3, blk->w, codes, scale, M, BITNET_A48_ACT_INT4, qkv, lin, lin_bytes, st));
+        A48_TRY(bitnet_a48_linear_multi(3, blk->w, codes, scale, M, dense_kind, qkv, lin, lin_bytes, st));
     }
     {
         int n = T * (hd / 2);
@@ -488,19 +491,26 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     } else {
         A48_TRY(launch_attn_tile<256>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     }
-    A48_TRY(a48_launch_topk_quant_int8(att, M, H, c.k_o, c.quant_eps, codes, scale, nullptr, st));
-    A48_TRY(linear(3, BITNET_A48_ACT_TOPK_INT8, tmp));
+    if (fp4) {  // the floating-point variant quantises the attention output densely (no top-K)
+        A48_TRY(a48_launch_quant_fp4(att, M, H, codes, scale, nullptr, 0.f, st));
+        A48_TRY(linear(3, BITNET_A48_ACT_FP4, tmp));
+    } else {
+        A48_TRY(a48_launch_topk_quant_int8(att, M, H, c.k_o, c.quant_eps, codes, scale, nullptr, st));
+        A48_TRY(linear(3, BITNET_A48_ACT_TOPK_INT8, tmp));
+    }
     const size_t nH4 = (size_t)M * H / 4, nF4 = (size_t)M * F / 4;
     // feed-forward sub-layer: h = x + attention output, formed (and written for the last residual) in the quantiser's load
     if (a48_topk_quant_fast_shape(H)) {
-        A48_TRY(a48_launch_quant_int4_add(X, tmp, hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+        if (fp4) A48_TRY(a48_launch_quant_fp4_add(X, tmp, hres, M, H, codes, scale, blk->g_ffn, c.norm_eps, st));
+        else A48_TRY(a48_launch_quant_int4_add(X, tmp, hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
     } else {
         add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
-        A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
+        if (fp4) A48_TRY(a48_launch_quant_fp4(hres, M, H, codes, scale, blk->g_ffn, c.norm_eps, st));
+        else A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
     }
     {
         float* gu[2] = {gate, up};
-        A48_TRY(bitnet_a48_linear_multi(2, blk->w + 4, codes, scale, M, BITNET_A48_ACT_INT4, gu, lin, lin_bytes, st));
+        A48_TRY(bitnet_a48_linear_multi(2, blk->w + 4, codes, scale, M, dense_kind, gu, lin, lin_bytes, st));
     }
     if (a48_topk_quant_fast_shape(F)) {
         // Eq. 5 inside the quantiser's load: the product up * ReLU(gate)^2 is never written

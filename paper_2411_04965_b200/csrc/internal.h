@@ -65,7 +65,10 @@ bitnet_a48_status a48_launch_quant_int4_add(const float* X, const float* R, floa
                                             cudaStream_t st);
 bitnet_a48_status a48_launch_topk_quant_int8_glu(const float* gate, const float* up, int M, int K, int k, float eps,
                                                  int8_t* codes, float* scale, cudaStream_t st);
-bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st);
+bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, const float* gain,
+                                       float norm_eps, cudaStream_t st);
+bitnet_a48_status a48_launch_quant_fp4_add(const float* X, const float* R, float* SUM, int M, int K, int8_t* codes,
+                                           float* scale, const float* gain, float norm_eps, cudaStream_t st);
 bitnet_a48_status a48_launch_compact_codes(const int8_t* codes, int M, int K, int cap, uint16_t* idx, int8_t* val,
                                            int32_t* count, cudaStream_t st);
 

@@ -39,7 +39,18 @@ __device__ __forceinline__ void rmsnorm_inplace(float4 (&v)[V], int t, int nv, i
 
 // ---------------------------------------------------------------------------- Eq. 7
 // ADD: the row is X + R (a residual connection), formed while loading and written to SUM for the later residual.
-template <int TPR, int V, bool NORM, bool ADD>
+// E2M1 grid code of x*2^b (Eq. 8-9 with E = 2, M = 1): the exponent of the binade, floored at 1, sets the step
+// 2^(e-1): 1 below 4, 2 in [4, 8), 4 from 8 on; the code is step * round(x*2^b / step), an integer in
+// {0, +-1, +-2, +-3, +-4, +-6, +-8, +-12}.  Evaluated in float64 like the rest of the scale arithmetic.
+__device__ __forceinline__ int fp4_grid_code(double xp) {
+    const double ax = fabs(xp);
+    const double inv_step = ax < 4.0 ? 1.0 : (ax < 8.0 ? 0.5 : 0.25), step = ax < 4.0 ? 1.0 : (ax < 8.0 ? 2.0 : 4.0);
+    return __double2int_rn(step * rint(xp * inv_step));
+}
+
+// FP4 false: Eq. 7 (absmean, codes in [-8, 7]).  FP4 true: Eq. 8-9 (MinMax E2M1, grid codes) with the same
+// fused front ends.
+template <int TPR, int V, bool NORM, bool ADD, bool FP4 = false>
 __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restrict__ X, int M, int K, double eps,
                                                             int8_t* __restrict__ codes, float* __restrict__ scale,
                                                             const float* __restrict__ gain, double norm_eps,
@@ -63,6 +74,25 @@ __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restr
         }
     }
     if (NORM) rmsnorm_inplace<TPR, V>(v, t, nv, K, gain, norm_eps, red, group);
+    uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
+    if constexpr (FP4) {
+        float gm = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i)
+            gm = fmaxf(fmaxf(fmaxf(gm, fabsf(v[i].x)), fmaxf(fabsf(v[i].y), fabsf(v[i].z))), fabsf(v[i].w));
+        const unsigned gmax = group_max<TPR>(__float_as_uint(gm), reinterpret_cast<unsigned*>(red), group);
+        const double amax = (double)__uint_as_float(gmax);
+        const double two_b = amax > 0.0 ? 12.0 / amax : 0.0;  // 2^b of Eq. 9
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            int idx = i * TPR + t;
+            if (idx < nv)
+                out[idx] = pack4(fp4_grid_code((double)v[i].x * two_b), fp4_grid_code((double)v[i].y * two_b),
+                                 fp4_grid_code((double)v[i].z * two_b), fp4_grid_code((double)v[i].w * two_b));
+        }
+        if (t == 0) scale[row] = (float)(amax / 12.0);
+        return;
+    }
     double s = 0.0;
 #pragma unroll
     for (int i = 0; i < V; ++i)
@@ -70,7 +100,6 @@ __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restr
     s = group_sum<TPR>(s, red, group);
     const double beta = s / (double)K;
     const double mult = sqrt(7.0) / (beta + eps);
-    uint32_t* out = reinterpret_cast<uint32_t*>(codes + (size_t)row * K);
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         int idx = i * TPR + t;
@@ -113,24 +142,27 @@ __global__ void __launch_bounds__(kBlock) quant_int4_generic_kernel(const float*
 }
 
 // ---------------------------------------------------------------------------- Eq. 8-9 (E2M1)
+template <bool NORM>
 __global__ void __launch_bounds__(kBlock) quant_fp4_generic_kernel(const float* __restrict__ X, int M, int K,
-                                                                   int8_t* __restrict__ codes,
-                                                                   float* __restrict__ scale) {
-    __shared__ unsigned red[kBlock / 32];
+                                                                   int8_t* __restrict__ codes, float* __restrict__ scale,
+                                                                   const float* __restrict__ gain, double norm_eps) {
+    __shared__ double red[kBlock / 32];
     const int row = blockIdx.x, t = threadIdx.x;
     const float* xr = X + (size_t)row * K;
+    double r = 1.0;
+    if (NORM) {
+        double ss = 0.0;
+        for (int j = t; j < K; j += kBlock) ss += (double)xr[j] * xr[j];
+        ss = group_sum<kBlock>(ss, red, 0);
+        r = 1.0 / sqrt(ss / (double)K + norm_eps);
+    }
+    auto val = [&](int j) -> float { return NORM ? (float)((double)xr[j] * r * (double)gain[j]) : xr[j]; };
     unsigned gmax = 0;
-    for (int j = t; j < K; j += kBlock) gmax = max(gmax, __float_as_uint(xr[j]) & 0x7fffffffu);
-    gmax = group_max<kBlock>(gmax, red, 0);
+    for (int j = t; j < K; j += kBlock) gmax = max(gmax, __float_as_uint(val(j)) & 0x7fffffffu);
+    gmax = group_max<kBlock>(gmax, reinterpret_cast<unsigned*>(red), 0);
     const double amax = (double)__uint_as_float(gmax);
     const double two_b = amax > 0.0 ? 12.0 / amax : 0.0;  // 2^b of Eq. 9 with E=2, M=1
-    for (int j = t; j < K; j += kBlock) {
-        double xp = (double)xr[j] * two_b;
-        double ax = fabs(xp);
-        int e = ax > 0.0 ? max(ilogb(ax), 1) : 1;  // exponent of the binade, floored at 1
-        double step = ldexp(1.0, e - 1);
-        codes[(size_t)row * K + j] = (int8_t)__double2int_rn(step * rint(xp / step));
-    }
+    for (int j = t; j < K; j += kBlock) codes[(size_t)row * K + j] = (int8_t)fp4_grid_code((double)val(j) * two_b);
     if (t == 0) scale[row] = (float)(amax / 12.0);
 }
 
@@ -175,15 +207,16 @@ __global__ void __launch_bounds__(kBlock) compact_codes_kernel(const int8_t* __r
     if (t == 0) count[row] = (int32_t)running;
 }
 
-template <bool NORM, bool ADD = false>
+template <bool NORM, bool ADD = false, bool FP4 = false>
 void launch_int4(const float* X, int M, int K, double eps, int8_t* codes, float* scale, const float* gain,
                  double norm_eps, cudaStream_t st, const float* R = nullptr, float* SUM = nullptr) {
     const int nv = K / 4;
     const bool fast = (K % 4 == 0) && nv <= 256 * 12;
-#define A48_Q4(TPR, V)                                                                                           \
-    quant_int4_kernel<TPR, V, NORM, ADD><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(         \
+#define A48_Q4(TPR, V)                                                                                             \
+    quant_int4_kernel<TPR, V, NORM, ADD, FP4><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(      \
         X, M, K, eps, codes, scale, gain, norm_eps, R, SUM)
-    if (!fast) quant_int4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, eps, codes, scale, gain, norm_eps);
+    if (!fast && FP4) quant_fp4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, codes, scale, gain, norm_eps);
+    else if (!fast) quant_int4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, eps, codes, scale, gain, norm_eps);
     else if (nv <= 32 * 4) A48_Q4(32, 4);
     else if (nv <= 64 * 4) A48_Q4(64, 4);
     else if (nv <= 128 * 4) A48_Q4(128, 4);
@@ -214,8 +247,20 @@ bitnet_a48_status a48_launch_quant_int4_add(const float* X, const float* R, floa
     return BITNET_A48_OK;
 }
 
-bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, cudaStream_t st) {
-    quant_fp4_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, codes, scale);
+// gain != nullptr: RMSNorm in front, as for the INT4 quantiser.
+bitnet_a48_status a48_launch_quant_fp4(const float* X, int M, int K, int8_t* codes, float* scale, const float* gain,
+                                       float norm_eps, cudaStream_t st) {
+    if (gain) launch_int4<true, false, true>(X, M, K, 0.0, codes, scale, gain, (double)norm_eps, st);
+    else launch_int4<false, false, true>(X, M, K, 0.0, codes, scale, nullptr, 0.0, st);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+// RMSNorm + FP4 of X + R with the sum written to SUM; shapes of the register kernels only.
+bitnet_a48_status a48_launch_quant_fp4_add(const float* X, const float* R, float* SUM, int M, int K, int8_t* codes,
+                                           float* scale, const float* gain, float norm_eps, cudaStream_t st) {
+    if (!((K % 4 == 0) && K / 4 <= 256 * 12) || !gain) return BITNET_A48_ERR_UNSUPPORTED;
+    launch_int4<true, true, true>(X, M, K, 0.0, codes, scale, gain, (double)norm_eps, st, R, SUM);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }

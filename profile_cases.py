@@ -52,7 +52,7 @@ def main():
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=11008)
     ap.add_argument("--K", type=int, default=4096)
-    ap.add_argument("--kind", choices=["int4", "topk"], default="int4")
+    ap.add_argument("--kind", choices=["int4", "topk", "fp4"], default="int4")
     ap.add_argument("--algo", type=int, default=a48.ALGO_AUTO)
     ap.add_argument("--copies", type=int, default=32)
     ap.add_argument("--reps", type=int, default=3)
@@ -64,11 +64,13 @@ def main():
     M, N, K = args.M, args.N, args.K
     out = {"case": args.case, "M": M, "N": N, "K": K, "kind": args.kind}
     if args.case == "quant":
-        x = (synth.gaussian_outlier_activations if args.kind == "int4" else synth.student_t3)(M, K, 11, device=dev)
+        x = (synth.student_t3 if args.kind == "topk" else synth.gaussian_outlier_activations)(M, K, 11, device=dev)
         codes = torch.empty(M, K, dtype=torch.int8, device=dev)
         scale = torch.empty(M, dtype=torch.float32, device=dev)
         if args.kind == "int4":
             ms = _time(lambda: a48.quant_int4(x, EPS, codes, scale), args.reps, stream)
+        elif args.kind == "fp4":
+            ms = _time(lambda: a48.quant_fp4(x, codes, scale), args.reps, stream)
         else:
             ms = _time(lambda: a48.topk_quant_int8(x, K // 2, EPS, codes, scale), args.reps, stream)
         out.update(ms=ms, gbs=(5.0 * M * K + 4 * M) / ms / 1e6)

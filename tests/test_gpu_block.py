@@ -10,12 +10,12 @@ pytestmark = pytest.mark.gpu
 BLOCK_TOL = 2e-3  # max |a-b| / max |b| over the block output
 
 
-def make_block(a48, dev, H, NH, F, seed, ctx_cap=0, scale=1.0):
+def make_block(a48, dev, H, NH, F, seed, ctx_cap=0, scale=1.0, **options):
     names = (("q", H, H), ("k", H, H), ("v", H, H), ("o", H, H), ("gate", F, H), ("up", F, H), ("down", H, F))
     lat = {n: synth.latent_weights(a, b, seed=seed * 10 + i) * scale for i, (n, a, b) in enumerate(names)}
     g1, g2 = synth.norm_gains(H, seed + 100), synth.norm_gains(H, seed + 101)
     packed = {n: a48.pack_ternary(lat[n].to(dev), 1e-5, a48.LAYOUT_ALL) for n in lat}
-    blk = a48.Block(packed, g1.to(dev), g2.to(dev), n_heads=NH, k_o=H // 2, k_down=F // 2, ctx_cap=ctx_cap)
+    blk = a48.Block(packed, g1.to(dev), g2.to(dev), n_heads=NH, k_o=H // 2, k_down=F // 2, ctx_cap=ctx_cap, **options)
     return blk, lat, g1, g2
 
 
@@ -123,3 +123,23 @@ def test_block_700m_shape_prefill_without_cache(a48, oracle, cuda_dev):
     assert np.abs(ref - x.numpy()).max() > 0.05 * np.abs(ref).max()
     assert rel_to_max(y.cpu().numpy(), ref) <= BLOCK_TOL
     assert rel_above_floor(y.cpu().numpy(), ref) <= BLOCK_TOL
+
+
+# The floating-point variant (Section 2.3): FP4 (Eq. 8-9) in front of q/k/v, the attention output projection (dense)
+# and gate/up; top-K + INT8 only in front of the down projection.
+@pytest.mark.parametrize("H,NH,F,B,T,pos0", [(256, 4, 768, 1, 32, 0), (512, 4, 1024, 2, 70, 0), (400, 4, 808, 1, 3, 40),
+                                             (4096, 32, 11008, 1, 6, 20), (1536, 16, 4096, 1, 40, 0)])
+def test_block_fp4_variant(a48, oracle, cuda_dev, H, NH, F, B, T, pos0):
+    cap, hd = 128, H // NH
+    blk, lat, g1, g2 = make_block(a48, cuda_dev, H, NH, F, seed=31, ctx_cap=cap, scale=3.0 if H >= 1536 else 6.0,
+                                  act_fp4=True)
+    x = synth.gaussian_outlier_activations(B * T, H, seed=32, count=max(2, H // 100))
+    kc, vc = synth.kv_cache(B, NH, cap, hd, seed=33), synth.kv_cache(B, NH, cap, hd, seed=34)
+    kc_d, vc_d = kc.to(cuda_dev), vc.to(cuda_dev)
+    y = blk.forward(x.to(cuda_dev), B, T, pos0=pos0, kcache=kc_d, vcache=vc_d)
+    ref, k_new, v_new = oracle.block_forward(x.numpy(), {n: v.numpy() for n, v in lat.items()}, g1.numpy(), g2.numpy(),
+                                             n_heads=NH, B=B, T=T, pos0=pos0, ctx_cap=cap, kcache=kc.numpy(),
+                                             vcache=vc.numpy(), k_o=H // 2, k_down=F // 2, nthreads=8, act_fp4=True)
+    assert np.abs(ref - x.numpy()).max() > 0.05 * np.abs(ref).max()
+    assert rel_to_max(y.cpu().numpy(), ref) <= BLOCK_TOL
+    assert rel_to_max(kc_d[:, :, pos0:pos0 + T].cpu().numpy(), k_new) <= 1e-5

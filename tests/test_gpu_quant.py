@@ -94,7 +94,7 @@ def test_topk_without_mask_output(a48, oracle, cuda_dev):
     assert np.array_equal(codes.cpu().numpy(), c_ref)
 
 
-@pytest.mark.parametrize("M,K", [(16, 512), (5, 250), (3, 4096)])
+@pytest.mark.parametrize("M,K", [(16, 512), (5, 250), (3, 4096), (9, 1536), (4, 3200), (6, 8640), (5, 11008), (2, 13004)])
 def test_quant_fp4_matches_oracle(a48, oracle, cuda_dev, M, K):
     x = synth.student_t3(M, K, seed=M * K)
     x[0] = 0.0
