@@ -259,6 +259,22 @@ bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const fl
                                            float* kcache_dev, float* vcache_dev, float* Y_dev, void* workspace_dev,
                                            size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Feed-forward sub-layer for M <= 8 tokens with the gate projection first (Section 2.1, paragraph after Eq. 5;
+ * Section 3 "Sparsity"): INT4 input (Eq. 7) -> gate BitLinear (Eq. 6) -> up BitLinear only for the output channels n
+ * with ReLU²(gate[m, n]) != 0 for some token m (the other rows of W_up are not read) -> Eq. 5 -> top-k + INT8
+ * (Eq. 1, 3) -> down BitLinear.  The result equals the dense evaluation of the same sub-layer.
+ * gate, up: [ffn, hidden]; down: [hidden, ffn]; hidden a multiple of 64.  X_dev fp32 [M, hidden] is the normalised
+ * input; Y_dev fp32 [M, hidden].  inter_dev: NULL or fp32 [M, ffn], receives Eq. 5's product (0 where skipped).
+ * rows_fetched_dev: NULL or one int32 that receives the number of rows of W_up that were read.
+ * workspace_dev: bitnet_a48_ffn_gate_first_workspace_bytes bytes.  Asynchronous on `stream`; allocates nothing. */
+bitnet_a48_status bitnet_a48_ffn_gate_first(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
+                                            const bitnet_a48_weight* down, const float* X_dev, int M, int k_down, float eps,
+                                            float* Y_dev, float* inter_dev, int32_t* rows_fetched_dev, void* workspace_dev,
+                                            size_t workspace_bytes, void* stream);
+size_t bitnet_a48_ffn_gate_first_workspace_bytes(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
+                                                 const bitnet_a48_weight* down, int M);
+
 /* Reads the device-side status words that kernels with bounded waits set when
  * a wait gives up (0 = no kernel has reported anything) and clears them.
  * Synchronises the device.  words_host receives 4 values: [0] error code,

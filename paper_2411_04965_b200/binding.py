@@ -32,7 +32,7 @@ EXPORTS = [
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
-    "bitnet_a48_weight_prefetch",
+    "bitnet_a48_weight_prefetch", "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
 ]
 
 
@@ -98,6 +98,10 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_linear_multi_workspace_bytes.restype = c_size_t
         L.bitnet_a48_linear_multi_workspace_bytes.argtypes = [c_int, POINTER(c_void_p), c_int]
         L.bitnet_a48_linear_decode_static.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
+        L.bitnet_a48_ffn_gate_first.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p,
+                                                c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.bitnet_a48_ffn_gate_first_workspace_bytes.restype = c_size_t
+        L.bitnet_a48_ffn_gate_first_workspace_bytes.argtypes = [c_void_p, c_void_p, c_void_p, c_int]
         _lib = L
     return _lib
 
@@ -261,6 +265,26 @@ def linear_decode_static(w: Weight, codes: torch.Tensor, scale: torch.Tensor, Y:
     assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and tuple(Y.shape) == (codes.shape[0], w.N)
     _check(lib().bitnet_a48_linear_decode_static(c_void_p(w.handle), _ptr(codes), _ptr(scale), codes.shape[0], _ptr(Y),
                                                  _stream(stream)), "linear_decode_static")
+    return Y
+
+
+def ffn_gate_first(gate: Weight, up: Weight, down: Weight, X: torch.Tensor, k_down: int, eps: float = 1e-5, Y=None,
+                   want_inter: bool = False, want_rows: bool = False, workspace=None, stream=None):
+    """Gate-first feed-forward sub-layer for up to 8 tokens.  Returns Y, or (Y, inter, rows_fetched) parts on request."""
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous() and X.shape[1] == gate.K
+    M = X.shape[0]
+    Y = Y if Y is not None else torch.empty(M, down.N, dtype=torch.float32, device=X.device)
+    inter = torch.empty(M, gate.N, dtype=torch.float32, device=X.device) if want_inter else None
+    rows = torch.zeros(4, dtype=torch.int32, device=X.device) if want_rows else None
+    if workspace is None:
+        need = int(lib().bitnet_a48_ffn_gate_first_workspace_bytes(c_void_p(gate.handle), c_void_p(up.handle),
+                                                                   c_void_p(down.handle), M))
+        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+    _check(lib().bitnet_a48_ffn_gate_first(c_void_p(gate.handle), c_void_p(up.handle), c_void_p(down.handle), _ptr(X), M,
+                                           k_down, eps, _ptr(Y), _ptr(inter), _ptr(rows), _ptr(workspace),
+                                           workspace.numel(), _stream(stream)), "ffn_gate_first")
+    if want_inter or want_rows:
+        return Y, inter, rows
     return Y
 
 
