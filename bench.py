@@ -55,7 +55,7 @@ NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part (2 x the 2.25 P
 SHAPE_3B = dict(H=3200, F=8640, NH=32, LAYERS=26)
 SHAPE_700M = dict(H=1536, F=4096, NH=16, LAYERS=24)  # 16 heads as the benchmark configuration fixes (head dim 96)
 SHAPE_7B = dict(H=H, F=F, NH=NH, LAYERS=LAYERS)
-ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "cpu")
+ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "gatefirst", "cpu")
 
 
 def proj_list(Hs, Fs):
@@ -478,6 +478,7 @@ def run_ours(args):
         sweep = bench_sweep(a48, synth, dev, stream)
     if "block" in legs:
         block = bench_block(a48, synth, dev, stream, layer)
+    gate_first = bench_gate_first(a48, synth, dev, stream) if "gatefirst" in legs else None
 
     cpu_baseline = None
     if rank == 0 and world == 1 and "cpu" in legs:
@@ -505,7 +506,7 @@ def run_ours(args):
                             "window": f"first {n_burst} passes of the timed region"},
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "rooflines": rooflines, "e2e": e2e,
             "cpu_baseline": cpu_baseline, "decode": decode, "decode_3b": decode3b, "prefill_700m": prefill700m,
-            "sweep": sweep, "block": block,
+            "sweep": sweep, "block": block, "ffn_gate_first": gate_first,
         }
         print(json.dumps(line))
     reps.close()
@@ -739,6 +740,52 @@ def bench_sweep(a48, synth, dev, stream, copies=12, reps=5):
     return {"points": points,
             "note": "bitnet_a48_linear alone (codes resident), time per call; dense_tops = 2*M*N*K / time, weight_gbs = "
                     "packed weight bytes / time"}
+
+
+def bench_gate_first(a48, synth, dev, stream, layers=16):
+    """Feed-forward sub-layer of the 7B shape for 1 and 4 tokens, dense against gate-first, over `layers` distinct
+    layers in one CUDA graph (0.54 GB of packed weights, larger than L2)."""
+    ws_ = []
+    for li in range(layers):
+        trip = []
+        for i, (n, k) in enumerate(((F, H), (F, H), (H, F))):
+            lat = synth.latent_weights(n, k, seed=3000 + li * 4 + i, device=dev)
+            trip.append(a48.pack_ternary(lat, EPS, a48.LAYOUT_DECODE))
+            del lat
+        ws_.append(trip)
+    dense_bytes = sum(w.packed_bytes for w in ws_[0])
+    out = {"dense_weight_bytes_per_layer": dense_bytes, "layers": layers}
+    for M in (1, 4):
+        x = synth.gaussian_outlier_activations(M, H, seed=70, device=dev)
+        y = torch.empty(M, H, dtype=torch.float32, device=dev)
+        work = torch.empty(a48.ffn_workspace_bytes(*ws_[0], M), dtype=torch.uint8, device=dev)
+        _, _, rows = a48.ffn_gate_first(*ws_[0], x, F // 2, EPS, want_rows=True)
+        torch.cuda.synchronize()
+        rows_fetched = int(rows[0])
+
+        def dense(st=None):
+            for g, u, d in ws_:
+                a48.ffn_dense(g, u, d, x, F // 2, EPS, Y=y, workspace=work, stream=st)
+
+        def gate_first(st=None):
+            for g, u, d in ws_:
+                a48.ffn_gate_first(g, u, d, x, F // 2, EPS, Y=y, workspace=work, stream=st)
+
+        ms_d = graph_time_ms(dense, stream, reps=10) / layers
+        ms_g = graph_time_ms(gate_first, stream, reps=10) / layers
+        up_bytes = ws_[0][1].packed_bytes
+        fetched = dense_bytes - up_bytes + up_bytes * rows_fetched / F
+        out[f"tokens_{M}"] = {"dense_us": ms_d * 1e3, "gate_first_us": ms_g * 1e3, "up_rows_fetched": rows_fetched,
+                              "up_rows_fetched_fraction": rows_fetched / F, "weight_bytes_fetched": fetched,
+                              "weight_bytes_fetched_fraction": fetched / dense_bytes,
+                              "dense_gbs": dense_bytes / ms_d / 1e6, "gate_first_algorithmic_gbs": fetched / ms_g / 1e6}
+    for trip in ws_:
+        for w in trip:
+            w.free()
+    out["note"] = ("bitnet_a48_ffn_dense against bitnet_a48_ffn_gate_first: INT4 quantiser, gate/up, Eq. 5, top-K + INT8, "
+                   "down; synthetic Gaussian latents give about half positive gates (the paper reports 67.5 % zero gates "
+                   "on trained 7B weights)")
+    return out
 
 
 def bench_block(a48, synth, dev, stream, layer):

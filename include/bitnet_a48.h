@@ -272,6 +272,12 @@ bitnet_a48_status bitnet_a48_ffn_gate_first(const bitnet_a48_weight* gate, const
                                             const bitnet_a48_weight* down, const float* X_dev, int M, int k_down, float eps,
                                             float* Y_dev, float* inter_dev, int32_t* rows_fetched_dev, void* workspace_dev,
                                             size_t workspace_bytes, void* stream);
+/* The same sub-layer evaluated densely (Eq. 5-7, Eq. 1, 3): gate and up as one fused launch over every row.  Same
+ * shapes, limits and workspace as bitnet_a48_ffn_gate_first (ffn a multiple of 4 and at most 12288); it is the
+ * reference point for what gate-first evaluation saves. */
+bitnet_a48_status bitnet_a48_ffn_dense(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
+                                       const bitnet_a48_weight* down, const float* X_dev, int M, int k_down, float eps,
+                                       float* Y_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 size_t bitnet_a48_ffn_gate_first_workspace_bytes(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
                                                  const bitnet_a48_weight* down, int M);
 

@@ -33,6 +33,7 @@ EXPORTS = [
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
     "bitnet_a48_weight_prefetch", "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
+    "bitnet_a48_ffn_dense",
 ]
 
 
@@ -100,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_linear_decode_static.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
         L.bitnet_a48_ffn_gate_first.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p,
                                                 c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.bitnet_a48_ffn_dense.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p, c_void_p,
+                                           c_size_t, c_void_p]
         L.bitnet_a48_ffn_gate_first_workspace_bytes.restype = c_size_t
         L.bitnet_a48_ffn_gate_first_workspace_bytes.argtypes = [c_void_p, c_void_p, c_void_p, c_int]
         _lib = L
@@ -285,6 +288,25 @@ def ffn_gate_first(gate: Weight, up: Weight, down: Weight, X: torch.Tensor, k_do
                                            workspace.numel(), _stream(stream)), "ffn_gate_first")
     if want_inter or want_rows:
         return Y, inter, rows
+    return Y
+
+
+def ffn_workspace_bytes(gate: Weight, up: Weight, down: Weight, M: int) -> int:
+    return int(lib().bitnet_a48_ffn_gate_first_workspace_bytes(c_void_p(gate.handle), c_void_p(up.handle),
+                                                               c_void_p(down.handle), M))
+
+
+def ffn_dense(gate: Weight, up: Weight, down: Weight, X: torch.Tensor, k_down: int, eps: float = 1e-5, Y=None,
+              workspace=None, stream=None):
+    """The feed-forward sub-layer for up to 8 tokens evaluated densely (the comparison point of ffn_gate_first)."""
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous() and X.shape[1] == gate.K
+    M = X.shape[0]
+    Y = Y if Y is not None else torch.empty(M, down.N, dtype=torch.float32, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(ffn_workspace_bytes(gate, up, down, M), dtype=torch.uint8, device=X.device)
+    _check(lib().bitnet_a48_ffn_dense(c_void_p(gate.handle), c_void_p(up.handle), c_void_p(down.handle), _ptr(X), M,
+                                      k_down, eps, _ptr(Y), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "ffn_dense")
     return Y
 
 

@@ -129,7 +129,48 @@ FfnWs ffn_ws(const bitnet_a48_weight* gate, const bitnet_a48_weight* down, int M
 extern "C" size_t bitnet_a48_ffn_gate_first_workspace_bytes(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
                                                             const bitnet_a48_weight* down, int M) {
     if (!gate || !up || !down || M <= 0) return 0;
-    return ffn_ws(gate, down, M).total;
+    const FfnWs o = ffn_ws(gate, down, M);
+    const bitnet_a48_weight* gu[2] = {gate, up};
+    const size_t multi = bitnet_a48_linear_multi_workspace_bytes(2, gu, M);  // the dense form's fused gate+up launch
+    return o.lin + (multi > o.total - o.lin ? multi : o.total - o.lin);
+}
+
+// The same sub-layer evaluated densely (gate and up as one fused launch over every row, Eq. 5 inside the top-K
+// quantiser's load): the reference point for what gate-first saves.
+extern "C" bitnet_a48_status bitnet_a48_ffn_dense(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,
+                                                  const bitnet_a48_weight* down, const float* X_dev, int M, int k_down,
+                                                  float eps, float* Y_dev, void* workspace_dev, size_t workspace_bytes,
+                                                  void* stream) {
+    if (!gate || !up || !down || !X_dev || !Y_dev || !workspace_dev) return BITNET_A48_ERR_INVALID_ARG;
+    const int H = gate->K, F = gate->N;
+    if (up->N != F || up->K != H || down->N != H || down->K != F) return BITNET_A48_ERR_SHAPE;
+    if (M <= 0 || M > 8 || !a48_topk_quant_fast_shape(F)) return BITNET_A48_ERR_UNSUPPORTED;
+    if (k_down < 1 || k_down > F || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
+    if (!a48_aligned16(X_dev) || !a48_aligned16(Y_dev) || !a48_aligned16(workspace_dev)) return BITNET_A48_ERR_ALIGNMENT;
+    const FfnWs o = ffn_ws(gate, down, M);
+    // the fused gate+up launch may want more scratch than either matrix alone
+    const bitnet_a48_weight* gu[2] = {gate, up};
+    const size_t multi = bitnet_a48_linear_multi_workspace_bytes(2, gu, M);
+    if (workspace_bytes < o.lin + (multi > o.total - o.lin ? multi : o.total - o.lin)) return BITNET_A48_ERR_NOMEM;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = static_cast<char*>(workspace_dev);
+    int8_t* codes4 = reinterpret_cast<int8_t*>(base + o.codes4);
+    float* scale4 = reinterpret_cast<float*>(base + o.scale4);
+    float* gate_y = reinterpret_cast<float*>(base + o.gate);
+    float* up_y = reinterpret_cast<float*>(base + o.inter);
+    int8_t* codes8 = reinterpret_cast<int8_t*>(base + o.codes8);
+    float* scale8 = reinterpret_cast<float*>(base + o.scale8);
+    void* lin = base + o.lin;
+    const size_t lin_bytes = workspace_bytes - o.lin;
+    A48_CUDA_TRY(cudaMemsetAsync(lin, 0, lin_bytes, st));
+    bitnet_a48_status s = bitnet_a48_quant_int4(X_dev, M, H, eps, codes4, scale4, stream);
+    if (s != BITNET_A48_OK) return s;
+    float* ys[2] = {gate_y, up_y};
+    s = bitnet_a48_linear_multi(2, gu, codes4, scale4, M, BITNET_A48_ACT_INT4, ys, lin, lin_bytes, stream);
+    if (s != BITNET_A48_OK) return s;
+    s = a48_launch_topk_quant_int8_glu(gate_y, up_y, M, F, k_down, eps, codes8, scale8, st);
+    if (s != BITNET_A48_OK) return s;
+    return bitnet_a48_linear(down, codes8, scale8, M, BITNET_A48_ACT_TOPK_INT8, Y_dev, nullptr, lin, lin_bytes, stream);
 }
 
 extern "C" bitnet_a48_status bitnet_a48_ffn_gate_first(const bitnet_a48_weight* gate, const bitnet_a48_weight* up,

@@ -42,6 +42,8 @@ def test_ffn_gate_first_matches_oracle(a48, oracle, cuda_dev, H, F, M):
     c8, s8, _ = a48.topk_quant_int8(prod, F // 2, EPS)
     y_dense = a48.linear(w["down"], c8, s8, a48.ACT_TOPK_INT8)
     assert torch.equal(inter, prod) and torch.equal(y, y_dense)
+    if F % 4 == 0:
+        assert torch.equal(a48.ffn_dense(w["gate"], w["up"], w["down"], x.to(cuda_dev), F // 2, EPS), y)
 
 
 def test_ffn_gate_first_argument_checks(a48, cuda_dev):
