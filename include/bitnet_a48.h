@@ -249,12 +249,21 @@ typedef struct {
 bitnet_a48_status bitnet_a48_block_create(const bitnet_a48_block_config* cfg, const bitnet_a48_weight* const weights[7],
                                           const float* gain_attn_dev, const float* gain_ffn_dev, bitnet_a48_block** out);
 void bitnet_a48_block_free(bitnet_a48_block* blk);
+/* Bytes of ONE cache buffer (keys or values) for B sequences of ctx_cap positions: B*n_heads*ctx_cap*head_dim*4 with
+ * kv_bits == 0; with kv_bits 4 or 3 the packed layout of Section 3's low-bit attention - per head vector a
+ * little-endian bit stream of kv_bits-bit unsigned codes (head_dim padded to a multiple of 32 entries), then one
+ * fp32 scale per head vector, then (3-bit only) the 4-bit codes of position 0.  The caller allocates it (16-byte
+ * aligned); its contents are written by bitnet_a48_block_forward only. */
+size_t bitnet_a48_kv_cache_bytes(const bitnet_a48_block* blk, int B);
 size_t bitnet_a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
 /* X_dev fp32 [B*T, hidden] -> Y_dev fp32 [B*T, hidden].  Tokens of batch b sit at
  * positions pos0..pos0+T-1; their keys/values are written into the caches at
  * those positions and attention reads positions 0..own position.  The caches
  * may be NULL only when pos0 == 0 and T is the whole sequence (keys/values then
- * live in the workspace).  All kernels run on `stream`; nothing synchronises. */
+ * live in the workspace).  With kv_bits != 0 the caches are packed buffers of bitnet_a48_kv_cache_bytes bytes
+ * (passed through the same pointers), head_dim <= 128, and a call is either a prefill from position 0 or a decode
+ * step of T <= 8 tokens (BITNET_A48_ERR_UNSUPPORTED otherwise); q_bits != 0 needs kv_bits != 0.
+ * All kernels run on `stream`; nothing synchronises. */
 bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const float* X_dev, int B, int T, int pos0,
                                            float* kcache_dev, float* vcache_dev, float* Y_dev, void* workspace_dev,
                                            size_t workspace_bytes, void* stream);

@@ -33,7 +33,7 @@ EXPORTS = [
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
     "bitnet_a48_weight_prefetch", "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
-    "bitnet_a48_ffn_dense",
+    "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes",
 ]
 
 
@@ -94,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_block_forward.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                                c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_kernel_status.argtypes = [POINTER(c_uint)]
+        L.bitnet_a48_kv_cache_bytes.restype = c_size_t
+        L.bitnet_a48_kv_cache_bytes.argtypes = [c_void_p, c_int]
         L.bitnet_a48_linear_multi.argtypes = [c_int, POINTER(c_void_p), c_void_p, c_void_p, c_int, c_int, POINTER(c_void_p),
                                               c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_linear_multi_workspace_bytes.restype = c_size_t
@@ -363,6 +365,10 @@ class Block:
             self.free()
         except Exception:
             pass
+
+    def kv_cache_bytes(self, B: int) -> int:
+        """Bytes of one cache buffer (keys or values) for B sequences; packed when kv_bits != 0."""
+        return int(lib().bitnet_a48_kv_cache_bytes(c_void_p(self.handle), B))
 
     def workspace_bytes(self, B: int, T: int) -> int:
         return int(lib().bitnet_a48_block_workspace_bytes(c_void_p(self.handle), B, T))

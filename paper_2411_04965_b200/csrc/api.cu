@@ -365,6 +365,12 @@ bitnet_a48_status bitnet_a48_block_create(const bitnet_a48_block_config* cfg, co
 
 void bitnet_a48_block_free(bitnet_a48_block* blk) { delete blk; }
 
+size_t bitnet_a48_kv_cache_bytes(const bitnet_a48_block* blk, int B) {
+    if (!blk || B <= 0 || blk->cfg.ctx_cap <= 0) return 0;
+    const bitnet_a48_block_config& c = blk->cfg;
+    return a48_kv_cache_bytes(B, c.n_heads, c.ctx_cap, c.hidden / c.n_heads, c.kv_bits);
+}
+
 size_t bitnet_a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T) {
     if (!blk || B <= 0 || T <= 0) return 0;
     return a48_block_workspace_bytes(blk, B, T);

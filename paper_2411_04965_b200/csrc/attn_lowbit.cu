@@ -1,0 +1,352 @@
+// Low-bit attention (Section 3, low-bit attention paragraph): post-RoPE absmax quantisation of the query, key and
+// value heads, a packed key/value cache of 4 or 3 bits per entry (the heads of position 0, the bos token, keep
+// 4 bits in a 3-bit cache), and the decode attention that reads it.
+//
+// Quantiser of one head vector x (one token, one head), Eq. 3 with b bits in place of 8: gamma = max|x|,
+// L = 2^(b-1) - 1, q = RoundClip(L/(gamma+eps) * x, -(L+1), L), value gamma/L * q; the unsigned integer
+// u = q + L + 1 is what the cache stores.  The scale arithmetic is float64 as in the other quantisers.
+//
+// Cache layout (one buffer for keys, one for values; bitnet_a48_kv_cache_bytes gives its size):
+//   codes  [B][n_heads][ctx_cap][row_bytes]   row = the head's entries as a little-endian bit stream, entry i at
+//                                             bits [i*b, (i+1)*b); row_bytes = b * head_dim_padded / 8 with the
+//                                             head dimension padded to a multiple of 32 entries (12- or 16-byte
+//                                             granules of 32 entries)
+//   scales [B][n_heads][ctx_cap] fp32         gamma / L
+//   bos    [B][n_heads][row_bytes at 4 bits]  only in a 3-bit cache: the 4-bit codes of position 0
+// A 3-bit cache holds 52 bytes per head vector of 128 entries where fp32 holds 512.
+#include "internal.h"
+
+namespace {
+
+__host__ __device__ inline int padded_dim(int hd) { return (hd + 31) / 32 * 32; }
+__host__ __device__ inline int row_bytes(int hd, int bits) { return padded_dim(hd) * bits / 8; }
+
+struct KvView {
+    uint8_t* codes;
+    float* scales;
+    uint8_t* bos;  // nullptr unless bits == 3
+    int bits, row, row4;
+};
+
+__host__ __device__ inline KvView kv_view(void* base, int B, int nh, int cap, int hd, int bits) {
+    KvView v;
+    v.bits = bits;
+    v.row = row_bytes(hd, bits);
+    v.row4 = row_bytes(hd, 4);
+    v.codes = static_cast<uint8_t*>(base);
+    const size_t codes_bytes = ((size_t)B * nh * cap * v.row + 15) / 16 * 16;
+    v.scales = reinterpret_cast<float*>(v.codes + codes_bytes);
+    const size_t scale_bytes = ((size_t)B * nh * cap * 4 + 15) / 16 * 16;
+    v.bos = bits == 3 ? v.codes + codes_bytes + scale_bytes : nullptr;
+    return v;
+}
+
+// One warp quantises one head vector held as hd <= 128 floats, lane l owning entries 4l..4l+3 (zero past hd).
+// Returns the codes of the lane (as unsigned u = q + L + 1, 0 for padding... padding stores u of q = 0) and the scale.
+__device__ __forceinline__ void quant_head_warp(const float (&x)[4], int bits, double eps, unsigned (&u)[4], float& scale_out) {
+    float gm = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+    const int L = (1 << (bits - 1)) - 1;
+    const double gamma = (double)gm;
+    const double s = (double)L / (gamma + eps);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int q = __double2int_rn(s * (double)x[i]);
+        q = q < -(L + 1) ? -(L + 1) : (q > L ? L : q);
+        u[i] = (unsigned)(q + L + 1);
+    }
+    scale_out = (float)(gamma / (double)L);
+}
+
+// Writes the warp's 128 (padded) entries of `bits` bits each as a bit stream: lane l's four entries are bits
+// [4l*bits, (4l+4)*bits).  With 4 bits that is two bytes per lane; with 3 bits twelve bits per lane, so lanes pair
+// up to three bytes.  Only the first row_bytes(hd) bytes exist.
+__device__ __forceinline__ void store_codes_warp(uint8_t* row, int nbytes, const unsigned (&u)[4], int bits, int lane) {
+    if (bits == 4) {
+        const unsigned v = u[0] | (u[1] << 4) | (u[2] << 8) | (u[3] << 12);
+        if (2 * lane + 1 < nbytes) *reinterpret_cast<uint16_t*>(row + 2 * lane) = (uint16_t)v;
+    } else {
+        const unsigned v = u[0] | (u[1] << 3) | (u[2] << 6) | (u[3] << 9);  // 12 bits
+        const unsigned other = __shfl_xor_sync(0xffffffffu, v, 1);
+        if ((lane & 1) == 0) {
+            const unsigned w = v | (other << 12);  // 24 bits of lanes l, l+1
+            const int at = 3 * (lane >> 1);
+            if (at + 2 < nbytes) {
+                row[at] = (uint8_t)w;
+                row[at + 1] = (uint8_t)(w >> 8);
+                row[at + 2] = (uint8_t)(w >> 16);
+            }
+        }
+    }
+}
+
+// RoPE on (i, i + hd/2) pairs for q and k, then the head quantisers.  One warp per (token, head); hd <= 128,
+// lane l owns entries 4l..4l+3 (the rotation partner of entry i sits in lane (l + hd/8) mod (hd/4)... fetched from
+// memory instead: every lane reads its four entries and their four partners).
+// table: nullptr (a few tokens: the angles are evaluated here) or cos/sin pairs [T][hd/2].
+// q is overwritten with the rotated (and, q_bits != 0, quantise-dequantised) query.  The rotated key and the value
+// go to the packed caches at position pos0 + t; dq_k / dq_v (may be nullptr) receive their dequantised fp32 values
+// laid out [B][nh][T][hd] for the prefill attention kernel.
+__global__ void __launch_bounds__(256) rope_quant_cache_kernel(float* __restrict__ q, const float* __restrict__ k,
+                                                               const float* __restrict__ v, const float2* __restrict__ table,
+                                                               double base, int B, int T, int nh,
+                                                               int hd, int pos0, int cap, int q_bits, int kv_bits, double eps,
+                                                               void* kcache, void* vcache, float* __restrict__ dq_k,
+                                                               float* __restrict__ dq_v) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= B * T * nh) return;
+    const int h = warp % nh, m = warp / nh, t = m % T, b = m / T;
+    const int half = hd / 2, pos = pos0 + t;
+    const size_t src = (size_t)m * nh * hd + (size_t)h * hd;
+    float qr[4], kr[4], vr[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int e = 4 * lane + i;
+        qr[i] = kr[i] = vr[i] = 0.f;
+        if (e < hd) {
+            const int j = e < half ? e : e - half;  // index of the rotation pair
+            float c, s;
+            if (table) {  // cos/sin of (pos0 + t) * base^(-j/half), evaluated in float64 by the caller's table kernel
+                const float2 cs = table[t * half + j];
+                c = cs.x;
+                s = cs.y;
+            } else {
+                const double ang = (double)pos * pow(base, -(double)j / (double)half);
+                double sn, cn;
+                sincos(ang, &sn, &cn);
+                c = (float)cn;
+                s = (float)sn;
+            }
+            const float ql = q[src + j], qh = q[src + j + half], kl = k[src + j], kh = k[src + j + half];
+            qr[i] = e < half ? ql * c - qh * s : qh * c + ql * s;
+            kr[i] = e < half ? kl * c - kh * s : kh * c + kl * s;
+            vr[i] = v[src + e];
+        }
+    }
+    __syncwarp();  // every lane has read the q entries it needs before any lane overwrites them
+    unsigned u[4];
+    float sc;
+    if (q_bits) {
+        quant_head_warp(qr, q_bits, eps, u, sc);
+        const int L = (1 << (q_bits - 1)) - 1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) qr[i] = sc * (float)((int)u[i] - (L + 1));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (4 * lane + i < hd) q[src + 4 * lane + i] = qr[i];
+    const int use_bits = (kv_bits == 3 && pos == 0) ? 4 : kv_bits;  // the bos heads keep 4 bits
+    const int L = (1 << (use_bits - 1)) - 1;
+    const size_t slot = ((size_t)b * nh + h) * cap + pos;
+    const size_t dq = (((size_t)b * nh + h) * T + t) * hd;
+    for (int which = 0; which < 2; ++which) {
+        const float(&x)[4] = which == 0 ? kr : vr;
+        KvView view = kv_view(which == 0 ? kcache : vcache, B, nh, cap, hd, kv_bits);
+        quant_head_warp(x, use_bits, eps, u, sc);
+        uint8_t* row = (kv_bits == 3 && pos == 0) ? view.bos + ((size_t)b * nh + h) * view.row4 : view.codes + slot * view.row;
+        store_codes_warp(row, use_bits == 4 ? view.row4 : view.row, u, use_bits, lane);
+        if (lane == 0) view.scales[slot] = sc;
+        float* out = which == 0 ? dq_k : dq_v;
+        if (out) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (4 * lane + i < hd) out[dq + 4 * lane + i] = sc * (float)((int)u[i] - (L + 1));
+        }
+    }
+}
+
+// Eight entries of a row as floats (u - offset, not yet scaled).  Lane `sub` of the 16 lanes that share a row owns
+// entries 8*sub..8*sub+7: one 32-bit word at 4 bits, 24 bits out of a 12-byte granule at 3 bits (the granule's three
+// words are loaded by all four lanes that share it).
+__device__ __forceinline__ void load8(const uint8_t* row, int bits, int sub, bool inside, float (&f)[8]) {
+    unsigned w;
+    if (!inside) {  // this lane's entries lie beyond the (padded) head: nothing is read
+        w = 0;
+    } else if (bits == 4) {
+        w = __ldg(reinterpret_cast<const unsigned*>(row) + sub);
+    } else {
+        const unsigned* g = reinterpret_cast<const unsigned*>(row) + 3 * (sub >> 2);
+        const unsigned w0 = __ldg(g), w1 = __ldg(g + 1), w2 = __ldg(g + 2);
+        const int i = sub & 3;  // bits [24 i, 24 i + 24) of the 96-bit granule
+        w = i == 0 ? w0 : (i == 1 ? __funnelshift_r(w0, w1, 24) : (i == 2 ? __funnelshift_r(w1, w2, 16) : (w2 >> 8)));
+    }
+    const unsigned mask = (1u << bits) - 1u;
+    const float offset = 8388608.f + (float)(1 << (bits - 1));  // 2^23 + L + 1
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        f[i] = __uint_as_float(0x4B000000u | ((w >> (bits * i)) & mask)) - offset;  // exact: u - (L + 1)
+}
+
+constexpr int ATTN_SPLITS = 8;
+
+__device__ __forceinline__ float ld_cluster_f32(const float* p, unsigned rank) {
+    float v;
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %1, %2;\n\tld.shared::cluster.f32 %0, [ra];\n\t}"
+        : "=f"(v)
+        : "r"((unsigned)__cvta_generic_to_shared(p)), "r"(rank));
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Decode attention over the packed cache for a few queries per sequence: the keys of one (query, head, batch) are
+// split over the ATTN_SPLITS CTAs of a cluster; inside a CTA every half-warp takes one key at a time (lane `sub`
+// of the half-warp owns entries 8 sub .. 8 sub + 7 of the head, head_dim <= 128), two keys in flight per half-warp;
+// online softmax per half-warp, then the same combination through shared memory and distributed shared memory as
+// the fp32 kernel.
+__global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __restrict__ q, const void* kcache, const void* vcache,
+                                                              int B, int T, int nh, int hd, int pos0, int cap, int kv_bits,
+                                                              float scale, float* __restrict__ out) {
+    constexpr int HALVES = 16;  // half-warps per CTA
+    __shared__ float sm_m[HALVES], sm_l[HALVES];
+    __shared__ float sm_o[HALVES][128];
+    __shared__ float cta_ml[2];
+    __shared__ float cta_o[128];
+    const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z / T, t = blockIdx.z % T;
+    const int lane = threadIdx.x & 31, sub = lane & 15, halfw = threadIdx.x >> 4;
+    const size_t H = (size_t)nh * hd;
+    const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
+    const KvView kview = kv_view(const_cast<void*>(kcache), B, nh, cap, hd, kv_bits);
+    const KvView vview = kv_view(const_cast<void*>(vcache), B, nh, cap, hd, kv_bits);
+    float qreg[8], o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int col = 8 * sub + i;
+        qreg[i] = col < hd ? qr[col] * scale : 0.f;
+        o[i] = 0.f;
+    }
+    float m = -INFINITY, l = 0.f;
+    const int n_keys = pos0 + t + 1;
+    const int per = (n_keys + ATTN_SPLITS - 1) / ATTN_SPLITS;
+    const int j_end = min(n_keys, (split + 1) * per);
+    const size_t head = (size_t)b * nh + h;
+    const unsigned half_mask = 0xffffu << (lane & 16);
+    const bool mine = 8 * sub < padded_dim(hd);
+    for (int j0 = split * per + halfw; j0 < j_end; j0 += 2 * HALVES) {
+        float kf[2][8], vf[2][8], ks[2], vs[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int j = j0 + HALVES * u;
+            const bool ok = j < j_end;
+            const int jj = ok ? j : j0;
+            const bool bos = kv_bits == 3 && jj == 0;
+            const size_t slot = head * cap + jj;
+            load8(bos ? kview.bos + head * kview.row4 : kview.codes + slot * kview.row, bos ? 4 : kv_bits, sub, mine, kf[u]);
+            load8(bos ? vview.bos + head * vview.row4 : vview.codes + slot * vview.row, bos ? 4 : kv_bits, sub, mine, vf[u]);
+            ks[u] = __ldg(kview.scales + slot);
+            vs[u] = __ldg(vview.scales + slot);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float dot = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dot += qreg[i] * kf[u][i];
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(half_mask, dot, off);
+            dot *= ks[u];
+            if (j0 + HALVES * u < j_end) {
+                const float m_new = fmaxf(m, dot);
+                const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+                const float pr = expf(dot - m_new);
+                l = l * corr + pr;
+                const float pv = pr * vs[u];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] = o[i] * corr + pv * vf[u][i];
+                m = m_new;
+            }
+        }
+    }
+    if (sub == 0) {
+        sm_m[halfw] = m;
+        sm_l[halfw] = l;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sm_o[halfw][8 * sub + i] = o[i];
+    __syncthreads();
+    if (threadIdx.x < 128) {
+        const int col = threadIdx.x;
+        float mm = -INFINITY;
+        for (int w = 0; w < HALVES; ++w) mm = fmaxf(mm, sm_m[w]);
+        float ll = 0.f, acc = 0.f;
+        for (int w = 0; w < HALVES; ++w) {
+            if (sm_m[w] == -INFINITY) continue;
+            const float f = expf(sm_m[w] - mm);
+            ll += sm_l[w] * f;
+            acc += sm_o[w][col] * f;
+        }
+        if (col == 0) {
+            cta_ml[0] = mm;
+            cta_ml[1] = ll;
+        }
+        cta_o[col] = acc;
+    }
+    cluster_sync_all();  // every CTA's partial is in its shared memory
+    constexpr int CPR = 128 / ATTN_SPLITS;  // columns finished by each rank
+    if (threadIdx.x < CPR) {
+        const int col = split * CPR + (int)threadIdx.x;
+        float pm[ATTN_SPLITS], pl[ATTN_SPLITS], po[ATTN_SPLITS];
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) {
+            pm[r] = ld_cluster_f32(&cta_ml[0], (unsigned)r);
+            pl[r] = ld_cluster_f32(&cta_ml[1], (unsigned)r);
+            po[r] = ld_cluster_f32(&cta_o[col], (unsigned)r);
+        }
+        float mm = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) mm = fmaxf(mm, pm[r]);
+        float ll = 0.f, acc = 0.f;
+#pragma unroll
+        for (int r = 0; r < ATTN_SPLITS; ++r) {
+            const float f = pm[r] == -INFINITY ? 0.f : expf(pm[r] - mm);
+            ll += pl[r] * f;
+            acc += po[r] * f;
+        }
+        if (col < hd) out[((size_t)b * T + t) * H + (size_t)h * hd + col] = acc / ll;
+    }
+    cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
+}
+
+}  // namespace
+
+size_t a48_kv_cache_bytes(int B, int nh, int cap, int hd, int bits) {
+    if (bits == 0) return (size_t)B * nh * cap * hd * 4;
+    const size_t codes = ((size_t)B * nh * cap * row_bytes(hd, bits) + 15) / 16 * 16;
+    const size_t scales = ((size_t)B * nh * cap * 4 + 15) / 16 * 16;
+    const size_t bos = bits == 3 ? ((size_t)B * nh * row_bytes(hd, 4) + 15) / 16 * 16 : 0;
+    return codes + scales + bos;
+}
+
+bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const float* v, const float2* table, double base,
+                                              int B, int T, int nh,
+                                              int hd, int pos0, int cap, int q_bits, int kv_bits, float eps, void* kcache,
+                                              void* vcache, float* dq_k, float* dq_v, cudaStream_t st) {
+    if (hd > 128 || hd % 4 != 0) return BITNET_A48_ERR_UNSUPPORTED;
+    const long long warps = (long long)B * T * nh;
+    const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
+    rope_quant_cache_kernel<<<blocks, 256, 0, st>>>(q, k, v, table, base, B, T, nh, hd, pos0, cap, q_bits, kv_bits, (double)eps, kcache,
+                                                    vcache, dq_k, dq_v);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache, const void* vcache, int B, int T, int nh,
+                                             int hd, int pos0, int cap, int kv_bits, float* out, cudaStream_t st) {
+    if (hd > 128) return BITNET_A48_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ATTN_SPLITS, (unsigned)nh, (unsigned)(B * T));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ATTN_SPLITS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_row_lowbit_kernel, q, kcache, vcache, B, T, nh, hd, pos0, cap, kv_bits,
+                                    1.f / sqrtf((float)hd), out));
+    return BITNET_A48_OK;
+}

@@ -432,6 +432,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     const bitnet_a48_block_config& c = blk->cfg;
     const int H = c.hidden, F = c.ffn, nh = c.n_heads, hd = H / nh, M = B * T;
     if (hd % 4 != 0 || hd > 256 || H % 4 != 0 || F % 4 != 0) return BITNET_A48_ERR_SHAPE;
+    if ((c.q_bits != 0 && c.q_bits != 4) || (c.kv_bits != 0 && c.kv_bits != 3 && c.kv_bits != 4)) return BITNET_A48_ERR_INVALID_ARG;
+    if ((c.q_bits != 0 || c.kv_bits != 0) && hd > 128) return BITNET_A48_ERR_UNSUPPORTED;
     if (B > 65535 || nh > 65535) return BITNET_A48_ERR_SHAPE;
     BlockWs o = block_ws(blk, B, T);
     char* base = static_cast<char*>(ws);
@@ -449,6 +451,7 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     void* lin = base + o.lin;
     const size_t lin_bytes = ws_bytes - o.lin;
     int cap = c.ctx_cap;
+    const bool caller_cache = kcache != nullptr;
     if (!kcache) {  // keys/values of this call only: keep them in the workspace
         kcache = reinterpret_cast<float*>(base + o.kc);
         vcache = reinterpret_cast<float*>(base + o.vc);
@@ -471,6 +474,28 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         float* qkv[3] = {q, k, v};
         A48_TRY(bitnet_a48_linear_multi(3, blk->w, codes, scale, M, dense_kind, qkv, lin, lin_bytes, st));
     }
+    const bool lowbit = c.q_bits != 0 || c.kv_bits != 0;
+    if (lowbit) {
+        // Section 3, low-bit attention: post-RoPE absmax quantisation of the heads; packed key/value cache
+        if (c.kv_bits != 0 && (!caller_cache || (T > 8 && pos0 != 0))) return BITNET_A48_ERR_UNSUPPORTED;
+        const bool inline_angles = T <= 8;
+        int n = T * (hd / 2);
+        if (!inline_angles) rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
+        float* dq_k = reinterpret_cast<float*>(base + o.kc);
+        float* dq_v = reinterpret_cast<float*>(base + o.vc);
+        if (c.kv_bits == 0) return BITNET_A48_ERR_UNSUPPORTED;  // quantised queries go with a quantised cache
+        const bool tile_path = T > 8;  // prefill from position 0: attention runs on the dequantised copies
+        A48_TRY(a48_launch_rope_quant_cache(q, k, v, inline_angles ? nullptr : rope, (double)c.rope_base, B, T, nh, hd, pos0,
+                                            c.ctx_cap, c.q_bits, c.kv_bits, c.quant_eps, kcache, vcache,
+                                            tile_path ? dq_k : nullptr, tile_path ? dq_v : nullptr, st));
+        if (!tile_path) {
+            A48_TRY(a48_launch_attn_row_lowbit(q, kcache, vcache, B, T, nh, hd, pos0, c.ctx_cap, c.kv_bits, att, st));
+        } else if (hd <= 64) {
+            A48_TRY(launch_attn_tile<64>(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, st));
+        } else {
+            A48_TRY(launch_attn_tile<128>(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, st));
+        }
+    } else {
     {
         int n = T * (hd / 2);
         const bool inline_angles = T <= 8;  // decode: every thread evaluates its own angle, one launch fewer
@@ -490,6 +515,7 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         A48_TRY(launch_attn_tile<128>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     } else {
         A48_TRY(launch_attn_tile<256>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+    }
     }
     if (fp4) {  // the floating-point variant quantises the attention output densely (no top-K)
         A48_TRY(a48_launch_quant_fp4(att, M, H, codes, scale, nullptr, 0.f, st));

@@ -109,6 +109,15 @@ bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int
                                            int M, float* Y, int32_t* acc, void* ws, size_t ws_bytes,
                                            cudaStream_t st);
 
+// ---- attn_lowbit.cu (Section 3, low-bit attention)
+size_t a48_kv_cache_bytes(int B, int nh, int cap, int hd, int bits);
+bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const float* v, const float2* table, double base,
+                                              int B, int T, int nh, int hd, int pos0, int cap, int q_bits, int kv_bits,
+                                              float eps, void* kcache, void* vcache, float* dq_k, float* dq_v,
+                                              cudaStream_t st);
+bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache, const void* vcache, int B, int T, int nh,
+                                             int hd, int pos0, int cap, int kv_bits, float* out, cudaStream_t st);
+
 // ---- block.cu
 size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
 bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X, int B, int T, int pos0,
