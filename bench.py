@@ -639,8 +639,10 @@ def bench_decode(a48, synth, dev, stream, peaks, rank, shape, tag):
     return out
 
 
-def bench_block_decode(a48, synth, dev, stream, shape, batches, ctx=2048, layer=None):
-    """One block forward per new token against a context of `ctx` cached positions, per batch size."""
+def bench_block_decode(a48, synth, dev, stream, shape, batches, ctx=2048, layer=None, q_bits=0, kv_bits=0):
+    """One block forward per new token against a context of `ctx` cached positions, per batch size.
+
+    kv_bits != 0: the packed low-bit cache, filled by a prefill of `ctx` tokens through the block itself."""
     Hs, Fs, nh = shape["H"], shape["F"], shape["NH"]
     own = layer is None
     if own:
@@ -648,12 +650,21 @@ def bench_block_decode(a48, synth, dev, stream, shape, batches, ctx=2048, layer=
     g1 = synth.norm_gains(Hs, 60, device=dev)
     g2 = synth.norm_gains(Hs, 61, device=dev)
     cap = ctx + 8
-    blk = a48.Block(layer.w, g1, g2, n_heads=nh, k_o=Hs // 2, k_down=Fs // 2, ctx_cap=cap)
+    blk = a48.Block(layer.w, g1, g2, n_heads=nh, k_o=Hs // 2, k_down=Fs // 2, ctx_cap=cap, q_bits=q_bits, kv_bits=kv_bits)
     out = {}
     for Bd in batches:
         xd = synth.gaussian_outlier_activations(Bd, Hs, seed=63, device=dev)
-        kcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=64, device=dev)
-        vcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=65, device=dev)
+        if kv_bits:
+            kcd = torch.zeros(blk.kv_cache_bytes(Bd), dtype=torch.uint8, device=dev)
+            vcd = torch.zeros_like(kcd)
+            xp = synth.gaussian_outlier_activations(Bd * ctx, Hs, seed=66, device=dev)
+            blk.forward(xp, Bd, ctx, 0, kcd, vcd)
+            torch.cuda.synchronize()
+            del xp
+            torch.cuda.empty_cache()
+        else:
+            kcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=64, device=dev)
+            vcd = synth.kv_cache(Bd, nh, cap, Hs // nh, seed=65, device=dev)
         yd = torch.empty_like(xd)
         wsd = torch.empty(blk.workspace_bytes(Bd, 1), dtype=torch.uint8, device=dev)
 
@@ -673,7 +684,8 @@ def bench_block_decode(a48, synth, dev, stream, shape, batches, ctx=2048, layer=
         ms = e0.elapsed_time(e1) / reps
         ms_g = graph_time_ms(call, stream, reps=reps)  # the call is stream-ordered, so a caller can capture it
         out[f"b{Bd}"] = {"tokens_per_s": Bd / (ms * 1e-3), "ms": ms, "context": ctx, "ms_cuda_graph": ms_g,
-                         "tokens_per_s_cuda_graph": Bd / (ms_g * 1e-3)}
+                         "tokens_per_s_cuda_graph": Bd / (ms_g * 1e-3),
+                         "kv_cache_bytes": 2 * (kcd.numel() * kcd.element_size())}
         del kcd, vcd
     blk.free()
     if own:
@@ -816,6 +828,9 @@ def bench_block(a48, synth, dev, stream, layer):
     torch.cuda.empty_cache()
     dec = bench_block_decode(a48, synth, dev, stream, SHAPE_7B, (1, 8), layer=layer)
     out["decode_b1"], out["decode_b8"] = dec["b1"], dec["b8"]
+    # the same steps with 4-bit queries and a 3-bit key/value cache (Section 3, low-bit attention)
+    low = bench_block_decode(a48, synth, dev, stream, SHAPE_7B, (1, 8), layer=layer, q_bits=4, kv_bits=3)
+    out["decode_b1_q4_kv3"], out["decode_b8_q4_kv3"] = low["b1"], low["b8"]
     out["note"] = "one 7B-shape block (fp32 attention glue included); tokens/s per block, not per model"
     return out
 

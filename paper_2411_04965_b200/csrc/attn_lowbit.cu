@@ -192,15 +192,45 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+constexpr int kChunkKeys = 256;  // keys staged in shared memory at a time
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+
+// Eight entries of a staged row (shared memory), as load8 does from global memory.
+__device__ __forceinline__ void unpack8(const uint8_t* row, int bits, int sub, bool inside, float (&f)[8]) {
+    unsigned w = 0;
+    if (inside) {
+        if (bits == 4) {
+            w = reinterpret_cast<const unsigned*>(row)[sub];
+        } else {
+            const unsigned* g = reinterpret_cast<const unsigned*>(row) + 3 * (sub >> 2);
+            const unsigned w0 = g[0], w1 = g[1], w2 = g[2];
+            const int i = sub & 3;
+            w = i == 0 ? w0 : (i == 1 ? __funnelshift_r(w0, w1, 24) : (i == 2 ? __funnelshift_r(w1, w2, 16) : (w2 >> 8)));
+        }
+    }
+    const unsigned mask = (1u << bits) - 1u;
+    const float offset = 8388608.f + (float)(1 << (bits - 1));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(0x4B000000u | ((w >> (bits * i)) & mask)) - offset;
+}
+
 // Decode attention over the packed cache for a few queries per sequence: the keys of one (query, head, batch) are
-// split over the ATTN_SPLITS CTAs of a cluster; inside a CTA every half-warp takes one key at a time (lane `sub`
-// of the half-warp owns entries 8 sub .. 8 sub + 7 of the head, head_dim <= 128), two keys in flight per half-warp;
-// online softmax per half-warp, then the same combination through shared memory and distributed shared memory as
-// the fp32 kernel.
+// split over the ATTN_SPLITS CTAs of a cluster.  A CTA copies its keys' codes and scales (contiguous in the cache:
+// 52 bytes per key at 3 bits) into shared memory with cp.async, up to kChunkKeys keys at a time, so that the whole
+// stretch is in flight at once; then every half-warp takes one key at a time (lane `sub` of the half-warp owns
+// entries 8 sub .. 8 sub + 7 of the head, head_dim <= 128) with online softmax per half-warp, and the partial
+// results are combined through shared memory and distributed shared memory as in the fp32 kernel.  In a 3-bit cache
+// position 0 (4-bit codes in the side table) is read straight from global memory by one half-warp.
+// Dynamic shared memory: K rows | V rows | K scales | V scales of one chunk (+ 3 keys of alignment slack each).
 __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __restrict__ q, const void* kcache, const void* vcache,
                                                               int B, int T, int nh, int hd, int pos0, int cap, int kv_bits,
                                                               float scale, float* __restrict__ out) {
     constexpr int HALVES = 16;  // half-warps per CTA
+    extern __shared__ __align__(16) uint8_t stage[];
     __shared__ float sm_m[HALVES], sm_l[HALVES];
     __shared__ float sm_o[HALVES][128];
     __shared__ float cta_ml[2];
@@ -211,6 +241,12 @@ __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __res
     const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
     const KvView kview = kv_view(const_cast<void*>(kcache), B, nh, cap, hd, kv_bits);
     const KvView vview = kv_view(const_cast<void*>(vcache), B, nh, cap, hd, kv_bits);
+    const int row = kview.row;
+    const size_t rows_bytes = ((size_t)(kChunkKeys + 3) * row + 15) / 16 * 16;
+    uint8_t* sk = stage;
+    uint8_t* sv = stage + rows_bytes;
+    float* sks = reinterpret_cast<float*>(stage + 2 * rows_bytes);
+    float* svs = sks + kChunkKeys + 4;
     float qreg[8], o[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -221,42 +257,55 @@ __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __res
     float m = -INFINITY, l = 0.f;
     const int n_keys = pos0 + t + 1;
     const int per = (n_keys + ATTN_SPLITS - 1) / ATTN_SPLITS;
-    const int j_end = min(n_keys, (split + 1) * per);
+    const int j_begin = split * per, j_end = min(n_keys, (split + 1) * per);
     const size_t head = (size_t)b * nh + h;
     const unsigned half_mask = 0xffffu << (lane & 16);
     const bool mine = 8 * sub < padded_dim(hd);
-    for (int j0 = split * per + halfw; j0 < j_end; j0 += 2 * HALVES) {
-        float kf[2][8], vf[2][8], ks[2], vs[2];
+    auto take = [&](const float (&kf)[8], const float (&vf)[8], float ks, float vs) {  // one key into the running softmax
+        float dot = 0.f;
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int j = j0 + HALVES * u;
-            const bool ok = j < j_end;
-            const int jj = ok ? j : j0;
-            const bool bos = kv_bits == 3 && jj == 0;
-            const size_t slot = head * cap + jj;
-            load8(bos ? kview.bos + head * kview.row4 : kview.codes + slot * kview.row, bos ? 4 : kv_bits, sub, mine, kf[u]);
-            load8(bos ? vview.bos + head * vview.row4 : vview.codes + slot * vview.row, bos ? 4 : kv_bits, sub, mine, vf[u]);
-            ks[u] = __ldg(kview.scales + slot);
-            vs[u] = __ldg(vview.scales + slot);
+        for (int i = 0; i < 8; ++i) dot += qreg[i] * kf[i];
+#pragma unroll
+        for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(half_mask, dot, off);
+        dot *= ks;
+        const float m_new = fmaxf(m, dot);
+        const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+        const float pr = expf(dot - m_new);
+        l = l * corr + pr;
+        const float pv = pr * vs;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = o[i] * corr + pv * vf[i];
+        m = m_new;
+    };
+    const bool bos_table = kv_bits == 3;  // position 0 is not in the 3-bit rows
+    if (bos_table && j_begin == 0 && j_end > 0 && halfw == 0) {
+        float kf[8], vf[8];
+        load8(kview.bos + head * kview.row4, 4, sub, mine, kf);
+        load8(vview.bos + head * vview.row4, 4, sub, mine, vf);
+        take(kf, vf, __ldg(kview.scales + head * cap), __ldg(vview.scales + head * cap));
+    }
+    for (int c0 = j_begin; c0 < j_end; c0 += kChunkKeys) {
+        const int c1 = min(c0 + kChunkKeys, j_end);
+        const int ca = c0 & ~3;  // copies start on a 16-byte boundary of the cache: four keys are a multiple of 16 bytes
+        const size_t first = head * cap + ca;
+        const int code_pieces = ((c1 - ca) * row + 15) / 16, scale_pieces = (c1 - ca + 3) / 4;
+        __syncthreads();  // the previous chunk has been consumed
+        for (int i = threadIdx.x; i < code_pieces; i += 256) {
+            cp_async16(sk + 16 * i, kview.codes + first * row + 16 * (size_t)i);
+            cp_async16(sv + 16 * i, vview.codes + first * row + 16 * (size_t)i);
         }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            float dot = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dot += qreg[i] * kf[u][i];
-#pragma unroll
-            for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(half_mask, dot, off);
-            dot *= ks[u];
-            if (j0 + HALVES * u < j_end) {
-                const float m_new = fmaxf(m, dot);
-                const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
-                const float pr = expf(dot - m_new);
-                l = l * corr + pr;
-                const float pv = pr * vs[u];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) o[i] = o[i] * corr + pv * vf[u][i];
-                m = m_new;
-            }
+        for (int i = threadIdx.x; i < scale_pieces; i += 256) {
+            cp_async16(sks + 4 * i, kview.scales + first + 4 * (size_t)i);
+            cp_async16(svs + 4 * i, vview.scales + first + 4 * (size_t)i);
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        for (int j = c0 + halfw; j < c1; j += HALVES) {
+            if (bos_table && j == 0) continue;
+            float kf[8], vf[8];
+            unpack8(sk + (size_t)(j - ca) * row, kv_bits, sub, mine, kf);
+            unpack8(sv + (size_t)(j - ca) * row, kv_bits, sub, mine, vf);
+            take(kf, vf, sks[j - ca], svs[j - ca]);
         }
     }
     if (sub == 0) {
@@ -316,7 +365,7 @@ size_t a48_kv_cache_bytes(int B, int nh, int cap, int hd, int bits) {
     const size_t codes = ((size_t)B * nh * cap * row_bytes(hd, bits) + 15) / 16 * 16;
     const size_t scales = ((size_t)B * nh * cap * 4 + 15) / 16 * 16;
     const size_t bos = bits == 3 ? ((size_t)B * nh * row_bytes(hd, 4) + 15) / 16 * 16 : 0;
-    return codes + scales + bos;
+    return codes + scales + bos + 16;  // (the attention kernel copies whole 16-byte pieces: slack for the last one)
 }
 
 bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const float* v, const float2* table, double base,
@@ -346,6 +395,8 @@ bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache,
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    const size_t rows_bytes = ((size_t)(kChunkKeys + 3) * row_bytes(hd, kv_bits) + 15) / 16 * 16;
+    cfg.dynamicSmemBytes = 2 * rows_bytes + 2 * (size_t)(kChunkKeys + 4) * sizeof(float);  // at most 36 KB
     A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_row_lowbit_kernel, q, kcache, vcache, B, T, nh, hd, pos0, cap, kv_bits,
                                     1.f / sqrtf((float)hd), out));
     return BITNET_A48_OK;

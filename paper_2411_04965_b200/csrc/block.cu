@@ -434,6 +434,7 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     if (hd % 4 != 0 || hd > 256 || H % 4 != 0 || F % 4 != 0) return BITNET_A48_ERR_SHAPE;
     if ((c.q_bits != 0 && c.q_bits != 4) || (c.kv_bits != 0 && c.kv_bits != 3 && c.kv_bits != 4)) return BITNET_A48_ERR_INVALID_ARG;
     if ((c.q_bits != 0 || c.kv_bits != 0) && hd > 128) return BITNET_A48_ERR_UNSUPPORTED;
+    if (c.kv_bits != 0 && c.ctx_cap % 4 != 0) return BITNET_A48_ERR_SHAPE;  // packed rows are copied in 16-byte pieces
     if (B > 65535 || nh > 65535) return BITNET_A48_ERR_SHAPE;
     BlockWs o = block_ws(blk, B, T);
     char* base = static_cast<char*>(ws);
