@@ -94,6 +94,7 @@ __global__ void __launch_bounds__(256) rope_quant_cache_kernel(float* __restrict
                                                                int hd, int pos0, int cap, int q_bits, int kv_bits, double eps,
                                                                void* kcache, void* vcache, float* __restrict__ dq_k,
                                                                float* __restrict__ dq_v) {
+    a48_pdl_prologue();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= B * T * nh) return;
     const int h = warp % nh, m = warp / nh, t = m % T, b = m / T;
@@ -235,6 +236,7 @@ __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __res
     __shared__ float sm_o[HALVES][128];
     __shared__ float cta_ml[2];
     __shared__ float cta_o[128];
+    a48_pdl_prologue();
     const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z / T, t = blockIdx.z % T;
     const int lane = threadIdx.x & 31, sub = lane & 15, halfw = threadIdx.x >> 4;
     const size_t H = (size_t)nh * hd;
@@ -375,9 +377,8 @@ bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const fl
     if (hd > 128 || hd % 4 != 0) return BITNET_A48_ERR_UNSUPPORTED;
     const long long warps = (long long)B * T * nh;
     const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-    rope_quant_cache_kernel<<<blocks, 256, 0, st>>>(q, k, v, table, base, B, T, nh, hd, pos0, cap, q_bits, kv_bits, (double)eps, kcache,
-                                                    vcache, dq_k, dq_v);
-    A48_CUDA_TRY(cudaGetLastError());
+    A48_CUDA_TRY(a48_launch_pdl(rope_quant_cache_kernel, dim3(blocks), dim3(256), 0, st, q, k, v, table, base, B, T, nh, hd, pos0,
+                                cap, q_bits, kv_bits, (double)eps, kcache, vcache, dq_k, dq_v));
     return BITNET_A48_OK;
 }
 
@@ -388,13 +389,15 @@ bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache,
     cfg.gridDim = dim3(ATTN_SPLITS, (unsigned)nh, (unsigned)(B * T));
     cfg.blockDim = dim3(256);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = ATTN_SPLITS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     const size_t rows_bytes = ((size_t)(kChunkKeys + 3) * row_bytes(hd, kv_bits) + 15) / 16 * 16;
     cfg.dynamicSmemBytes = 2 * rows_bytes + 2 * (size_t)(kChunkKeys + 4) * sizeof(float);  // at most 36 KB
     A48_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_row_lowbit_kernel, q, kcache, vcache, B, T, nh, hd, pos0, cap, kv_bits,

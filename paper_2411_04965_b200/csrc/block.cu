@@ -64,6 +64,7 @@ __global__ void rope_table_kernel(int pos0, int T, int half, double base, float2
 __global__ void rope_cache_kernel(float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                                   const float2* __restrict__ table, double base, int B, int T, int nh, int hd, int pos0,
                                   int cap, float* __restrict__ kcache, float* __restrict__ vcache) {
+    a48_pdl_prologue();
     const int half = hd / 2;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     size_t total = (size_t)B * T * nh * half;
@@ -269,6 +270,7 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
     __shared__ float sm_o[8][COLS];
     __shared__ float cta_ml[2];  // this CTA's running max and sum, read by the peers
     __shared__ float cta_o[COLS];
+    a48_pdl_prologue();
     const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z / T, t = blockIdx.z % T;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t H = (size_t)nh * hd;
@@ -384,18 +386,21 @@ cudaError_t launch_attn_row(const float* q, const float* kcache, const float* vc
     cfg.gridDim = dim3(ATTN_SPLITS, (unsigned)nh, (unsigned)(B * T));
     cfg.blockDim = dim3(256);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = ATTN_SPLITS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, attn_row_kernel<CPL>, q, kcache, vcache, T, nh, hd, pos0, cap,
                               1.f / sqrtf((float)hd), out);
 }
 
 __global__ void add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ y, size_t n4) {
+    a48_pdl_prologue();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
     float4 x = reinterpret_cast<const float4*>(a)[i], z = reinterpret_cast<const float4*>(b)[i];
@@ -502,9 +507,9 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         const bool inline_angles = T <= 8;  // decode: every thread evaluates its own angle, one launch fewer
         if (!inline_angles) rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
         size_t total = (size_t)M * nh * (hd / 2);
-        rope_cache_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(q, k, v, inline_angles ? nullptr : rope,
-                                                                          (double)c.rope_base, B, T, nh, hd, pos0, cap,
-                                                                          kcache, vcache);
+        A48_CUDA_TRY(a48_launch_pdl(rope_cache_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, q, k, v,
+                                    inline_angles ? nullptr : rope, (double)c.rope_base, B, T, nh, hd, pos0, cap, kcache,
+                                    vcache));
     }
     if (T <= 8) {
         if (hd <= 64) A48_CUDA_TRY(launch_attn_row<2>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
@@ -531,7 +536,7 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         if (fp4) A48_TRY(a48_launch_quant_fp4_add(X, tmp, hres, M, H, codes, scale, blk->g_ffn, c.norm_eps, st));
         else A48_TRY(a48_launch_quant_int4_add(X, tmp, hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
     } else {
-        add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(X, tmp, hres, nH4);
+        A48_CUDA_TRY(a48_launch_pdl(add_kernel, dim3((unsigned)((nH4 + 255) / 256)), dim3(256), 0, st, X, tmp, hres, nH4));
         if (fp4) A48_TRY(a48_launch_quant_fp4(hres, M, H, codes, scale, blk->g_ffn, c.norm_eps, st));
         else A48_TRY(a48_launch_quant_int4(hres, M, H, c.quant_eps, codes, scale, blk->g_ffn, c.norm_eps, st));
     }
@@ -547,7 +552,7 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
     }
     A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));
-    add_kernel<<<(unsigned)((nH4 + 255) / 256), 256, 0, st>>>(hres, tmp, Y, nH4);
+    A48_CUDA_TRY(a48_launch_pdl(add_kernel, dim3((unsigned)((nH4 + 255) / 256)), dim3(256), 0, st, hres, tmp, Y, nH4));
 #undef A48_TRY
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;

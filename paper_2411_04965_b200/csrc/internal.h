@@ -12,6 +12,32 @@
         if (err__ != cudaSuccess) return BITNET_A48_ERR_CUDA; \
     } while (0)
 
+// Launch with programmatic dependent launch allowed: the kernel may be made resident while the kernel ahead of it in
+// the stream still runs.  Kernels launched this way call a48_pdl_prologue() before they touch memory, which waits
+// for that predecessor to complete, so the ordering a plain launch gives is kept and only the launch latency is
+// hidden (it is several microseconds per launch in a decode step made of a dozen tiny kernels).
+#ifdef __CUDACC__
+__device__ __forceinline__ void a48_pdl_prologue() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t a48_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                         Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 static inline bool a48_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int a48_round_up(int x, int m) { return (x + m - 1) / m * m; }
 

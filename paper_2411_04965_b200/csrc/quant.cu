@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restr
                                                             const float* __restrict__ R, float* __restrict__ SUM) {
     constexpr int G = kBlock / TPR;
     __shared__ double red[kBlock / 32];
+    a48_pdl_prologue();
     const int group = threadIdx.x / TPR, t = threadIdx.x % TPR;
     const int row = blockIdx.x * G + group;
     if (row >= M) return;
@@ -213,8 +214,8 @@ void launch_int4(const float* X, int M, int K, double eps, int8_t* codes, float*
     const int nv = K / 4;
     const bool fast = (K % 4 == 0) && nv <= 256 * 12;
 #define A48_Q4(TPR, V)                                                                                             \
-    quant_int4_kernel<TPR, V, NORM, ADD, FP4><<<(M + (kBlock / TPR) - 1) / (kBlock / TPR), kBlock, 0, st>>>(      \
-        X, M, K, eps, codes, scale, gain, norm_eps, R, SUM)
+    a48_launch_pdl(quant_int4_kernel<TPR, V, NORM, ADD, FP4>, dim3((M + (kBlock / TPR) - 1) / (kBlock / TPR)),    \
+                   dim3(kBlock), 0, st, X, M, K, eps, codes, scale, gain, norm_eps, R, SUM)
     if (!fast && FP4) quant_fp4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, codes, scale, gain, norm_eps);
     else if (!fast) quant_int4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, eps, codes, scale, gain, norm_eps);
     else if (nv <= 32 * 4) A48_Q4(32, 4);

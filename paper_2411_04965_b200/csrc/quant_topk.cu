@@ -208,6 +208,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     __shared__ unsigned cand_idx[G][kCand];
     __shared__ unsigned sel[G][8];
     __shared__ unsigned red[kBlock / 32];
+    a48_pdl_prologue();
     const int group = threadIdx.x / TPR, t = threadIdx.x % TPR;
     const int row = blockIdx.x * G + group;
     if (row >= M) return;
@@ -445,7 +446,8 @@ __global__ void __launch_bounds__(kBlock)
 template <int TPR, int V, bool GLU, bool EXACT>
 void launch_one(const float* X, const float* U, int M, int K, int k, double e, int8_t* codes, float* scale, cudaStream_t st) {
     constexpr int G = kBlock / TPR;
-    topk_quant_int8_kernel<TPR, V, GLU, EXACT><<<(M + G - 1) / G, kBlock, 0, st>>>(X, U, M, K, k, e, codes, scale);
+    a48_launch_pdl(topk_quant_int8_kernel<TPR, V, GLU, EXACT>, dim3((M + G - 1) / G), dim3(kBlock), 0, st, X, U, M, K, k, e, codes,
+                   scale);
 }
 
 template <bool GLU>
