@@ -98,11 +98,6 @@ bitnet_a48_status bitnet_a48_weight_unpack_layout(const bitnet_a48_weight* w, un
 bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int* K, unsigned* layout_flags);
 /* Bytes of packed weight data a kernel reads for this matrix (N*K/4 rounded up per row). */
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w);
-/* Asks the GPU to pull one packed layout of the matrix (BITNET_A48_LAYOUT_DECODE or _GEMM) into its L2 cache.
- * A hint with no effect on results: a decode loop calls it on a second stream for the matrix it will need next,
- * so that the bytes leave HBM while the current BitLinear still runs (at batch 1 a 7B-shape matrix is about
- * 1.7 us of HBM time but several us of launch and dependency latency).  Enqueues one small kernel on `stream`. */
-bitnet_a48_status bitnet_a48_weight_prefetch(const bitnet_a48_weight* w, unsigned layout, void* stream);
 void bitnet_a48_weight_free(bitnet_a48_weight* w);
 
 /* ---------------------------------------------------------------------------
@@ -150,8 +145,10 @@ bitnet_a48_status bitnet_a48_quant_fp4(const float* X_dev, int M, int K, int8_t*
  *   Y[m,n]   = fp32(acc[m,n]) · (scale[m] · alpha)
  * codes_dev int8 [M,K], scale_dev fp32 [M], Y_dev fp32 [M,N]; acc_dev is NULL or
  * int32 [M,N] (the raw accumulators, for parity checks).  `kind` tells which
- * quantiser made the codes (it selects the zero-skipping decode path for
- * top-K inputs at M == 1; the result does not depend on it).
+ * quantiser made the codes (the result does not depend on it; for top-K inputs at
+ * M == 1 it lets the call take the zero-skipping kernel when the handle carries the
+ * SPARSE layout but not the DECODE one - with both present the dense streaming
+ * kernel is the faster of the two at model shapes and is taken).
  * workspace_dev: at least bitnet_a48_linear_workspace_bytes(w, M) bytes, or NULL
  * when that is 0.  The decode kernel (M <= 8) adds the partial sums of tiles that
  * two CTAs share into this scratch: it must be zero-filled before its first use
@@ -172,7 +169,7 @@ size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
 /* Several BitLinears on the SAME activation codes (Eq. 6: q, k and v share the attention input; gate and up
  * share the FFN input): Y_dev[j] = BitLinear(weights[j]) for j < count, all weights with the same K.
  * For M <= 8 and count <= 4 with the DECODE layout this is one launch that streams the matrices as one
- * sequence of tiles (a launch costs more than the HBM time of one 7B-shape matrix); for 9..1023 tokens,
+ * sequence of tiles (a launch costs more than the HBM time of one 7B-shape matrix); for 9..383 tokens,
  * count <= 4 and the GEMM layout it is one launch of the tensor-core kernel over the tiles of all matrices;
  * otherwise it is `count` calls of bitnet_a48_linear one after the other.  Results are identical to separate
  * calls.

@@ -32,7 +32,7 @@ EXPORTS = [
     "bitnet_a48_block_free", "bitnet_a48_block_workspace_bytes", "bitnet_a48_block_forward",
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
-    "bitnet_a48_weight_prefetch", "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
+    "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
     "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes",
 ]
 
@@ -72,7 +72,6 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_weight_unpack.argtypes = [c_void_p, c_void_p, POINTER(c_float), c_void_p]
         L.bitnet_a48_weight_unpack_layout.argtypes = [c_void_p, c_uint, c_void_p, c_void_p]
         L.bitnet_a48_weight_dims.argtypes = [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_uint)]
-        L.bitnet_a48_weight_prefetch.argtypes = [c_void_p, c_uint, c_void_p]
         L.bitnet_a48_weight_free.argtypes = [c_void_p]
         L.bitnet_a48_weight_free.restype = None
         L.bitnet_a48_quant_int4.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p]
@@ -157,10 +156,6 @@ def pack_ternary(W: torch.Tensor, eps: float = 1e-5, layouts: int = LAYOUT_ALL, 
     out = c_void_p(0)
     _check(lib().bitnet_a48_pack_ternary(_ptr(W), N, K, eps, layouts, byref(out), _stream(stream)), "pack_ternary")
     return Weight(out.value, N, K, layouts)
-
-
-def weight_prefetch(w: Weight, layout: int = LAYOUT_DECODE, stream=None):
-    _check(lib().bitnet_a48_weight_prefetch(c_void_p(w.handle), layout, _stream(stream)), "weight_prefetch")
 
 
 def weight_unpack(w: Weight, stream=None):

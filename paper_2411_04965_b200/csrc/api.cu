@@ -124,12 +124,6 @@ bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int
 
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w) { return w ? (size_t)w->N * w->K4 : 0; }
 
-bitnet_a48_status bitnet_a48_weight_prefetch(const bitnet_a48_weight* w, unsigned layout, void* stream) {
-    if (!w) return BITNET_A48_ERR_INVALID_ARG;
-    if (!have_device()) return BITNET_A48_ERR_CUDA;
-    return a48_launch_prefetch(w, layout, (cudaStream_t)stream);
-}
-
 void bitnet_a48_weight_free(bitnet_a48_weight* w) {
     if (!w) return;
     free_weight_buffers(w);
@@ -191,19 +185,32 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
         return BITNET_A48_ERR_ALIGNMENT;
     if (!have_device()) return BITNET_A48_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    if (algo == BITNET_A48_ALGO_AUTO) {
+    const bool automatic = algo == BITNET_A48_ALGO_AUTO;
+    if (automatic) {
         // At the 3B/7B shapes one launch is latency-bound, and the dense kernel (dp4a on whole rows) beats the
         // zero-skipping one although it moves twice the bytes; the latter is taken when it is the only one possible.
         if (a48_decode_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE;
         else if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE_SPARSE;
-        else if (M >= 1024 && a48_gemm_pair_supported(w, M))
-            algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // measured 4-16 % ahead of the single-CTA form from 1024 tokens on
+        else if (M >= 384 && a48_gemm_pair_supported(w, M))
+            algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // measured 3-11 % ahead of the single-CTA form from 384 tokens on
         else if (a48_gemm_tcgen05_supported(w, M, false))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05;
         else
             algo = BITNET_A48_ALGO_SIMPLE;
+    }
+    if (automatic && algo == BITNET_A48_ALGO_GEMM_TCGEN05_PAIR) {
+        // the pair form can still decline (a device that cannot host a two-CTA cluster of this size, a shape beyond its
+        // index arithmetic): the library's own choice then falls back to the single-CTA form, then to the simple kernel
+        bitnet_a48_status s = a48_launch_gemm_pair(w, codes_dev, scale_dev, M, Y_dev, acc_dev, st);
+        if (s != BITNET_A48_ERR_UNSUPPORTED && s != BITNET_A48_ERR_SHAPE) return s;
+        algo = a48_gemm_tcgen05_supported(w, M, false) ? BITNET_A48_ALGO_GEMM_TCGEN05 : BITNET_A48_ALGO_SIMPLE;
+    }
+    if (automatic && algo == BITNET_A48_ALGO_GEMM_TCGEN05) {
+        bitnet_a48_status s = a48_launch_gemm_tcgen05(w, codes_dev, scale_dev, M, Y_dev, acc_dev, false, st);
+        if (s != BITNET_A48_ERR_UNSUPPORTED && s != BITNET_A48_ERR_SHAPE) return s;
+        algo = BITNET_A48_ALGO_SIMPLE;
     }
     switch (algo) {
         case BITNET_A48_ALGO_SIMPLE:
@@ -269,8 +276,8 @@ bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* co
     {  // beyond the decode kernel's token count: one tensor-core launch over the tiles of all matrices
         bool any_decode = false;
         for (int j = 0; j < count; ++j) any_decode = any_decode || a48_decode_supported(weights[j], M);
-        // (from 1024 tokens on a launch per matrix on CTA pairs is faster than the grouped single-CTA launch)
-        if (!any_decode && M < 1024 && a48_gemm_tcgen05_multi_supported(count, weights, M))
+        // (from 384 tokens on a launch per matrix on CTA pairs is faster than the grouped single-CTA launch)
+        if (!any_decode && M < 384 && a48_gemm_tcgen05_multi_supported(count, weights, M))
             return a48_launch_gemm_tcgen05_multi(count, weights, codes_dev, scale_dev, M, Y_dev, (cudaStream_t)stream);
     }
     for (int j = 0; j < count; ++j) {

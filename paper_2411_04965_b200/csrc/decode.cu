@@ -682,41 +682,3 @@ extern "C" bitnet_a48_status bitnet_a48_linear_decode_static(const bitnet_a48_we
     A48_CUDA_TRY(cudaMemsetAsync(g_static_scratch_ptr[dev], 0, bytes, st));
     return a48_launch_decode(w, codes_dev, scale_dev, M, Y_dev, nullptr, g_static_scratch_ptr[dev], bytes, st);
 }
-
-// ---------------------------------------------------------------------------------------------------------------
-// L2 prefetch of a packed matrix: lets a decode loop pull the next matrix out of HBM while the current one computes.
-namespace {
-
-constexpr uint32_t kPrefetchChunk = 8192;
-
-__global__ void __launch_bounds__(32) prefetch_l2_kernel(const uint8_t* __restrict__ base, size_t bytes) {
-    const size_t stride = (size_t)gridDim.x * blockDim.x * kPrefetchChunk;
-    for (size_t off = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * kPrefetchChunk; off < bytes; off += stride) {
-        const size_t left = bytes - off;
-        const uint32_t size = (uint32_t)(left < kPrefetchChunk ? left : kPrefetchChunk) & ~15u;  // a multiple of 16 bytes
-        if (size) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(size) : "memory");
-    }
-}
-
-}  // namespace
-
-bitnet_a48_status a48_launch_prefetch(const bitnet_a48_weight* w, unsigned layout, cudaStream_t st) {
-    const uint8_t* base = nullptr;
-    size_t bytes = 0;
-    if (layout == BITNET_A48_LAYOUT_DECODE && w->decode) {
-        base = w->decode;
-        bytes = (size_t)((w->N + 15) / 16) * (w->Kp / 128) * UNIT_BYTES;  // the tiles that hold real rows
-    } else if (layout == BITNET_A48_LAYOUT_GEMM && w->gemm) {
-        base = w->gemm;
-        bytes = (size_t)w->Np * w->Kp / 4;
-    } else {
-        return BITNET_A48_ERR_UNSUPPORTED;
-    }
-    const size_t chunks = (bytes + kPrefetchChunk - 1) / kPrefetchChunk;
-    unsigned blocks = (unsigned)((chunks + 31) / 32);
-    if (blocks > (unsigned)sm_count()) blocks = (unsigned)sm_count();
-    if (blocks == 0) return BITNET_A48_OK;
-    prefetch_l2_kernel<<<blocks, 32, 0, st>>>(base, bytes);
-    A48_CUDA_TRY(cudaGetLastError());
-    return BITNET_A48_OK;
-}

@@ -1,6 +1,6 @@
 // Zero-skipping decode BitLinear for one token whose codes come from the top-K quantiser (Eq. 1): only the
-// weight rows of input channels with a non-zero code are fetched, which is what the paper means by sparsity
-// reducing "the I/O of weight".  It reads the channel-major layout (row k = the 2-bit codes of every output for
+// weight rows of input channels with a non-zero code are fetched: the saving in weight traffic that the paper
+// attributes to activation sparsity (Section 1; Eq. 1).  It reads the channel-major layout (row k = the 2-bit codes of every output for
 // channel k, see SparseLayout), so skipping a channel skips one contiguous row.
 //
 // Grid: (blocks of 1024 outputs) x (segments of the channel range).  A CTA first lists the non-zero channels of
@@ -99,8 +99,10 @@ int sm_count() {
 
 }  // namespace
 
+// The segments of one output meet in a 64-bit word whose low 40 bits add up one biased sum (about 2^31) per
+// segment: at most 255 segments of at most MAX_SEG channels keep that sum below 2^40.
 bool a48_decode_sparse_supported(const bitnet_a48_weight* w, int M) {
-    return w->sparse != nullptr && M == 1 && w->K < (1 << 24);
+    return w->sparse != nullptr && M == 1 && (w->K + MAX_SEG - 1) / MAX_SEG <= 255;
 }
 
 size_t a48_decode_sparse_workspace_bytes(const bitnet_a48_weight* w, int M) {
@@ -117,11 +119,12 @@ bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int
     const int nblocks = (w->N + NB - 1) / NB;
     int nseg = (2 * sm_count() + nblocks - 1) / nblocks;  // about two CTAs per SM
     if (nseg < 1) nseg = 1;
+    if (nseg > 255) nseg = 255;  // what the meeting word has room for
     int seg_len = (w->K + nseg - 1) / nseg;
     if (seg_len < 32) seg_len = 32;
     if (seg_len > MAX_SEG) seg_len = MAX_SEG;
     nseg = (w->K + seg_len - 1) / seg_len;
-    if (nseg > 65535) return BITNET_A48_ERR_UNSUPPORTED;
+    if (nseg > 255) return BITNET_A48_ERR_UNSUPPORTED;  // (also what a48_decode_sparse_supported promises)
     dim3 grid((unsigned)nblocks, (unsigned)nseg);
     decode_sparse_kernel<<<grid, THREADS, 0, st>>>(reinterpret_cast<const uint32_t*>(w->sparse), row_words, codes, scale,
                                                   w->alpha_dev, Y, acc, static_cast<unsigned long long*>(ws), w->N,

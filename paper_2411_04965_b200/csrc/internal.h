@@ -130,7 +130,6 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
                                           const float* scale, int M, float* const* Y, int32_t* const* acc, void* ws,
                                           size_t ws_bytes, cudaStream_t st);
 bitnet_a48_status a48_read_decode_status(unsigned int words_host[4]);
-bitnet_a48_status a48_launch_prefetch(const bitnet_a48_weight* w, unsigned layout, cudaStream_t st);
 bitnet_a48_status a48_launch_decode_sparse(const bitnet_a48_weight* w, const int8_t* codes, const float* scale,
                                            int M, float* Y, int32_t* acc, void* ws, size_t ws_bytes,
                                            cudaStream_t st);

@@ -121,3 +121,24 @@ def test_decode_sparse_matches_oracle(a48, oracle, cuda_dev, N, K, kfrac):
         assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
         assert int(scratch.count_nonzero()) == 0
     w.free()
+
+
+def test_decode_sparse_segment_bound(a48, oracle, cuda_dev):
+    # the segments of an output meet in one 64-bit word that has room for 255 of them (512 channels each): the widest
+    # supported row is exact, one channel more is declined before anything is launched
+    N, K = 48, 255 * 512
+    W = synth.latent_weights(N, K, seed=77)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_SPARSE)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    x = synth.student_t3(1, K, seed=78)
+    codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+    c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS)
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, _ = oracle.linear(c_ref, d_ref, t_ref, alpha)
+    _, acc = a48.linear(w, codes, scale, a48.ACT_TOPK_INT8, a48.ALGO_DECODE_SPARSE, want_acc=True)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    wide = a48.pack_ternary(synth.latent_weights(16, K + 16, seed=79).to(cuda_dev), EPS, a48.LAYOUT_SPARSE)
+    with pytest.raises(a48.A48Error) as e:
+        a48.linear(wide, torch.zeros(1, K + 16, dtype=torch.int8, device=cuda_dev), torch.ones(1, device=cuda_dev),
+                   a48.ACT_TOPK_INT8, a48.ALGO_DECODE_SPARSE)
+    assert e.value.code == 4

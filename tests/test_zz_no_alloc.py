@@ -30,6 +30,22 @@ def test_static_scratch_decode_matches_workspace_decode(a48, cuda_dev):
     assert a48.kernel_status() == [0, 0, 0, 0]
 
 
+def test_static_scratch_decode_at_its_limit_and_after_a_smaller_call(a48, cuda_dev):
+    # 16384 output features fill the built-in array exactly; the call before it used (and cleared) only a small part
+    # of the array, so the large call meets a region no earlier call of this test has cleared
+    small = a48.pack_ternary(synth.latent_weights(320, 2048, seed=8).to(cuda_dev), EPS, a48.LAYOUT_DECODE)
+    large = a48.pack_ternary(synth.latent_weights(16384, 256, seed=9).to(cuda_dev), EPS, a48.LAYOUT_DECODE)
+    for w, M in ((small, 3), (large, 8), (small, 1), (large, 2)):
+        x = synth.gaussian_outlier_activations(M, w.K, seed=91 + M).to(cuda_dev)
+        codes, scale = a48.quant_int4(x, EPS)
+        expected = a48.linear(w, codes, scale, a48.ACT_INT4, a48.ALGO_DECODE)
+        got = torch.full((M, w.N), float("nan"), device=cuda_dev)
+        a48.linear_decode_static(w, codes, scale, got)
+        torch.cuda.synchronize()
+        assert torch.equal(got, expected)
+    assert a48.kernel_status() == [0, 0, 0, 0]
+
+
 def test_static_scratch_decode_rejects_what_it_cannot_hold(a48, cuda_dev):
     wide = a48.pack_ternary(synth.latent_weights(16400, 128, seed=6).to(cuda_dev), EPS, a48.LAYOUT_DECODE)
     codes = torch.zeros(1, 128, dtype=torch.int8, device=cuda_dev)
