@@ -56,6 +56,9 @@ typedef enum {
 /* One int8 code per weight (4x the packed size); only the shared-memory-operand
  * variant of the tensor-core kernel reads it.  Not part of LAYOUT_ALL. */
 #define BITNET_A48_LAYOUT_I8 8u
+/* Five codes per byte (b = sum (t_i + 1) 3^i, 1.6 bits per weight: the "1.58-bit" of Section 1 rounded up to whole
+ * bytes), row-major, rows padded to 16 bytes; read by the BITNET_A48_ALGO_DECODE_TRIT5 kernel.  Not part of LAYOUT_ALL. */
+#define BITNET_A48_LAYOUT_TRIT5 16u
 
 /* Kernel selection for bitnet_a48_linear_ex (tests and benchmarks force one). */
 typedef enum {
@@ -65,7 +68,8 @@ typedef enum {
     BITNET_A48_ALGO_DECODE = 3,       /* M <= 8: streams every weight byte once */
     BITNET_A48_ALGO_DECODE_SPARSE = 4, /* M == 1: fetches only channels whose code is non-zero */
     BITNET_A48_ALGO_GEMM_TCGEN05_I8 = 5, /* comparison variant: int8 weight copy staged through shared memory */
-    BITNET_A48_ALGO_GEMM_TCGEN05_PAIR = 6 /* tcgen05 cta_group::2: two SMs per tile of 256 weight rows */
+    BITNET_A48_ALGO_GEMM_TCGEN05_PAIR = 6, /* tcgen05 cta_group::2: two SMs per tile of 256 weight rows */
+    BITNET_A48_ALGO_DECODE_TRIT5 = 7  /* M <= 8 over the five-codes-per-byte layout (a fifth fewer weight bytes) */
 } bitnet_a48_algo;
 
 typedef struct bitnet_a48_weight bitnet_a48_weight; /* packed ternary matrix + alpha + N, K */
@@ -98,6 +102,8 @@ bitnet_a48_status bitnet_a48_weight_unpack_layout(const bitnet_a48_weight* w, un
 bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int* K, unsigned* layout_flags);
 /* Bytes of packed weight data a kernel reads for this matrix (N*K/4 rounded up per row). */
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w);
+/* Bytes of one optional layout (a single BITNET_A48_LAYOUT_* bit) as stored, 0 if the handle does not carry it. */
+size_t bitnet_a48_weight_layout_bytes(const bitnet_a48_weight* w, unsigned layout);
 void bitnet_a48_weight_free(bitnet_a48_weight* w);
 
 /* ---------------------------------------------------------------------------

@@ -18,9 +18,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libbitnet_a48.so")
 
 ACT_INT4, ACT_TOPK_INT8, ACT_FP4 = 0, 1, 2
-LAYOUT_GEMM, LAYOUT_DECODE, LAYOUT_SPARSE, LAYOUT_ALL, LAYOUT_I8 = 1, 2, 4, 7, 8
+LAYOUT_GEMM, LAYOUT_DECODE, LAYOUT_SPARSE, LAYOUT_ALL, LAYOUT_I8, LAYOUT_TRIT5 = 1, 2, 4, 7, 8, 16
 ALGO_AUTO, ALGO_SIMPLE, ALGO_GEMM_TCGEN05, ALGO_DECODE, ALGO_DECODE_SPARSE, ALGO_GEMM_TCGEN05_I8 = 0, 1, 2, 3, 4, 5
 ALGO_GEMM_TCGEN05_PAIR = 6
+ALGO_DECODE_TRIT5 = 7
 
 EXPORTS = [
     "bitnet_a48_status_string", "bitnet_a48_pack_ternary", "bitnet_a48_weight_unpack",
@@ -33,7 +34,7 @@ EXPORTS = [
     "bitnet_a48_kernel_status", "bitnet_a48_linear_decode_static", "bitnet_a48_linear_multi",
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
     "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
-    "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes",
+    "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes", "bitnet_a48_weight_layout_bytes",
 ]
 
 
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
                      "bitnet_a48_bitlinear_host_workspace_bytes", "bitnet_a48_block_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         L.bitnet_a48_weight_packed_bytes.argtypes = [c_void_p]
+        L.bitnet_a48_weight_layout_bytes.restype = c_size_t
+        L.bitnet_a48_weight_layout_bytes.argtypes = [c_void_p, c_uint]
         L.bitnet_a48_linear_workspace_bytes.argtypes = [c_void_p, c_int]
         L.bitnet_a48_bitlinear_host_workspace_bytes.argtypes = [c_void_p, c_int]
         L.bitnet_a48_block_workspace_bytes.argtypes = [c_void_p, c_int, c_int]
@@ -148,6 +151,9 @@ class Weight:
     @property
     def packed_bytes(self) -> int:
         return int(lib().bitnet_a48_weight_packed_bytes(c_void_p(self.handle)))
+
+    def layout_bytes(self, layout: int) -> int:
+        return int(lib().bitnet_a48_weight_layout_bytes(c_void_p(self.handle), layout))
 
 
 def pack_ternary(W: torch.Tensor, eps: float = 1e-5, layouts: int = LAYOUT_ALL, stream=None) -> Weight:

@@ -26,6 +26,7 @@ void free_weight_buffers(bitnet_a48_weight* w) {
     cudaFree(w->decode);
     cudaFree(w->sparse);
     cudaFree(w->i8);
+    cudaFree(w->trit5);
 }
 
 bitnet_a48_status check_act_args(const void* X, int M, int K, const void* codes, const void* scale) {
@@ -57,7 +58,7 @@ const char* bitnet_a48_status_string(bitnet_a48_status s) {
 
 bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, float eps, unsigned layout_flags,
                                           bitnet_a48_weight** out, void* stream) {
-    if (!W_dev || !out || (layout_flags & ~(BITNET_A48_LAYOUT_ALL | BITNET_A48_LAYOUT_I8)) || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
+    if (!W_dev || !out || (layout_flags & ~(BITNET_A48_LAYOUT_ALL | BITNET_A48_LAYOUT_I8 | BITNET_A48_LAYOUT_TRIT5)) || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
     if (N <= 0 || K <= 0 || K >= (1 << 24) || (size_t)N * (size_t)K >= ((size_t)1 << 40)) return BITNET_A48_ERR_SHAPE;
     if (!a48_aligned16(W_dev)) return BITNET_A48_ERR_ALIGNMENT;
     if (!have_device()) return BITNET_A48_ERR_CUDA;
@@ -71,6 +72,7 @@ bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, floa
     w->flags = layout_flags;
     w->decode_bytes = (size_t)w->Np * w->Kp / 4;
     w->sparse_bytes = (size_t)K * w->Np / 4;
+    w->trit5_row = a48_round_up((K + 4) / 5, 16);
     bool ok = cudaMalloc(&w->alpha_dev, 16) == cudaSuccess && cudaMalloc(&w->alpha64_dev, 16) == cudaSuccess &&
               cudaMalloc(&w->partial_dev, 1024 * sizeof(double)) == cudaSuccess &&
               cudaMalloc(&w->l0, (size_t)N * w->K4) == cudaSuccess;
@@ -78,6 +80,7 @@ bitnet_a48_status bitnet_a48_pack_ternary(const float* W_dev, int N, int K, floa
     if (ok && (layout_flags & BITNET_A48_LAYOUT_DECODE)) ok = cudaMalloc(&w->decode, w->decode_bytes) == cudaSuccess;
     if (ok && (layout_flags & BITNET_A48_LAYOUT_SPARSE)) ok = cudaMalloc(&w->sparse, w->sparse_bytes) == cudaSuccess;
     if (ok && (layout_flags & BITNET_A48_LAYOUT_I8)) ok = cudaMalloc(&w->i8, (size_t)w->Np * w->Kp) == cudaSuccess;
+    if (ok && (layout_flags & BITNET_A48_LAYOUT_TRIT5)) ok = cudaMalloc(&w->trit5, (size_t)N * w->trit5_row) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         free_weight_buffers(w);
@@ -123,6 +126,18 @@ bitnet_a48_status bitnet_a48_weight_dims(const bitnet_a48_weight* w, int* N, int
 }
 
 size_t bitnet_a48_weight_packed_bytes(const bitnet_a48_weight* w) { return w ? (size_t)w->N * w->K4 : 0; }
+
+size_t bitnet_a48_weight_layout_bytes(const bitnet_a48_weight* w, unsigned layout) {
+    if (!w) return 0;
+    switch (layout) {
+        case BITNET_A48_LAYOUT_GEMM: return w->gemm ? (size_t)w->Np * w->Kp / 4 : 0;
+        case BITNET_A48_LAYOUT_DECODE: return w->decode ? w->decode_bytes : 0;
+        case BITNET_A48_LAYOUT_SPARSE: return w->sparse ? w->sparse_bytes : 0;
+        case BITNET_A48_LAYOUT_I8: return w->i8 ? (size_t)w->Np * w->Kp : 0;
+        case BITNET_A48_LAYOUT_TRIT5: return w->trit5 ? (size_t)w->N * w->trit5_row : 0;
+        default: return 0;
+    }
+}
 
 void bitnet_a48_weight_free(bitnet_a48_weight* w) {
     if (!w) return;
@@ -178,7 +193,7 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
                                        int M, bitnet_a48_act kind, bitnet_a48_algo algo, float* Y_dev,
                                        int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
     if (!w || !codes_dev || !scale_dev || !Y_dev) return BITNET_A48_ERR_INVALID_ARG;
-    if ((int)kind < 0 || (int)kind > 2 || (int)algo < 0 || (int)algo > 6) return BITNET_A48_ERR_INVALID_ARG;
+    if ((int)kind < 0 || (int)kind > 2 || (int)algo < 0 || (int)algo > 7) return BITNET_A48_ERR_INVALID_ARG;
     if (M <= 0) return BITNET_A48_ERR_SHAPE;
     if (!a48_aligned16(codes_dev) || !a48_aligned16(scale_dev) || !a48_aligned16(Y_dev) || !a48_aligned16(acc_dev) ||
         !a48_aligned16(workspace_dev))
@@ -193,6 +208,8 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
             algo = BITNET_A48_ALGO_DECODE;
         else if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE_SPARSE;
+        else if (a48_decode_trit5_supported(w, M) && !w->gemm)
+            algo = BITNET_A48_ALGO_DECODE_TRIT5;  // a handle packed for decode at 1.6 bits per weight only
         else if (M >= 384 && a48_gemm_pair_supported(w, M))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // measured 3-11 % ahead of the single-CTA form from 384 tokens on
         else if (a48_gemm_tcgen05_supported(w, M, false))
@@ -226,6 +243,8 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
         case BITNET_A48_ALGO_DECODE:
             if (!a48_decode_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
             return a48_launch_decode(w, codes_dev, scale_dev, M, Y_dev, acc_dev, workspace_dev, workspace_bytes, st);
+        case BITNET_A48_ALGO_DECODE_TRIT5:
+            return a48_launch_decode_trit5(w, codes_dev, scale_dev, M, Y_dev, acc_dev, st);
         case BITNET_A48_ALGO_DECODE_SPARSE:
             if (!a48_decode_sparse_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
             return a48_launch_decode_sparse(w, codes_dev, scale_dev, M, Y_dev, acc_dev, workspace_dev,

@@ -59,6 +59,8 @@ struct bitnet_a48_weight {
     uint8_t* decode;       // fragment-major layout (or NULL)
     uint8_t* sparse;       // channel-major layout (or NULL)
     int8_t* i8;            // int8 codes [Np][Kp], zero padded (or NULL)
+    uint8_t* trit5;        // five codes per byte, row-major, trit5_row bytes per row (or NULL)
+    int trit5_row;         // ceil(K/5) rounded up to 16
     size_t decode_bytes, sparse_bytes;
     // false until the first decode launch: that one is fully ordered after the packing kernels, later ones may
     // start fetching weights while the kernel ahead of them in the stream is still finishing
@@ -142,6 +144,11 @@ bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const fl
                                               cudaStream_t st);
 bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache, const void* vcache, int B, int T, int nh,
                                              int hd, int pos0, int cap, int kv_bits, float* out, cudaStream_t st);
+
+// ---- decode_trit5.cu
+bool a48_decode_trit5_supported(const bitnet_a48_weight* w, int M);
+bitnet_a48_status a48_launch_decode_trit5(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
+                                          int32_t* acc, cudaStream_t st);
 
 // ---- block.cu
 size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);

@@ -117,6 +117,30 @@ __global__ void expand_i8_kernel(const uint8_t* __restrict__ l0, int N, int K, i
     dst[idx] = (n < N && k < K) ? (int8_t)a48_l0_code(l0, K4, n, k) : (int8_t)0;
 }
 
+// Five codes per byte: b = sum_i (t_i + 1) * 3^i over channels 5j .. 5j+4 of a row (code 0 past K and in the row padding).
+__global__ void pack_trit5_kernel(const uint8_t* __restrict__ l0, int N, int K, int K4, int row_bytes, uint8_t* __restrict__ dst) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)N * row_bytes) return;
+    const int n = (int)(idx / row_bytes), j = (int)(idx % row_bytes);
+    unsigned b = 0, pw = 1;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const int k = 5 * j + i;
+        b += (unsigned)((k < K ? a48_l0_code(l0, K4, n, k) : 0) + 1) * pw;
+        pw *= 3;
+    }
+    dst[idx] = (uint8_t)b;
+}
+
+__global__ void unpack_trit5_kernel(const uint8_t* __restrict__ src, int N, int K, int row_bytes, int8_t* __restrict__ codes) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)N * K) return;
+    const int n = (int)(idx / K), k = (int)(idx % K);
+    unsigned b = src[(size_t)n * row_bytes + k / 5];
+    for (int i = 0; i < k % 5; ++i) b /= 3;
+    codes[idx] = (int8_t)((int)(b % 3) - 1);
+}
+
 template <class Layout>
 void run_relayout(const bitnet_a48_weight* w, Layout lay, uint8_t* dst, size_t bytes, cudaStream_t st) {
     size_t nwords = bytes / 4;
@@ -146,6 +170,10 @@ bitnet_a48_status a48_launch_pack(bitnet_a48_weight* w, const float* W_dev, floa
     if (w->gemm) run_relayout(w, GemmLayout{w->Kp}, w->gemm, (size_t)w->Np * w->Kp / 4, st);
     if (w->decode) run_relayout(w, DecodeLayout{w->Kp}, w->decode, w->decode_bytes, st);
     if (w->sparse) run_relayout(w, SparseLayout{w->Np}, w->sparse, w->sparse_bytes, st);
+    if (w->trit5) {
+        size_t nb = (size_t)w->N * w->trit5_row;
+        pack_trit5_kernel<<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(w->l0, w->N, w->K, w->K4, w->trit5_row, w->trit5);
+    }
     if (w->i8) {
         size_t n8 = (size_t)w->Np * w->Kp;
         expand_i8_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(w->l0, w->N, w->K, w->K4, w->Np, w->Kp, w->i8);
@@ -169,7 +197,10 @@ bitnet_a48_status a48_launch_unpack_layout(const bitnet_a48_weight* w, unsigned 
         run_unpack_layout(w, DecodeLayout{w->Kp}, w->decode, w->decode_bytes, codes_dev, st);
     else if (layout == BITNET_A48_LAYOUT_SPARSE && w->sparse)
         run_unpack_layout(w, SparseLayout{w->Np}, w->sparse, w->sparse_bytes, codes_dev, st);
-    else
+    else if (layout == BITNET_A48_LAYOUT_TRIT5 && w->trit5) {
+        size_t n = (size_t)w->N * w->K;
+        unpack_trit5_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w->trit5, w->N, w->K, w->trit5_row, codes_dev);
+    } else
         return BITNET_A48_ERR_UNSUPPORTED;
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;

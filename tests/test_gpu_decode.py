@@ -142,3 +142,35 @@ def test_decode_sparse_segment_bound(a48, oracle, cuda_dev):
         a48.linear(wide, torch.zeros(1, K + 16, dtype=torch.int8, device=cuda_dev), torch.ones(1, device=cuda_dev),
                    a48.ACT_TOPK_INT8, a48.ALGO_DECODE_SPARSE)
     assert e.value.code == 4
+
+
+@pytest.mark.parametrize("N,K", [(16, 128), (130, 144), (1000, 250), (3200, 3200), (4096, 11008), (11008, 4096), (257, 129)])
+@pytest.mark.parametrize("M", [1, 3, 8])
+def test_decode_trit5_matches_oracle(a48, oracle, cuda_dev, N, K, M):
+    # five ternary codes per byte (1.6 bits per weight): the packed bytes are the base-3 numbers of the oracle's codes,
+    # the layout unpacks to the same matrix, and the kernel that reads it gives the oracle's accumulators
+    W = synth.latent_weights(N, K, seed=N + K + 5)
+    w = a48.pack_ternary(W.to(cuda_dev), EPS, a48.LAYOUT_TRIT5)
+    t_ref, alpha = oracle.ternarise(W.numpy(), EPS)
+    assert np.array_equal(a48.weight_unpack_layout(w, a48.LAYOUT_TRIT5).cpu().numpy(), t_ref)
+    row = ((K + 4) // 5 + 15) // 16 * 16
+    assert w.layout_bytes(a48.LAYOUT_TRIT5) == N * row and row * 8 <= 1.6 * K + 16 * 8 + 8
+    kind = "int4" if M != 3 else "topk"
+    if kind == "int4":
+        x = synth.gaussian_outlier_activations(M, K, seed=N)
+        codes, scale = a48.quant_int4(x.to(cuda_dev), EPS)
+        c_ref, d_ref = oracle.quant_int4(x.numpy(), EPS)
+        act = a48.ACT_INT4
+    else:
+        x = synth.student_t3(M, K, seed=N)
+        codes, scale, _ = a48.topk_quant_int8(x.to(cuda_dev), K // 2, EPS)
+        c_ref, d_ref, _ = oracle.topk_quant_int8(x.numpy(), K // 2, EPS)
+        act = a48.ACT_TOPK_INT8
+    assert np.array_equal(codes.cpu().numpy(), c_ref)
+    acc_ref, y_ref = oracle.linear(c_ref, d_ref, t_ref, alpha, nthreads=8)
+    y, acc = a48.linear(w, codes, scale, act, a48.ALGO_DECODE_TRIT5, want_acc=True)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert max_rel_err(y.cpu().numpy(), y_ref) <= 1e-5
+    y2 = a48.linear(w, codes, scale, act, a48.ALGO_AUTO)  # the handle carries nothing else: AUTO takes this kernel
+    assert torch.equal(y, y2)
+    w.free()

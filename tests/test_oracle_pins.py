@@ -264,3 +264,19 @@ def test_compacted_rows_reproduce_the_dense_contraction(oracle):
     acc_dense, y_dense = oracle.linear(codes, d, t, alpha)
     acc_list, y_list = oracle.linear_from_lists(lists, d, t, alpha)
     assert np.array_equal(acc_dense, acc_list) and np.array_equal(y_dense, y_list)
+
+
+def test_five_codes_per_byte_is_the_base3_number_of_the_codes():
+    # the densest whole-byte packing of ternary codes (Section 1 counts log2(3) = 1.58 bits per weight): 3^5 = 243
+    # values fit a byte, so five codes cost 8 bits = 1.6 bits each, and the packing is invertible
+    import itertools
+    import math
+    seen = set()
+    for t in itertools.product((-1, 0, 1), repeat=5):
+        b = sum((ti + 1) * 3 ** i for i, ti in enumerate(t))
+        assert 0 <= b <= 242
+        back = tuple((b // 3 ** i) % 3 - 1 for i in range(5))
+        assert back == t
+        seen.add(b)
+    assert len(seen) == 243 and 3 ** 5 <= 256 < 3 ** 6
+    assert 8 / 5 == 1.6 and math.log2(3) < 1.6
