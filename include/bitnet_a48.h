@@ -172,6 +172,21 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
                                        int32_t* acc_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 size_t bitnet_a48_linear_workspace_bytes(const bitnet_a48_weight* w, int M);
 
+/* ---------------------------------------------------------------------------
+ * bf16 activations at the boundary (Section 1: the activations around the 4- and 8-bit codes are what is left to move
+ * once the weights are 1.58-bit; bf16 halves those bytes).  The quantisers read bf16 rows, widened exactly to fp32
+ * and then quantised as Eq. 7 / Eq. 1 + 3 say (same codes and scales as the fp32 entry points give on the widened
+ * values); the contraction writes bf16(Y) = round-to-nearest-even of the fp32 result of Eq. 1 / Eq. 6.
+ * X_bf16_dev uint16 [M, K] (bf16 bit patterns), K a multiple of 8 and at most 12288; Y_bf16_dev uint16 [M, N].
+ * bitnet_a48_linear_bf16 picks its kernel like bitnet_a48_linear (decode for M <= 8, tensor-core forms above). */
+bitnet_a48_status bitnet_a48_quant_int4_bf16(const uint16_t* X_bf16_dev, int M, int K, float eps, int8_t* codes_dev,
+                                             float* scale_dev, void* stream);
+bitnet_a48_status bitnet_a48_topk_quant_int8_bf16(const uint16_t* X_bf16_dev, int M, int K, int k, float eps,
+                                                  int8_t* codes_dev, float* scale_dev, void* stream);
+bitnet_a48_status bitnet_a48_linear_bf16(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
+                                         int M, bitnet_a48_act kind, uint16_t* Y_bf16_dev, void* workspace_dev,
+                                         size_t workspace_bytes, void* stream);
+
 /* Several BitLinears on the SAME activation codes (Eq. 6: q, k and v share the attention input; gate and up
  * share the FFN input): Y_dev[j] = BitLinear(weights[j]) for j < count, all weights with the same K.
  * For M <= 8 and count <= 4 with the DECODE layout this is one launch that streams the matrices as one

@@ -35,6 +35,7 @@ EXPORTS = [
     "bitnet_a48_linear_multi_workspace_bytes", "bitnet_a48_bitlinear_host_async",
     "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
     "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes", "bitnet_a48_weight_layout_bytes",
+    "bitnet_a48_quant_int4_bf16", "bitnet_a48_topk_quant_int8_bf16", "bitnet_a48_linear_bf16",
 ]
 
 
@@ -96,6 +97,10 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_block_forward.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                                c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_kernel_status.argtypes = [POINTER(c_uint)]
+        L.bitnet_a48_quant_int4_bf16.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p]
+        L.bitnet_a48_topk_quant_int8_bf16.argtypes = [c_void_p, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p]
+        L.bitnet_a48_linear_bf16.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t,
+                                             c_void_p]
         L.bitnet_a48_kv_cache_bytes.restype = c_size_t
         L.bitnet_a48_kv_cache_bytes.argtypes = [c_void_p, c_int]
         L.bitnet_a48_linear_multi.argtypes = [c_int, POINTER(c_void_p), c_void_p, c_void_p, c_int, c_int, POINTER(c_void_p),
@@ -200,6 +205,42 @@ def topk_quant_int8(X: torch.Tensor, k: int, eps: float = 1e-5, codes=None, scal
     _check(lib().bitnet_a48_topk_quant_int8(_ptr(X), M, K, k, eps, _ptr(codes), _ptr(scale), _ptr(mask_bits),
                                             _stream(stream)), "topk_quant_int8")
     return codes, scale, mask_bits
+
+
+def quant_int4_bf16(X: torch.Tensor, eps: float = 1e-5, codes=None, scale=None, stream=None):
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and X.dim() == 2
+    M, K = X.shape
+    codes = codes if codes is not None else torch.empty(M, K, dtype=torch.int8, device=X.device)
+    scale = scale if scale is not None else torch.empty(M, dtype=torch.float32, device=X.device)
+    _check(lib().bitnet_a48_quant_int4_bf16(_ptr(X), M, K, eps, _ptr(codes), _ptr(scale), _stream(stream)),
+           "quant_int4_bf16")
+    return codes, scale
+
+
+def topk_quant_int8_bf16(X: torch.Tensor, k: int, eps: float = 1e-5, codes=None, scale=None, stream=None):
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and X.dim() == 2
+    M, K = X.shape
+    codes = codes if codes is not None else torch.empty(M, K, dtype=torch.int8, device=X.device)
+    scale = scale if scale is not None else torch.empty(M, dtype=torch.float32, device=X.device)
+    _check(lib().bitnet_a48_topk_quant_int8_bf16(_ptr(X), M, K, k, eps, _ptr(codes), _ptr(scale), _stream(stream)),
+           "topk_quant_int8_bf16")
+    return codes, scale
+
+
+def linear_bf16(w: Weight, codes: torch.Tensor, scale: torch.Tensor, kind: int = ACT_INT4, Y=None, workspace=None,
+                stream=None):
+    """BitLinear with a bf16 output (round-to-nearest-even of the fp32 result)."""
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.is_contiguous() and codes.shape[1] == w.K
+    M = codes.shape[0]
+    Y = Y if Y is not None else torch.empty(M, w.N, dtype=torch.bfloat16, device=codes.device)
+    assert Y.dtype == torch.bfloat16 and Y.is_contiguous()
+    need = linear_workspace_bytes(w, M)
+    if workspace is None and need:
+        workspace = torch.zeros(need, dtype=torch.uint8, device=codes.device)
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib().bitnet_a48_linear_bf16(c_void_p(w.handle), _ptr(codes), _ptr(scale), M, kind, _ptr(Y), _ptr(workspace),
+                                        ws_bytes, _stream(stream)), "linear_bf16")
+    return Y
 
 
 def quant_fp4(X: torch.Tensor, codes=None, scale=None, stream=None):

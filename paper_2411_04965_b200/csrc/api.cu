@@ -3,6 +3,8 @@
 
 #include "internal.h"
 
+thread_local int a48_y_bf16 = 0;
+
 namespace {
 
 constexpr int kMaxFeatures = 1 << 20;
@@ -206,9 +208,9 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
         // zero-skipping one although it moves twice the bytes; the latter is taken when it is the only one possible.
         if (a48_decode_supported(w, M))
             algo = BITNET_A48_ALGO_DECODE;
-        else if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M))
+        else if (M == 1 && kind == BITNET_A48_ACT_TOPK_INT8 && a48_decode_sparse_supported(w, M) && !a48_y_bf16)
             algo = BITNET_A48_ALGO_DECODE_SPARSE;
-        else if (a48_decode_trit5_supported(w, M) && !w->gemm)
+        else if (a48_decode_trit5_supported(w, M) && !w->gemm && !a48_y_bf16)
             algo = BITNET_A48_ALGO_DECODE_TRIT5;  // a handle packed for decode at 1.6 bits per weight only
         else if (M >= 384 && a48_gemm_pair_supported(w, M))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // measured 3-11 % ahead of the single-CTA form from 384 tokens on
@@ -259,6 +261,33 @@ bitnet_a48_status bitnet_a48_linear(const bitnet_a48_weight* w, const int8_t* co
                                     void* workspace_dev, size_t workspace_bytes, void* stream) {
     return bitnet_a48_linear_ex(w, codes_dev, scale_dev, M, kind, BITNET_A48_ALGO_AUTO, Y_dev, acc_dev,
                                 workspace_dev, workspace_bytes, stream);
+}
+
+bitnet_a48_status bitnet_a48_linear_bf16(const bitnet_a48_weight* w, const int8_t* codes_dev, const float* scale_dev,
+                                         int M, bitnet_a48_act kind, uint16_t* Y_bf16_dev, void* workspace_dev,
+                                         size_t workspace_bytes, void* stream) {
+    a48_y_bf16 = 1;  // the kernels this call launches store bf16
+    const bitnet_a48_status s = bitnet_a48_linear_ex(w, codes_dev, scale_dev, M, kind, BITNET_A48_ALGO_AUTO,
+                                                     reinterpret_cast<float*>(Y_bf16_dev), nullptr, workspace_dev,
+                                                     workspace_bytes, stream);
+    a48_y_bf16 = 0;
+    return s;
+}
+
+bitnet_a48_status bitnet_a48_quant_int4_bf16(const uint16_t* X_bf16_dev, int M, int K, float eps, int8_t* codes_dev,
+                                             float* scale_dev, void* stream) {
+    bitnet_a48_status s = check_act_args(X_bf16_dev, M, K, codes_dev, scale_dev);
+    if (s != BITNET_A48_OK) return s;
+    if (!(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
+    return a48_launch_quant_int4_bf16(X_bf16_dev, M, K, eps, codes_dev, scale_dev, (cudaStream_t)stream);
+}
+
+bitnet_a48_status bitnet_a48_topk_quant_int8_bf16(const uint16_t* X_bf16_dev, int M, int K, int k, float eps,
+                                                  int8_t* codes_dev, float* scale_dev, void* stream) {
+    bitnet_a48_status s = check_act_args(X_bf16_dev, M, K, codes_dev, scale_dev);
+    if (s != BITNET_A48_OK) return s;
+    if (k < 1 || k > K || !(eps >= 0.f)) return BITNET_A48_ERR_INVALID_ARG;
+    return a48_launch_topk_quant_int8_bf16(X_bf16_dev, M, K, k, eps, codes_dev, scale_dev, (cudaStream_t)stream);
 }
 
 size_t bitnet_a48_linear_multi_workspace_bytes(int count, const bitnet_a48_weight* const weights[], int M) {

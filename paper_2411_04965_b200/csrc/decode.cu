@@ -135,6 +135,7 @@ struct DecodeParams {
     int tile_aligned;     // pieces end on tile boundaries: no tile is shared, the scratch stays untouched
     int piece_q, piece_r; // the first piece_r pieces hold piece_q + 1 items (tiles if tile_aligned, else units), the rest piece_q
     int act_row_bytes;    // padded K + 16
+    int y_bf16;           // outputs are bf16 instead of fp32
 };
 
 __device__ __forceinline__ int matrix_of(const DecodeParams& p, int tile) {
@@ -492,7 +493,7 @@ __global__ void __launch_bounds__(32 * NW, ONE_TOKEN ? 2 : 1) decode_kernel(cons
         if (n < p.N[j]) {
             const int v = (int)sum - csum[m];
             const size_t o = (size_t)m * p.N[j] + (size_t)n;
-            p.Y[j][o] = (float)v * (p.scale[m] * __ldg(p.alpha[j]));  // prefactors of Eq. 2, 3 and 7
+            a48_store_y(p.Y[j], o, (float)v * (p.scale[m] * __ldg(p.alpha[j])), p.y_bf16);  // prefactors of Eq. 2, 3 and 7
             if (p.acc[j]) p.acc[j][o] = v;
         }
     }
@@ -568,6 +569,7 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     if (ntiles * p.kchunks >= (1ll << 31)) return BITNET_A48_ERR_UNSUPPORTED;
     p.units = (int)(ntiles * p.kchunks);
     p.act_row_bytes = w->Kp + 16;
+    p.y_bf16 = a48_y_bf16;
     // one piece per SM unless a piece would then not fit: at most MAX_SHARE units and MAX_TILES tiles per piece
     long long grid = sm_count();
     if (grid > p.units) grid = p.units;

@@ -280,6 +280,7 @@ struct GemmParams {
     const uint8_t* wt[MAX_MATS];   // tile-major packed weights (TS)
     const float* alpha[MAX_MATS];  // device scalars
     float* Y[MAX_MATS];            // [M, N_j]
+    int y_bf16;                    // outputs are bf16 instead of fp32
     int N[MAX_MATS];
     int tile_base[MAX_MATS + 1];
     int count;
@@ -583,7 +584,11 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
                 float* yp = p.Y[mj] + o;
                 const float* sp = p.scale + mrow;
                 // y = fp32(acc) * (scale[m] * alpha): the prefactors of Eq. 2, 3 and 7
-                if (valid >= 32) {
+                if (p.y_bf16) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) a48_store_y(p.Y[mj], o + (size_t)j * N, (float)(int)r[j] * (__ldg(sp + j) * alpha), 1);
+                } else if (valid >= 32) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
@@ -628,7 +633,7 @@ __global__ void __launch_bounds__((Cfg<TS, TM>::NUM_THREADS), 1)
                         if (q < p.ksplit) sum += slots[(q * per + row) * TILE_N + nl];
                     const int m = m0 + rank * per + row;
                     const size_t e = (size_t)m * N + n;
-                    p.Y[mj][e] = (float)sum * (__ldg(p.scale + m) * alpha);
+                    a48_store_y(p.Y[mj], e, (float)sum * (__ldg(p.scale + m) * alpha), p.y_bf16);
                     if (p.acc) p.acc[e] = sum;
                 }
             }
@@ -695,6 +700,7 @@ struct PairParams {
     const float* alpha;
     const float* scale;
     float* Y;
+    int y_bf16;  // outputs are bf16 instead of fp32
     int32_t* acc;
     int M, N, kblocks, n_pairs, m_tiles;
     int n_tiles128;  // 128-row weight tiles in the packed layout; an odd count leaves the last pair's second CTA
@@ -893,7 +899,11 @@ __global__ void __launch_bounds__(PC::NUM_THREADS, 1)
                 if (n >= p.N) continue;
                 float* yp = p.Y + o;
                 const float* sp = p.scale + mrow;
-                if (valid >= 32) {
+                if (p.y_bf16) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < valid) a48_store_y(p.Y, o + (size_t)j * p.N, (float)(int)r[j] * (__ldg(sp + j) * alpha), 1);
+                } else if (valid >= 32) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         *yp = (float)(int)r[j] * (__ldg(sp + j) * alpha);
@@ -1059,6 +1069,7 @@ bitnet_a48_status launch(int count, const bitnet_a48_weight* const* ws, const in
     }
     p.scale = scale;
     p.acc = acc;
+    p.y_bf16 = a48_y_bf16;
     p.M = M;
     p.K = w->K;
     p.kblocks = w->Kp / BK;
@@ -1098,6 +1109,7 @@ bitnet_a48_status launch_pair(const bitnet_a48_weight* w, const int8_t* codes, c
     p.alpha = w->alpha_dev;
     p.scale = scale;
     p.Y = Y;
+    p.y_bf16 = a48_y_bf16;
     p.acc = acc;
     p.M = M;
     p.N = w->N;

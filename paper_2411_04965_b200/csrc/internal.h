@@ -38,6 +38,19 @@ static inline cudaError_t a48_launch_pdl(void (*kernel)(KArgs...), dim3 grid, di
 }
 #endif
 
+// Output element type of the contraction kernels for the call in flight on this host thread: 0 = fp32, 1 = bf16
+// (round to nearest even of the fp32 result).  Set by bitnet_a48_linear_bf16 around its dispatch, read by the
+// launchers, which pass it to their kernels as a parameter.
+extern thread_local int a48_y_bf16;
+#ifdef __CUDACC__
+#include <cuda_bf16.h>
+// Stores y as element `index` of an fp32 or a bf16 array.
+__device__ __forceinline__ void a48_store_y(float* base, size_t index, float y, int bf16) {
+    if (bf16) reinterpret_cast<__nv_bfloat16*>(base)[index] = __float2bfloat16_rn(y);
+    else base[index] = y;
+}
+#endif
+
 static inline bool a48_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int a48_round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -88,6 +101,11 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
 bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k, float eps, int8_t* codes,
                                              float* scale, uint32_t* mask_bits, cudaStream_t st);
 bool a48_topk_quant_fast_shape(int K);
+// bf16 rows in (widened exactly to fp32), otherwise as the fp32 forms
+bitnet_a48_status a48_launch_quant_int4_bf16(const uint16_t* X, int M, int K, float eps, int8_t* codes, float* scale,
+                                             cudaStream_t st);
+bitnet_a48_status a48_launch_topk_quant_int8_bf16(const uint16_t* X, int M, int K, int k, float eps, int8_t* codes,
+                                                  float* scale, cudaStream_t st);
 bitnet_a48_status a48_launch_quant_int4_add(const float* X, const float* R, float* SUM, int M, int K, float eps,
                                             int8_t* codes, float* scale, const float* gain, float norm_eps,
                                             cudaStream_t st);

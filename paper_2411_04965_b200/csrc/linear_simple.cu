@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(256) linear_simple_kernel(const uint8_t* __res
                                                             const int8_t* __restrict__ codes,
                                                             const float* __restrict__ scale,
                                                             const float* __restrict__ alpha, int M, int N, int K,
-                                                            float* __restrict__ Y, int32_t* __restrict__ acc_out) {
+                                                            float* __restrict__ Y, int32_t* __restrict__ acc_out, int y_bf16) {
     __shared__ uint32_t sa[BM][BK / 4 + 1];
     __shared__ uint32_t sw[BN][BK / 4 + 1];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // tx: outputs tx, tx+32; ty: tokens 4ty..4ty+3
@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(256) linear_simple_kernel(const uint8_t* __res
         for (int j = 0; j < 2; ++j) {
             int n = n0 + tx + 32 * j;
             if (n >= N) continue;
-            Y[(size_t)m * N + n] = (float)acc[i][j] * s;
+            a48_store_y(Y, (size_t)m * N + n, (float)acc[i][j] * s, y_bf16);
             if (acc_out) acc_out[(size_t)m * N + n] = acc[i][j];
         }
     }
@@ -78,7 +78,7 @@ bitnet_a48_status a48_launch_linear_simple(const bitnet_a48_weight* w, const int
                                            int M, float* Y, int32_t* acc, cudaStream_t st) {
     dim3 grid((w->N + BN - 1) / BN, (M + BM - 1) / BM);
     if (grid.y > 65535) return BITNET_A48_ERR_SHAPE;
-    linear_simple_kernel<<<grid, 256, 0, st>>>(w->l0, w->K4, codes, scale, w->alpha_dev, M, w->N, w->K, Y, acc);
+    linear_simple_kernel<<<grid, 256, 0, st>>>(w->l0, w->K4, codes, scale, w->alpha_dev, M, w->N, w->K, Y, acc, a48_y_bf16);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }

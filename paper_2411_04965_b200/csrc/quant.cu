@@ -50,7 +50,7 @@ __device__ __forceinline__ int fp4_grid_code(double xp) {
 
 // FP4 false: Eq. 7 (absmean, codes in [-8, 7]).  FP4 true: Eq. 8-9 (MinMax E2M1, grid codes) with the same
 // fused front ends.
-template <int TPR, int V, bool NORM, bool ADD, bool FP4 = false>
+template <int TPR, int V, bool NORM, bool ADD, bool FP4 = false, bool BF16IN = false>
 __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restrict__ X, int M, int K, double eps,
                                                             int8_t* __restrict__ codes, float* __restrict__ scale,
                                                             const float* __restrict__ gain, double norm_eps,
@@ -62,12 +62,12 @@ __global__ void __launch_bounds__(kBlock) quant_int4_kernel(const float* __restr
     const int row = blockIdx.x * G + group;
     if (row >= M) return;
     const int nv = K >> 2;
-    const float4* xr = reinterpret_cast<const float4*>(X + (size_t)row * K);
+    const void* xr = row_ptr<BF16IN>(X, (size_t)row, K);
     float4 v[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         int idx = i * TPR + t;
-        v[i] = idx < nv ? __ldg(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[i] = idx < nv ? load_row4<BF16IN>(xr, idx) : make_float4(0.f, 0.f, 0.f, 0.f);
         if (ADD && idx < nv) {
             const float4 r = __ldg(reinterpret_cast<const float4*>(R + (size_t)row * K) + idx);
             v[i] = make_float4(v[i].x + r.x, v[i].y + r.y, v[i].z + r.z, v[i].w + r.w);
@@ -208,13 +208,13 @@ __global__ void __launch_bounds__(kBlock) compact_codes_kernel(const int8_t* __r
     if (t == 0) count[row] = (int32_t)running;
 }
 
-template <bool NORM, bool ADD = false, bool FP4 = false>
+template <bool NORM, bool ADD = false, bool FP4 = false, bool BF16IN = false>
 void launch_int4(const float* X, int M, int K, double eps, int8_t* codes, float* scale, const float* gain,
                  double norm_eps, cudaStream_t st, const float* R = nullptr, float* SUM = nullptr) {
     const int nv = K / 4;
     const bool fast = (K % 4 == 0) && nv <= 256 * 12;
 #define A48_Q4(TPR, V)                                                                                             \
-    a48_launch_pdl(quant_int4_kernel<TPR, V, NORM, ADD, FP4>, dim3((M + (kBlock / TPR) - 1) / (kBlock / TPR)),    \
+    a48_launch_pdl(quant_int4_kernel<TPR, V, NORM, ADD, FP4, BF16IN>, dim3((M + (kBlock / TPR) - 1) / (kBlock / TPR)),    \
                    dim3(kBlock), 0, st, X, M, K, eps, codes, scale, gain, norm_eps, R, SUM)
     if (!fast && FP4) quant_fp4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, codes, scale, gain, norm_eps);
     else if (!fast) quant_int4_generic_kernel<NORM><<<M, kBlock, 0, st>>>(X, M, K, eps, codes, scale, gain, norm_eps);
@@ -233,6 +233,14 @@ bitnet_a48_status a48_launch_quant_int4(const float* X, int M, int K, float eps,
                                         const float* gain, float norm_eps, cudaStream_t st) {
     if (gain) launch_int4<true>(X, M, K, (double)eps, codes, scale, gain, (double)norm_eps, st);
     else launch_int4<false>(X, M, K, (double)eps, codes, scale, nullptr, 0.0, st);
+    A48_CUDA_TRY(cudaGetLastError());
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_launch_quant_int4_bf16(const uint16_t* X, int M, int K, float eps, int8_t* codes, float* scale,
+                                             cudaStream_t st) {
+    if (!((K % 4 == 0) && K / 4 <= 256 * 12)) return BITNET_A48_ERR_UNSUPPORTED;  // the register kernels only
+    launch_int4<false, false, false, true>(reinterpret_cast<const float*>(X), M, K, (double)eps, codes, scale, nullptr, 0.0, st);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
 }

@@ -89,4 +89,20 @@ __device__ __forceinline__ unsigned group_excl_scan(unsigned cnt, unsigned* red,
     return base + incl - cnt;
 }
 
+// Four consecutive entries of a row that is fp32 or (BF16) bf16 in memory; `row` is the row's first byte.  A bf16
+// value widens to fp32 exactly: its 16 bits are the upper half of the fp32 pattern.
+template <bool BF16>
+__device__ __forceinline__ float4 load_row4(const void* row, int idx) {
+    if (BF16) {
+        const uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + idx);
+        return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                           __uint_as_float(u.y & 0xffff0000u));
+    }
+    return __ldg(reinterpret_cast<const float4*>(row) + idx);
+}
+template <bool BF16>
+__device__ __forceinline__ const void* row_ptr(const void* X, size_t row, int K) {
+    return reinterpret_cast<const char*>(X) + row * (size_t)K * (BF16 ? 2 : 4);
+}
+
 }  // namespace a48q

@@ -79,7 +79,7 @@ __device__ __forceinline__ void scan_bins(const unsigned* hist, unsigned kr, uns
 // the ranking list holds): the row is read again (it is in L2), a group-wide scan per 4*TPR entries numbers the
 // entries equal to tau so that the lowest indices win, float64 rounding throughout.  Not unrolled: it is rarely run
 // and must not crowd the instruction cache of the common path.
-template <int TPR, bool GLU>
+template <int TPR, bool GLU, bool BF16IN = false>
 __device__ __noinline__ void cold_final(const float* __restrict__ xrow, const float* __restrict__ urow, int K, unsigned tau,
                                         unsigned keep_eq, bool ordered, double mult, int8_t* __restrict__ crow,
                                         uint32_t* __restrict__ mrow, unsigned* red, int group, int t) {
@@ -90,7 +90,7 @@ __device__ __noinline__ void cold_final(const float* __restrict__ xrow, const fl
     for (int i0 = 0; i0 < nv; i0 += TPR) {
         const int idx = i0 + t;
         const bool valid = idx < nv;
-        float4 x = valid ? __ldg(reinterpret_cast<const float4*>(xrow) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 x = valid ? load_row4<BF16IN>(xrow, idx) : make_float4(0.f, 0.f, 0.f, 0.f);
         if (GLU && valid) {
             const float4 u = __ldg(reinterpret_cast<const float4*>(urow) + idx);
             auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
@@ -157,7 +157,7 @@ __device__ __forceinline__ bool bin_lower_end(unsigned b, float lo, float inv_w,
 }
 
 // Cold path of one row: exact 4-pass radix select over the row re-read from memory, then cold_final.
-template <int TPR, bool GLU>
+template <int TPR, bool GLU, bool BF16IN>
 __device__ __noinline__ void cold_row(const float* __restrict__ xrow, const float* __restrict__ urow, int K, int k, double mult,
                                       int8_t* __restrict__ crow, unsigned* hist, unsigned* sel, unsigned* red, int group,
                                       int t) {
@@ -170,7 +170,7 @@ __device__ __noinline__ void cold_row(const float* __restrict__ xrow, const floa
         group_sync<TPR>(group);
 #pragma unroll 1
         for (int idx = t; idx < nv; idx += TPR) {
-            float4 x = __ldg(reinterpret_cast<const float4*>(xrow) + idx);
+            float4 x = load_row4<BF16IN>(xrow, idx);
             if (GLU) {
                 const float4 u = __ldg(reinterpret_cast<const float4*>(urow) + idx);
                 auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
@@ -191,13 +191,13 @@ __device__ __noinline__ void cold_row(const float* __restrict__ xrow, const floa
         eq_total = sel[2];
         group_sync<TPR>(group);  // sel is rewritten by the next scan only after every thread has read it
     }
-    cold_final<TPR, GLU>(xrow, urow, K, prefix, kr, eq_total != kr, mult, crow, nullptr, red, group, t);
+    cold_final<TPR, GLU, BF16IN>(xrow, urow, K, prefix, kr, eq_total != kr, mult, crow, nullptr, red, group, t);
 }
 
 // GLU: the row to quantise is up * ReLU(gate)^2 (Eq. 5), formed while loading: X is the gate projection and U the up
 // projection, and the product never goes to memory.
 // EXACT: V == ceil(K/4 / TPR), so only the last of a thread's V vectors can lie beyond the row.
-template <int TPR, int V, bool GLU, bool EXACT>
+template <int TPR, int V, bool GLU, bool EXACT, bool BF16IN = false>
 __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     topk_quant_int8_kernel(const float* __restrict__ X, const float* __restrict__ U, int M, int K, int k, double eps,
                            int8_t* __restrict__ codes, float* __restrict__ scale) {
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
     const int row = blockIdx.x * G + group;
     if (row >= M) return;
     const int nv = K >> 2;
-    const float4* xr = reinterpret_cast<const float4*>(X + (size_t)row * K);
+    const void* xr = row_ptr<BF16IN>(X, (size_t)row, K);
     // whether this thread's vector i lies inside the row: known at compile time for all but the last when EXACT
     const bool last_ok = (V - 1) * TPR + t < nv;
     auto inside = [&](int i) { return (EXACT && i < V - 1) ? true : (EXACT ? last_ok : i * TPR + t < nv); };
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         const int idx = i * TPR + t;
-        v[i] = inside(i) ? __ldg(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[i] = inside(i) ? load_row4<BF16IN>(xr, idx) : make_float4(0.f, 0.f, 0.f, 0.f);
         if (GLU && inside(i)) {
             const float4 u = __ldg(reinterpret_cast<const float4*>(U + (size_t)row * K) + idx);
             auto f = [](float gg, float uu) { float r = gg > 0.f ? gg : 0.f; return uu * (r * r); };
@@ -314,8 +314,8 @@ __global__ void __launch_bounds__(kBlock, V <= 4 ? 5 : 4)
         kr = sl[1];
     }
     if (mode == 2u) {
-        cold_row<TPR, GLU>(X + (size_t)row * K, GLU ? U + (size_t)row * K : nullptr, K, k, mult, codes + (size_t)row * K, h1,
-                           sl, red, group, t);
+        cold_row<TPR, GLU, BF16IN>(reinterpret_cast<const float*>(xr), GLU ? U + (size_t)row * K : nullptr, K, k, mult,
+                                   codes + (size_t)row * K, h1, sl, red, group, t);
         return;
     }
 
@@ -443,18 +443,18 @@ __global__ void __launch_bounds__(kBlock)
     if (t == 0) scale[row] = (float)(gamma / 127.0);
 }
 
-template <int TPR, int V, bool GLU, bool EXACT>
+template <int TPR, int V, bool GLU, bool EXACT, bool BF16IN>
 void launch_one(const float* X, const float* U, int M, int K, int k, double e, int8_t* codes, float* scale, cudaStream_t st) {
     constexpr int G = kBlock / TPR;
-    a48_launch_pdl(topk_quant_int8_kernel<TPR, V, GLU, EXACT>, dim3((M + G - 1) / G), dim3(kBlock), 0, st, X, U, M, K, k, e, codes,
+    a48_launch_pdl(topk_quant_int8_kernel<TPR, V, GLU, EXACT, BF16IN>, dim3((M + G - 1) / G), dim3(kBlock), 0, st, X, U, M, K, k, e, codes,
                    scale);
 }
 
-template <bool GLU>
+template <bool GLU, bool BF16IN = false>
 bitnet_a48_status launch_topk(const float* X, const float* U, int M, int K, int k, double e, int8_t* codes, float* scale,
                               cudaStream_t st) {
     const int nv = K / 4;
-#define A48_TK(TPR, V, EXACT) launch_one<TPR, V, GLU, EXACT>(X, U, M, K, k, e, codes, scale, st)
+#define A48_TK(TPR, V, EXACT) launch_one<TPR, V, GLU, EXACT, BF16IN>(X, U, M, K, k, e, codes, scale, st)
     if (nv <= 32 * 4) A48_TK(32, 4, false);
     else if (nv <= 64 * 4) A48_TK(64, 4, false);
     else if (nv <= 128 * 4) A48_TK(128, 4, false);
@@ -493,6 +493,12 @@ bitnet_a48_status a48_launch_topk_quant_int8(const float* X, int M, int K, int k
     topk_quant_int8_generic_kernel<<<M, kBlock, 0, st>>>(X, M, K, k, (double)eps, codes, scale, mask_bits);
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_launch_topk_quant_int8_bf16(const uint16_t* X, int M, int K, int k, float eps, int8_t* codes,
+                                                  float* scale, cudaStream_t st) {
+    if (!a48_topk_quant_fast_shape(K)) return BITNET_A48_ERR_UNSUPPORTED;  // the register kernels only
+    return launch_topk<false, true>(reinterpret_cast<const float*>(X), nullptr, M, K, k, (double)eps, codes, scale, st);
 }
 
 // Top-K + INT8 of up * ReLU(gate)^2 (Eq. 5 fused into the quantiser's load); shapes of the register kernels only.
