@@ -55,7 +55,7 @@ NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part (2 x the 2.25 P
 SHAPE_3B = dict(H=3200, F=8640, NH=32, LAYERS=26)
 SHAPE_700M = dict(H=1536, F=4096, NH=16, LAYERS=24)  # 16 heads as the benchmark configuration fixes (head dim 96)
 SHAPE_7B = dict(H=H, F=F, NH=NH, LAYERS=LAYERS)
-ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "gatefirst", "cpu")
+ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "gatefirst", "formats", "cpu")
 
 
 def proj_list(Hs, Fs):
@@ -479,6 +479,10 @@ def run_ours(args):
     if "block" in legs:
         block = bench_block(a48, synth, dev, stream, layer)
     gate_first = bench_gate_first(a48, synth, dev, stream) if "gatefirst" in legs else None
+    formats = None
+    if "formats" in legs:
+        formats = bench_formats(a48, synth, dev, stream, peaks, layer)
+        rooflines.extend(formats.pop("rooflines"))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and "cpu" in legs:
@@ -506,7 +510,7 @@ def run_ours(args):
                             "window": f"first {n_burst} passes of the timed region"},
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "rooflines": rooflines, "e2e": e2e,
             "cpu_baseline": cpu_baseline, "decode": decode, "decode_3b": decode3b, "prefill_700m": prefill700m,
-            "sweep": sweep, "block": block, "ffn_gate_first": gate_first,
+            "sweep": sweep, "block": block, "ffn_gate_first": gate_first, "formats": formats,
         }
         print(json.dumps(line))
     reps.close()
@@ -752,6 +756,92 @@ def bench_sweep(a48, synth, dev, stream, copies=12, reps=5):
     return {"points": points,
             "note": "bitnet_a48_linear alone (codes resident), time per call; dense_tops = 2*M*N*K / time, weight_gbs = "
                     "packed weight bytes / time"}
+
+
+def time_ms(fn, stream, reps, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def bench_formats(a48, synth, dev, stream, peaks, layer):
+    """The other number formats of the library on the 7B shape: FP4 quantiser (Eq. 8-9), bf16 activations at the
+    boundary, and the five-codes-per-byte weight layout in a decode chain."""
+    M = M_PREFILL
+    out, roof = {}, []
+
+    def hbm(kernel, ms, bytes_):
+        gbs = bytes_ / (ms * 1e-3) / 1e9
+        return {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "traffic": None, "avg_launch_ms": ms,
+                "algorithmic_bytes_per_launch": bytes_, "peak_source": f"hbm_gbs of {peaks['source']} peaks"}
+
+    x = synth.gaussian_outlier_activations(M, H, seed=45, device=dev)
+    codes = torch.empty(M, H, dtype=torch.int8, device=dev)
+    scale = torch.empty(M, dtype=torch.float32, device=dev)
+    ms = time_ms(lambda: a48.quant_fp4(x, codes, scale), stream, 50)
+    roof.append(hbm("FP4 (E2M1) quantiser, 16384 x 4096 (Eq. 8-9)", ms, 5.0 * M * H + 4.0 * M))
+    # bf16 in, bf16 out: INT4 quantiser and the gate projection
+    xb = x.to(torch.bfloat16)
+    ms = time_ms(lambda: a48.quant_int4_bf16(xb, EPS, codes, scale), stream, 50)
+    roof.append(hbm("INT4 quantiser from bf16 rows, 16384 x 4096 (Eq. 7)", ms, 3.0 * M * H + 4.0 * M))
+    sb = synth.student_t3(M, F, seed=46, device=dev).to(torch.bfloat16)
+    codes_f = torch.empty(M, F, dtype=torch.int8, device=dev)
+    ms = time_ms(lambda: a48.topk_quant_int8_bf16(sb, F // 2, EPS, codes_f, scale), stream, 20)
+    roof.append(hbm("top-K + INT8 quantiser from bf16 rows, 16384 x 11008 (Eq. 1, 3)", ms, 3.0 * M * F + 4.0 * M))
+    del sb, codes_f
+    a48.quant_int4(x, EPS, codes, scale)
+    y32 = torch.empty(M, F, dtype=torch.float32, device=dev)
+    y16 = torch.empty(M, F, dtype=torch.bfloat16, device=dev)
+    ops = 2.0 * M * F * H
+    ms32 = time_ms(lambda: a48.linear(layer.w["gate"], codes, scale, a48.ACT_INT4, Y=y32), stream, 100)
+    ms16 = time_ms(lambda: a48.linear_bf16(layer.w["gate"], codes, scale, a48.ACT_INT4, Y=y16), stream, 100)
+    out["gate_projection_16384_tokens"] = {"fp32_out_ms": ms32, "fp32_out_tops": ops / ms32 / 1e9, "bf16_out_ms": ms16,
+                                           "bf16_out_tops": ops / ms16 / 1e9,
+                                           "note": "bitnet_a48_linear against bitnet_a48_linear_bf16, 100 calls each"}
+    del y32, y16, x, xb
+    torch.cuda.empty_cache()
+    # five codes per byte: the seven matrices of 16 distinct layers in one CUDA graph (0.65 GB >> L2), 1 and 8 tokens
+    layers = 16
+    ws5, ws2 = [], []
+    for li in range(layers):
+        for i, (name, n, k, kind) in enumerate(PROJ):
+            lat = synth.ternary_latents(n, k, seed=5000 + li * 8 + i, device=dev)
+            w = a48.pack_ternary(lat, EPS, a48.LAYOUT_TRIT5 | a48.LAYOUT_DECODE)
+            ws5.append((w, n, k, kind))
+            del lat
+    b5 = sum(w.layout_bytes(a48.LAYOUT_TRIT5) for w, *_ in ws5)
+    b2 = sum(w.packed_bytes for w, *_ in ws5)
+    out["trit5"] = {"bytes_five_per_byte": b5, "bytes_two_bit": b2, "ratio": b5 / b2, "layers": layers}
+    for Mt in (1, 8):
+        c4, d4 = a48.quant_int4(synth.gaussian_outlier_activations(Mt, H, seed=50, device=dev), EPS)
+        c8h, d8h, _ = a48.topk_quant_int8(synth.student_t3(Mt, H, seed=51, device=dev), H // 2, EPS)
+        c8f, d8f, _ = a48.topk_quant_int8(synth.student_t3(Mt, F, seed=52, device=dev), F // 2, EPS)
+        yh = torch.empty(Mt, H, dtype=torch.float32, device=dev)
+        yf = torch.empty(Mt, F, dtype=torch.float32, device=dev)
+        wsp = torch.zeros(max(a48.linear_workspace_bytes(w, Mt) for w, *_ in ws5[:7]), dtype=torch.uint8, device=dev)
+
+        def chain(algo, st=None):
+            for w, n, k, kind in ws5:
+                c, d, act = (c4, d4, a48.ACT_INT4) if kind == "int4" else ((c8h, d8h, a48.ACT_TOPK_INT8) if k == H else (c8f, d8f, a48.ACT_TOPK_INT8))
+                a48.linear(w, c, d, act, algo, Y=yf if n == F else yh, workspace=wsp, stream=st)
+
+        ms5 = graph_time_ms(lambda st=None: chain(a48.ALGO_DECODE_TRIT5, st), stream, reps=10)
+        ms2 = graph_time_ms(lambda st=None: chain(a48.ALGO_DECODE, st), stream, reps=10)
+        out["trit5"][f"tokens_{Mt}"] = {"five_per_byte_ms": ms5, "five_per_byte_gbs": b5 / ms5 / 1e6, "two_bit_ms": ms2,
+                                        "two_bit_gbs": b2 / ms2 / 1e6,
+                                        "note": "one launch per matrix in both chains (no fused q/k/v, gate/up launches)"}
+    for w, *_ in ws5:
+        w.free()
+    out["rooflines"] = roof
+    return out
 
 
 def bench_gate_first(a48, synth, dev, stream, layers=16):

@@ -5,15 +5,20 @@
 // Base-3 digits do not come apart with shifts and masks, so a byte is decoded through a 243-entry table in shared
 // memory (two words per entry: the int8 codes t_0..t_3, and t_4), and the token codes are staged once per CTA in
 // the matching groups of five (two words per group: x_0..x_3, and x_4).  Each table lookup then feeds two dp4a.
+// The lanes of a warp look up unrelated bytes, so the table is kept in 16 copies, lane l reading copy l % 16: an
+// entry's copies fill one 128-byte line, every lane pair has banks of its own, and no lookup waits for another.
 // One warp owns a row at a time and streams it with 16-byte loads.  This trades arithmetic for bytes: a fifth
 // fewer bytes from HBM, about twice the instructions per weight of the 2-bit kernels.
 #include "internal.h"
 
 namespace {
 
-constexpr int kThreads = 256, kWarps = kThreads / 32;
+constexpr int kThreads = 512, kWarps = kThreads / 32;  // one CTA per SM: staging the codes and the table is paid once
 
-// Dynamic shared memory: xg [MT][groups] uint2 | lut [243] uint2.
+constexpr int kLutCopies = 16;
+constexpr int kMaxPieces = 5;  // 16-byte pieces of a row per lane: rows of up to 5 * 32 * 16 * 5 = 12800 channels
+
+// Dynamic shared memory: xg [MT][groups] uint2 | lut [243][kLutCopies] uint2.
 template <int MT>
 __global__ void __launch_bounds__(kThreads) decode_trit5_kernel(const uint8_t* __restrict__ wt, int row_bytes, const int8_t* __restrict__ codes,
                                                                 const float* __restrict__ scale, const float* __restrict__ alpha,
@@ -24,49 +29,74 @@ __global__ void __launch_bounds__(kThreads) decode_trit5_kernel(const uint8_t* _
     uint2* xg = reinterpret_cast<uint2*>(smem);
     uint2* lut = xg + (size_t)MT * groups;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int b = threadIdx.x; b < 243; b += kThreads) {
+    for (int i = threadIdx.x; i < 243 * kLutCopies; i += kThreads) {
+        const int b = i / kLutCopies;
         int d[5], v = b;
 #pragma unroll
         for (int i = 0; i < 5; ++i) {
             d[i] = v % 3 - 1;
             v /= 3;
         }
-        lut[b] = make_uint2((uint32_t)(d[0] & 0xff) | ((uint32_t)(d[1] & 0xff) << 8) | ((uint32_t)(d[2] & 0xff) << 16) |
+        lut[i] = make_uint2((uint32_t)(d[0] & 0xff) | ((uint32_t)(d[1] & 0xff) << 8) | ((uint32_t)(d[2] & 0xff) << 16) |
                                 ((uint32_t)(d[3] & 0xff) << 24),
                             (uint32_t)(d[4] & 0xff));
     }
-    for (int i = threadIdx.x; i < MT * groups; i += kThreads) {
-        const int m = i / groups, g = i % groups;
-        uint32_t lo = 0, hi = 0;
-        if (m < M) {
+    // the token codes, 16 at a time, scattered to their groups of five (byte j of a group's two words is code 5g + j;
+    // group g = 16 p + s is the s-th byte of the 16-byte piece p that lane p % 32 loads: stored [m][s][p], so that the
+    // 32 lanes of a warp, which hold consecutive pieces, read consecutive words)
+    for (int i = threadIdx.x; i < MT * groups; i += kThreads) xg[i] = make_uint2(0u, 0u);
+    __syncthreads();
+    {
+        uint8_t* xb = reinterpret_cast<uint8_t*>(xg);
+        const int chunks = (K + 15) / 16;
+        for (int i = threadIdx.x; i < M * chunks; i += kThreads) {
+            const int m = i / chunks, k0 = 16 * (i % chunks);
+            __align__(16) uint8_t c[16];
+            if (k0 + 16 <= K && (K & 15) == 0) {
+                *reinterpret_cast<uint4*>(c) = __ldg(reinterpret_cast<const uint4*>(codes + (size_t)m * K + k0));
+            } else {
 #pragma unroll
-            for (int j = 0; j < 5; ++j) {
-                const int k = 5 * g + j;
-                const uint32_t c = k < K ? (uint32_t)(uint8_t)codes[(size_t)m * K + k] : 0u;
-                if (j < 4) lo |= c << (8 * j);
-                else hi = c;
+                for (int q = 0; q < 16; ++q) c[q] = k0 + q < K ? (uint8_t)codes[(size_t)m * K + k0 + q] : (uint8_t)0;
+            }
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int k = k0 + q, g = k / 5, j = k - 5 * g;
+                if (k < K) xb[(((size_t)m * 16 + (g & 15)) * (groups / 16) + (g >> 4)) * 8 + j] = c[q];
             }
         }
-        // group g = 16 p + s is the s-th byte of the 16-byte piece p that lane p % 32 loads: stored [m][s][p], so that
-        // the 32 lanes of a warp, which hold consecutive pieces, read consecutive words
-        xg[((size_t)m * 16 + (g & 15)) * (groups / 16) + (g >> 4)] = make_uint2(lo, hi);
     }
     __syncthreads();
     const float al = __ldg(alpha);
     const int pieces = row_bytes / 16;
-    for (int n = blockIdx.x * kWarps + warp; n < N; n += gridDim.x * kWarps) {
+    // A warp's rows are walked with the next row's pieces already requested (up to kMaxPieces 16-byte pieces per lane,
+    // i.e. rows of up to 12800 channels), so that a lane always has a row's worth of loads in flight.
+    const int stride = gridDim.x * kWarps;
+    uint4 cur[kMaxPieces], nxt[kMaxPieces];
+    auto fetch = [&](int n, uint4 (&dst)[kMaxPieces]) {
+        const uint4* row = reinterpret_cast<const uint4*>(wt + (size_t)n * row_bytes);
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i) {
+            const int p = lane + 32 * i;
+            dst[i] = (n < N && p < pieces) ? __ldg(row + p) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    int n = blockIdx.x * kWarps + warp;
+    fetch(n, cur);
+    for (; n < N; n += stride) {
+        fetch(n + stride, nxt);
         int acc[MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m) acc[m] = 0;
-        const uint4* row = reinterpret_cast<const uint4*>(wt + (size_t)n * row_bytes);
-        for (int p = lane; p < pieces; p += 32) {
-            const uint4 w4 = __ldg(row + p);
-            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i) {
+            const int p = lane + 32 * i;
+            if (p >= pieces) break;
+            const uint32_t w[4] = {cur[i].x, cur[i].y, cur[i].z, cur[i].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    const uint2 t = lut[(w[j] >> (8 * b)) & 0xffu];
+                    const uint2 t = lut[((w[j] >> (8 * b)) & 0xffu) * kLutCopies + (lane & (kLutCopies - 1))];
 #pragma unroll
                     for (int m = 0; m < MT; ++m) {
                         const uint2 x = xg[((size_t)m * 16 + 4 * j + b) * pieces + p];
@@ -75,6 +105,8 @@ __global__ void __launch_bounds__(kThreads) decode_trit5_kernel(const uint8_t* _
                 }
             }
         }
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i) cur[i] = nxt[i];
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
             int v = acc[m];
@@ -91,18 +123,18 @@ __global__ void __launch_bounds__(kThreads) decode_trit5_kernel(const uint8_t* _
 }  // namespace
 
 bool a48_decode_trit5_supported(const bitnet_a48_weight* w, int M) {
-    return w->trit5 != nullptr && M >= 1 && M <= 8 && (size_t)8 * w->trit5_row * 8 + 243 * 8 <= 200 * 1024;
+    return w->trit5 != nullptr && M >= 1 && M <= 8 && w->trit5_row <= kMaxPieces * 32 * 16 && (size_t)8 * w->trit5_row * 8 + 243 * 8 * kLutCopies <= 200 * 1024;
 }
 
 bitnet_a48_status a48_launch_decode_trit5(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
                                           int32_t* acc, cudaStream_t st) {
     if (!a48_decode_trit5_supported(w, M)) return BITNET_A48_ERR_UNSUPPORTED;
     const int mt = M == 1 ? 1 : (M == 2 ? 2 : (M <= 4 ? 4 : 8));
-    const size_t smem = (size_t)mt * w->trit5_row * 8 + 243 * 8;
+    const size_t smem = (size_t)mt * w->trit5_row * 8 + 243 * 8 * kLutCopies;
     int dev = 0, sms = 0;
     A48_CUDA_TRY(cudaGetDevice(&dev));
     A48_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    int grid = sms * 4;
+    int grid = sms;
     if (grid * kWarps > w->N) grid = (w->N + kWarps - 1) / kWarps;
 #define A48_T5(MT)                                                                                                          \
     do {                                                                                                                     \
