@@ -4,6 +4,7 @@
 #include "internal.h"
 
 thread_local int a48_y_bf16 = 0;
+thread_local const float* a48_decode_residual = nullptr;
 
 namespace {
 

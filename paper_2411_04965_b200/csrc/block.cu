@@ -551,8 +551,16 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         relu2glu_kernel<<<(unsigned)((nF4 + 255) / 256), 256, 0, st>>>(gate, up, nF4);
         A48_TRY(a48_launch_topk_quant_int8(gate, M, F, c.k_down, c.quant_eps, codes, scale, nullptr, st));
     }
-    A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));
-    A48_CUDA_TRY(a48_launch_pdl(add_kernel, dim3((unsigned)((nH4 + 255) / 256)), dim3(256), 0, st, hres, tmp, Y, nH4));
+    if (a48_decode_supported(blk->w[6], M)) {
+        // a few tokens: the last residual add rides in the decode kernel's epilogue (one launch fewer)
+        a48_decode_residual = hres;
+        s = linear(6, BITNET_A48_ACT_TOPK_INT8, Y);
+        a48_decode_residual = nullptr;
+        if (s != BITNET_A48_OK) return s;
+    } else {
+        A48_TRY(linear(6, BITNET_A48_ACT_TOPK_INT8, tmp));
+        A48_CUDA_TRY(a48_launch_pdl(add_kernel, dim3((unsigned)((nH4 + 255) / 256)), dim3(256), 0, st, hres, tmp, Y, nH4));
+    }
 #undef A48_TRY
     A48_CUDA_TRY(cudaGetLastError());
     return BITNET_A48_OK;

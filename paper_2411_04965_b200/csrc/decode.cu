@@ -136,6 +136,7 @@ struct DecodeParams {
     int piece_q, piece_r; // the first piece_r pieces hold piece_q + 1 items (tiles if tile_aligned, else units), the rest piece_q
     int act_row_bytes;    // padded K + 16
     int y_bf16;           // outputs are bf16 instead of fp32
+    const float* residual;  // fp32 [M, N_0] added to the outputs of matrix 0, or nullptr
 };
 
 __device__ __forceinline__ int matrix_of(const DecodeParams& p, int tile) {
@@ -493,7 +494,9 @@ __global__ void __launch_bounds__(32 * NW, ONE_TOKEN ? 2 : 1) decode_kernel(cons
         if (n < p.N[j]) {
             const int v = (int)sum - csum[m];
             const size_t o = (size_t)m * p.N[j] + (size_t)n;
-            a48_store_y(p.Y[j], o, (float)v * (p.scale[m] * __ldg(p.alpha[j])), p.y_bf16);  // prefactors of Eq. 2, 3 and 7
+            float y = (float)v * (p.scale[m] * __ldg(p.alpha[j]));  // prefactors of Eq. 2, 3 and 7
+            if (p.residual) y += p.residual[o];
+            a48_store_y(p.Y[j], o, y, p.y_bf16);
             if (p.acc[j]) p.acc[j][o] = v;
         }
     }
@@ -570,6 +573,7 @@ bitnet_a48_status a48_launch_decode_multi(int count, const bitnet_a48_weight* co
     p.units = (int)(ntiles * p.kchunks);
     p.act_row_bytes = w->Kp + 16;
     p.y_bf16 = a48_y_bf16;
+    p.residual = count == 1 ? a48_decode_residual : nullptr;
     // one piece per SM unless a piece would then not fit: at most MAX_SHARE units and MAX_TILES tiles per piece
     long long grid = sm_count();
     if (grid > p.units) grid = p.units;

@@ -42,6 +42,10 @@ static inline cudaError_t a48_launch_pdl(void (*kernel)(KArgs...), dim3 grid, di
 // (round to nearest even of the fp32 result).  Set by bitnet_a48_linear_bf16 around its dispatch, read by the
 // launchers, which pass it to their kernels as a parameter.
 extern thread_local int a48_y_bf16;
+// A residual to add in the decode kernel's epilogue for the call in flight on this host thread (fp32 [M, N], or
+// nullptr): Y = R + fp32(acc)*(scale*alpha), the sum a separate elementwise kernel would form.  Set by the block's
+// decode step around its last BitLinear; honoured by the single-matrix decode launch only.
+extern thread_local const float* a48_decode_residual;
 #ifdef __CUDACC__
 #include <cuda_bf16.h>
 // Stores y as element `index` of an fp32 or a bf16 array.
