@@ -172,6 +172,12 @@ bool a48_decode_trit5_supported(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_decode_trit5(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
                                           int32_t* acc, cudaStream_t st);
 
+// ---- attn_mma.cu (prefill attention on the tensor cores, split-bf16 operands)
+bool a48_attn_mma_supported(int hd);
+size_t a48_attn_mma_workspace_bytes(int B, int nh, int hd, int T, int n_keys);
+bitnet_a48_status a48_launch_attn_mma(const float* q, const float* kcache, const float* vcache, int B, int T, int nh, int hd,
+                                      int pos0, int cap, float* out, void* ws, cudaStream_t st);
+
 // ---- block.cu
 size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
 bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X, int B, int T, int pos0,
