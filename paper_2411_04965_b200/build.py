@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbitnet_a48.so")
-SOURCES = ["api.cu", "pack.cu", "quant.cu", "quant_topk.cu", "linear_simple.cu", "gemm_tcgen05.cu", "decode.cu", "decode_sparse.cu", "block.cu", "ffn_gate_first.cu", "attn_lowbit.cu", "decode_trit5.cu", "attn_mma.cu"]
+SOURCES = ["api.cu", "pack.cu", "quant.cu", "quant_topk.cu", "linear_simple.cu", "gemm_tcgen05.cu", "decode.cu", "decode_sparse.cu", "block.cu", "ffn_gate_first.cu", "attn_lowbit.cu", "decode_trit5.cu", "attn_tcgen05.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

@@ -1,0 +1,578 @@
+// Causal softmax attention for prefill on the fifth-generation tensor cores (the block glue around the BitLinears,
+// Section 2.1).
+//
+// Attention is two contractions per head, S = Q K^T and O = P V.  The block's tolerance against the float64 oracle
+// does not allow plain bf16 or tf32 operands: a score that is 1e-3 off moves its probability by as much, and the
+// quantisers that follow the attention turn a 1e-5 difference into flipped codes.  So every operand is split into
+// three bf16 numbers, x = x0 + x1 + x2 with x0 = bf16(x), x1 = bf16(x - x0), x2 = bf16(x - x0 - x1) (the subtractions
+// are exact, the three carry the 24 significant bits of x), and every product is the six MMAs x_i * y_j with
+// i + j <= 2.  What is dropped is below 2^-24 of a product.  The tensor core adds to its accumulator with less care
+// than an fp32 add (measured with mma.sync: truncation), so the leading products (part 0 times part 0) and the five
+// correction products (2^-8 and less of the leading ones) go to accumulators of their own, and the running output
+// lives in registers: every key tile is contracted into a fresh accumulator and added in fp32.
+//
+// Kernels.  attn_split_kernel writes the parts of the queries of the call and of the keys of positions
+// [0, pos0 + T) as bf16 arrays [part][B * heads][rows padded to a tile][head dim padded to 64 or 128];
+// attn_split_vt_kernel writes the parts of the values transposed, [part][B * heads][head dim][keys], so that both
+// operands of both contractions are K-major.  attn_tc_kernel: one CTA per (128 queries, head, sequence), 1 per SM.
+//   warp 8, one lane: tensor copies (TMA, 128-byte swizzle) of the query parts once and of one key tile (64 keys) and
+//     one value tile at a time, and all tcgen05.mma: S(t) = Q K(t)^T with both operands in shared memory, O(t) =
+//     P(t) V(t) with P in tensor memory.  Keys and values have one buffer each: K(t+1) is requested when S(t) has
+//     completed, V(t+1) when O(t) has, and S(t+1) is issued right behind O(t), so the copies and the softmax of
+//     the next tile overlap the MMAs of this one.
+//   warps 0-7: two threads per query row (tensor-memory lane), each with half of the tile's keys and half of the head
+//     dimension: read S, exchange the row maximum through shared memory, exponentials, split P into parts, store them
+//     to tensor memory, rescale the running output, then add O(t).
+// Every wait is bounded; a wait that gives up records itself (bitnet_a48_kernel_status) and lets every later wait of
+// the CTA fall through, so the kernel ends by itself; the issuer then waits for its copies in flight before it leaves.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace {
+
+constexpr int TQ = 128;  // queries per CTA = MMA M = tensor-memory lanes
+constexpr int TK = 64;   // keys per tile: one 128-byte swizzle row of bf16
+constexpr int NS = 3;    // parts per operand
+constexpr int SOFTMAX_WARPS = 8, THREADS = 32 * (SOFTMAX_WARPS + 1);
+constexpr int TMEM_COLS = 512;
+// tensor-memory columns: S leading | S corrections | O(t) leading | O(t) corrections | P parts (two keys per column)
+constexpr int COL_S = 0, COL_SC = 64, COL_O = 128, COL_OC = 256, COL_P = 384;
+constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
+constexpr unsigned long long kDrainClocks = 400000000ull;  // what the issuer grants its copies in flight when it gives up
+
+__device__ unsigned int g_attn_status[4];
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Once any wait of the CTA has given up (*abort_flag), every wait returns at once.
+__device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id, uint32_t iter,
+                                            unsigned long long limit) {
+    const unsigned long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag && limit == kWaitClocks) return;
+            if (clock64() - t0 > limit) {
+                *abort_flag = 1;
+                if (atomicCAS(&g_attn_status[0], 0u, (unsigned)BITNET_A48_ERR_TIMEOUT) == 0u) {
+                    g_attn_status[1] = id;
+                    g_attn_status[2] = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+                    g_attn_status[3] = iter;
+                }
+                return;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t id, uint32_t iter) {
+    if (mbar_try(bar, parity)) return;
+    if (*abort_flag) return;
+    mbar_wait_slow(bar, parity, abort_flag, id, iter, kWaitClocks);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 operands, fp32 accumulators
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Shared-memory matrix descriptor of a K-major operand tile whose rows are 128 bytes (64 bf16), laid down by TMA with
+// the 128-byte swizzle: 8-row groups are 1024 bytes apart.  16 elements further along K = +32 bytes = +2 in the
+// address field.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void softmax_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * SOFTMAX_WARPS) : "memory"); }
+
+// a pair of floats: the bf16x2 word of their leading parts (first value in the low half); x and y keep the rest
+__device__ __forceinline__ uint32_t take_part(float& x, float& y) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(&h);
+    x -= __uint_as_float(w << 16);
+    y -= __uint_as_float(w & 0xffff0000u);
+    return w;
+}
+// 2^x, two units in the last place at most; 2^-inf = 0
+__device__ __forceinline__ float exp2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// src rows of hd floats -> NS parts (part_stride elements apart) of rows of hdp bf16, zero past hd and for rows >=
+// rows_valid.  mode 0: queries, src = q [B*T][nh*hd], row (b, h, r) = token r of sequence b; mode 1: cache
+// [B][nh][cap][hd].
+__global__ void __launch_bounds__(256) attn_split_kernel(const float* __restrict__ src, int mode, int B, int nh, int hd, int hdp,
+                                                         int rows_valid, int rows_pad, int T, int cap,
+                                                         __nv_bfloat16* __restrict__ parts, size_t part_stride) {
+    a48_pdl_prologue();
+    const int pairs = hdp / 2;
+    const size_t total = (size_t)B * nh * rows_pad * pairs;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % pairs) * 2;
+        const size_t row = i / pairs;
+        const int r = (int)(row % rows_pad);
+        const size_t bh = row / rows_pad;
+        const int h = (int)(bh % nh), b = (int)(bh / nh);
+        float x = 0.f, y = 0.f;
+        if (r < rows_valid && c < hd) {
+            const float* p = mode == 0 ? src + ((size_t)b * T + r) * ((size_t)nh * hd) + (size_t)h * hd + c
+                                       : src + (((size_t)b * nh + h) * cap + r) * hd + c;
+            x = p[0];
+            y = c + 1 < hd ? p[1] : 0.f;
+        }
+#pragma unroll
+        for (int a = 0; a < NS; ++a) reinterpret_cast<uint32_t*>(parts + a * part_stride)[i] = take_part(x, y);
+    }
+}
+
+// The values of one head and 64 positions, transposed: vcache [B*nh][cap][hd] -> parts [part][B*nh][hdp][k_pad].
+// grid (k_pad / 64, B * nh); dynamic shared memory 64 * (hdp + 1) floats.
+__global__ void __launch_bounds__(256) attn_split_vt_kernel(const float* __restrict__ vcache, int hd, int hdp, int n_keys, int k_pad,
+                                                            int cap, __nv_bfloat16* __restrict__ parts, size_t part_stride) {
+    extern __shared__ float vt_tile[];  // [64 keys][hdp + 1]
+    a48_pdl_prologue();
+    const int k0 = blockIdx.x * TK, ld = hdp + 1;
+    const size_t bh = blockIdx.y;
+    for (int i = threadIdx.x; i < TK * hdp; i += blockDim.x) {
+        const int key = i / hdp, d = i - key * hdp;
+        vt_tile[key * ld + d] = (k0 + key < n_keys && d < hd) ? vcache[(bh * cap + k0 + key) * hd + d] : 0.f;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < hdp * (TK / 2); i += blockDim.x) {
+        const int d = i / (TK / 2), kp = i - d * (TK / 2);
+        float x = vt_tile[(2 * kp) * ld + d], y = vt_tile[(2 * kp + 1) * ld + d];
+        const size_t o = ((bh * hdp + d) * (size_t)k_pad + k0) / 2 + kp;
+#pragma unroll
+        for (int a = 0; a < NS; ++a) reinterpret_cast<uint32_t*>(parts + a * part_stride)[o] = take_part(x, y);
+    }
+}
+
+struct AttnParams {
+    int T, t_pad, n_keys, k_pad, nh, hd, pos0, bh_total;
+    float scale;
+    float* out;
+};
+
+template <int HDP>
+struct AttnCfg {
+    static constexpr int KB = HDP / 64;                     // 128-byte blocks per operand row of the first contraction
+    static constexpr int Q_BLOCK = TQ * 128, K_BLOCK = TK * 128, V_PART = HDP * 128;
+    static constexpr int Q_BYTES = NS * KB * Q_BLOCK, K_BYTES = NS * KB * K_BLOCK, V_BYTES = NS * V_PART;
+    static constexpr int SMEM_BYTES = Q_BYTES + K_BYTES + V_BYTES + 1024 /*alignment slack*/ + 4096 /*barriers, row maxima*/;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(COL_O + HDP <= COL_OC && COL_OC + HDP <= COL_P && COL_P + NS * TK / 2 <= TMEM_COLS, "tensor memory budget");
+};
+
+// barrier ids reported through the status words
+enum { WAIT_Q = 20, WAIT_K = 21, WAIT_V = 22, WAIT_S = 23, WAIT_O = 24, WAIT_P = 25, WAIT_DRAIN = 26 };
+
+template <int HDP>
+__global__ void __launch_bounds__(THREADS, 1)
+    attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    using C = AttnCfg<HDP>;
+    constexpr int KB = C::KB, OD = HDP / 2;  // OD: head dims per softmax thread
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* ctrl = smem + C::Q_BYTES + C::K_BYTES + C::V_BYTES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 64);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 68);
+    float* row_max = reinterpret_cast<float*>(ctrl + 1024);  // [tile parity][half][row]
+    const uint32_t sq = smem_u32(smem), sk = sq + C::Q_BYTES, sv = sk + C::K_BYTES;
+    const uint32_t bar_q = smem_u32(ctrl), bar_k = bar_q + 8, bar_v = bar_q + 16, bar_s = bar_q + 24, bar_o = bar_q + 32,
+                   bar_p = bar_q + 40;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar_q, 1);
+        mbar_init(bar_k, 1);
+        mbar_init(bar_v, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        mbar_init(bar_p, 32 * SOFTMAX_WARPS);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == SOFTMAX_WARPS) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    a48_pdl_prologue();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * TQ;  // the tiles with the most keys first
+    const int h = blockIdx.y, b = blockIdx.z, bh = b * p.nh + h;
+    const int keys_needed = min(p.n_keys, p.pos0 + min(q0 + TQ, p.T));  // causal: nothing beyond the last query's position
+    const int n_tiles = (keys_needed + TK - 1) / TK;
+
+    if (warp == SOFTMAX_WARPS) {
+        if (lane == 0) {
+            // ------------------------------------------------------------- copies and MMAs
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+            int k_issued = 0, v_issued = 0;
+            auto load_k = [&](int t) {
+                mbar_expect_tx(bar_k, C::K_BYTES);
+#pragma unroll
+                for (int a = 0; a < NS; ++a)
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb)
+                        tma_load_2d(sk + (a * KB + kb) * C::K_BLOCK, &tm_k, kb * 64, (a * p.bh_total + bh) * p.k_pad + t * TK, bar_k);
+                ++k_issued;
+            };
+            auto load_v = [&](int t) {
+                mbar_expect_tx(bar_v, C::V_BYTES);
+#pragma unroll
+                for (int a = 0; a < NS; ++a) tma_load_2d(sv + a * C::V_PART, &tm_v, t * TK, (a * p.bh_total + bh) * HDP, bar_v);
+                ++v_issued;
+            };
+            mbar_expect_tx(bar_q, C::Q_BYTES);
+#pragma unroll
+            for (int a = 0; a < NS; ++a)
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+                    tma_load_2d(sq + (a * KB + kb) * C::Q_BLOCK, &tm_q, kb * 64, (a * p.bh_total + bh) * p.t_pad + q0, bar_q);
+            load_k(0);
+            load_v(0);
+            constexpr uint32_t idesc_s = idesc_bf16(TQ, TK), idesc_o = idesc_bf16(TQ, HDP);
+            const uint32_t t_s = tmem_base + COL_S, t_sc = tmem_base + COL_SC, t_o = tmem_base + COL_O, t_oc = tmem_base + COL_OC,
+                           t_p = tmem_base + COL_P;
+            // the correction products, smallest first: (part of A, part of B)
+            constexpr int CA[5] = {0, 1, 2, 0, 1}, CB[5] = {2, 1, 0, 1, 0};
+            mbar_wait(bar_q, 0, abort_flag, WAIT_Q, 0);
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t par = t & 1;
+                mbar_wait(bar_k, par, abort_flag, WAIT_K, t);
+                tc_fence_after();
+                // ---- S(t) = Q K(t)^T: HDP / 16 steps of six MMAs
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint64_t qd[NS], kd[NS];
+#pragma unroll
+                        for (int a = 0; a < NS; ++a) {
+                            qd[a] = smem_desc_sw128(sq + (a * KB + kb) * C::Q_BLOCK) + 2 * j;
+                            kd[a] = smem_desc_sw128(sk + (a * KB + kb) * C::K_BLOCK) + 2 * j;
+                        }
+                        mma_ss(t_s, qd[0], kd[0], idesc_s, (kb | j) != 0);
+#pragma unroll
+                        for (int c = 0; c < 5; ++c) mma_ss(t_sc, qd[CA[c]], kd[CB[c]], idesc_s, (kb | j | c) != 0);
+                    }
+                tc_commit(bar_s);
+                if (t > 0) {  // O(t-1) has read the value tile: request the next one
+                    mbar_wait(bar_o, par ^ 1, abort_flag, WAIT_O, t);
+                    load_v(t);
+                }
+                mbar_wait(bar_s, par, abort_flag, WAIT_S, t);  // S(t) has read the key tile: request the next one
+                if (t + 1 < n_tiles) load_k(t + 1);
+                mbar_wait(bar_p, par, abort_flag, WAIT_P, t);
+                mbar_wait(bar_v, par, abort_flag, WAIT_V, t);
+                tc_fence_after();
+                // ---- O(t) = P(t) V(t): four steps of 16 keys
+#pragma unroll
+                for (int j = 0; j < TK / 16; ++j) {
+                    uint64_t vd[NS];
+#pragma unroll
+                    for (int a = 0; a < NS; ++a) vd[a] = smem_desc_sw128(sv + a * C::V_PART) + 2 * j;
+                    mma_ts(t_o, t_p + 8 * j, vd[0], idesc_o, j != 0);
+#pragma unroll
+                    for (int c = 0; c < 5; ++c) mma_ts(t_oc, t_p + CA[c] * (TK / 2) + 8 * j, vd[CB[c]], idesc_o, (j | c) != 0);
+                }
+                tc_commit(bar_o);
+            }
+            mbar_wait(bar_o, (n_tiles - 1) & 1, abort_flag, WAIT_O, n_tiles);
+            if (*abort_flag) {  // a wait gave up: the copies in flight must land before the shared memory goes back
+                mbar_wait_slow(bar_q, 0, abort_flag, WAIT_DRAIN, 0, kDrainClocks);
+                mbar_wait_slow(bar_k, (k_issued - 1) & 1, abort_flag, WAIT_DRAIN, 1, kDrainClocks);
+                mbar_wait_slow(bar_v, (v_issued - 1) & 1, abort_flag, WAIT_DRAIN, 2, kDrainClocks);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------- softmax and running output
+        const int quad = warp & 3, half = warp >> 2;
+        const int row = quad * 32 + lane, q = q0 + row;
+        const uint32_t lanes = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int lim = min(p.pos0 + q, p.n_keys - 1);  // the last key this query sees
+        float o[OD];
+#pragma unroll
+        for (int d = 0; d < OD; ++d) o[d] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;
+        for (int t = 0; t < n_tiles; ++t) {
+            const uint32_t par = t & 1;
+            float s[32];
+            float mx = -INFINITY;
+            mbar_wait(bar_s, par, abort_flag, WAIT_S, t);
+            tc_fence_after();
+            {
+                uint32_t lead[32], corr[32];
+                tmem_ld32(lanes + COL_S + 32 * half, lead);
+                tmem_ld32(lanes + COL_SC + 32 * half, corr);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int key0 = t * TK + 32 * half;
+                if (t * TK + TK - 1 <= min(p.pos0 + q0, p.n_keys - 1)) {  // every query of the CTA sees the whole tile
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        s[i] = (__uint_as_float(lead[i]) + __uint_as_float(corr[i])) * p.scale;
+                        mx = fmaxf(mx, s[i]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float v = (__uint_as_float(lead[i]) + __uint_as_float(corr[i])) * p.scale;
+                        s[i] = key0 + i <= lim ? v : -INFINITY;
+                        mx = fmaxf(mx, s[i]);
+                    }
+                }
+            }
+            row_max[(par * 2 + half) * TQ + row] = mx;
+            softmax_warps_sync();
+            mx = fmaxf(mx, row_max[(par * 2 + (half ^ 1)) * TQ + row]);
+            // exp(s - m) as 2^((s - m) log2 e): the difference is formed first, so the constant's rounding only
+            // touches the probability relatively.  Key 0 is visible to every query, so m_new is finite.
+            constexpr float kLog2e = 1.4426950408889634f;
+            const float m_new = fmaxf(m_run, mx);
+            const float corr = exp2_approx((m_run - m_new) * kLog2e);
+            m_run = m_new;
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                s[i] = exp2_approx((s[i] - m_new) * kLog2e);
+                sum += s[i];
+            }
+            l_run = l_run * corr + sum;
+#pragma unroll
+            for (int a = 0; a < NS; ++a) {
+                uint32_t w[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) w[i] = take_part(s[2 * i], s[2 * i + 1]);
+                tmem_st16(lanes + COL_P + a * (TK / 2) + 16 * half, w);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(bar_p);
+            if (__any_sync(0xffffffffu, corr != 1.f)) {  // (the maximum settles after a few tiles)
+#pragma unroll
+                for (int d = 0; d < OD; ++d) o[d] *= corr;
+            }
+            mbar_wait(bar_o, par, abort_flag, WAIT_O, t);
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < OD; c0 += 32) {
+                uint32_t lead[32], corr2[32];
+                tmem_ld32(lanes + COL_O + half * OD + c0, lead);
+                tmem_ld32(lanes + COL_OC + half * OD + c0, corr2);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c0 + i] += __uint_as_float(lead[i]) + __uint_as_float(corr2[i]);
+            }
+        }
+        // ---- out = O / l (the two halves of a row add their sums)
+        const int lb = n_tiles & 1;  // the buffer the last tile did not use
+        row_max[(lb * 2 + half) * TQ + row] = l_run;
+        softmax_warps_sync();
+        const float inv = 1.f / (l_run + row_max[(lb * 2 + (half ^ 1)) * TQ + row]);
+        if (q < p.T) {
+            float* dst = p.out + ((size_t)b * p.T + q) * ((size_t)p.nh * p.hd) + (size_t)h * p.hd + half * OD;
+            const int valid = p.hd - half * OD;  // head dims of this half that exist
+            if ((p.hd & 3) == 0) {
+#pragma unroll
+                for (int d = 0; d < OD; d += 4)
+                    if (d < valid) *reinterpret_cast<float4*>(dst + d) = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
+            } else {
+#pragma unroll
+                for (int d = 0; d < OD; ++d)
+                    if (d < valid) dst[d] = o[d] * inv;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == SOFTMAX_WARPS) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major, box = 64 columns (128 bytes) x box_rows, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_hdp(int hd) { return hd <= 64 ? 64 : 128; }
+
+struct Extents {
+    int hdp, t_pad, k_pad;
+    size_t q_part, kv_part;  // elements per part
+};
+Extents extents(int B, int nh, int hd, int T, int n_keys) {
+    Extents e;
+    e.hdp = pick_hdp(hd);
+    e.t_pad = (T + TQ - 1) / TQ * TQ;
+    e.k_pad = (n_keys + TK - 1) / TK * TK;
+    e.q_part = (size_t)B * nh * e.t_pad * e.hdp;
+    e.kv_part = (size_t)B * nh * e.k_pad * e.hdp;
+    return e;
+}
+
+template <int HDP>
+bitnet_a48_status launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int B,
+                              cudaStream_t st) {
+    using C = AttnCfg<HDP>;
+    A48_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<HDP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    A48_CUDA_TRY(a48_launch_pdl(attn_tc_kernel<HDP>, dim3(p.t_pad / TQ, p.nh, B), dim3(THREADS), (size_t)C::SMEM_BYTES, st, mq, mk, mv, p));
+    return BITNET_A48_OK;
+}
+
+}  // namespace
+
+bool a48_attn_tc_supported(int hd) { return hd >= 1 && hd <= 128; }
+
+// Scratch for the split operands: the parts of the queries (rows padded to 128), of the keys and of the transposed
+// values (positions padded to 64).
+size_t a48_attn_tc_workspace_bytes(int B, int nh, int hd, int T, int n_keys) {
+    const Extents e = extents(B, nh, hd, T, n_keys);
+    return NS * 2 * (e.q_part + 2 * e.kv_part);
+}
+
+// q [B*T][nh*hd] (already rotated); kcache / vcache fp32 [B][nh][cap][hd] holding positions [0, pos0 + T).
+bitnet_a48_status a48_launch_attn_tc(const float* q, const float* kcache, const float* vcache, int B, int T, int nh, int hd, int pos0,
+                                     int cap, float* out, void* ws, cudaStream_t st) {
+    if (!a48_attn_tc_supported(hd) || B > 65535 || nh > 65535) return BITNET_A48_ERR_UNSUPPORTED;
+    const int n_keys = pos0 + T;
+    const Extents e = extents(B, nh, hd, T, n_keys);
+    const size_t bh = (size_t)B * nh;
+    if (NS * bh * (size_t)(e.t_pad > e.k_pad ? e.t_pad : e.k_pad) >= (1ull << 31) || NS * bh * e.hdp >= (1ull << 31))
+        return BITNET_A48_ERR_UNSUPPORTED;  // tensor-copy coordinates are 32-bit
+    __nv_bfloat16* qs = static_cast<__nv_bfloat16*>(ws);
+    __nv_bfloat16* ks = qs + NS * e.q_part;
+    __nv_bfloat16* vs = ks + NS * e.kv_part;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, qs, NS * bh * e.t_pad, e.hdp, TQ) || !make_map(&mk, ks, NS * bh * e.k_pad, e.hdp, TK) ||
+        !make_map(&mv, vs, NS * bh * e.hdp, e.k_pad, e.hdp))
+        return BITNET_A48_ERR_CUDA;
+    int dev = 0, sms = 0;
+    A48_CUDA_TRY(cudaGetDevice(&dev));
+    A48_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const dim3 grid(sms * 8), block(256);
+    A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel, grid, block, 0, st, q, 0, B, nh, hd, e.hdp, T, e.t_pad, T, cap, qs, e.q_part));
+    A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel, grid, block, 0, st, kcache, 1, B, nh, hd, e.hdp, n_keys, e.k_pad, T, cap, ks, e.kv_part));
+    A48_CUDA_TRY(a48_launch_pdl(attn_split_vt_kernel, dim3(e.k_pad / TK, (unsigned)bh), block, (size_t)TK * (e.hdp + 1) * sizeof(float), st,
+                                vcache, hd, e.hdp, n_keys, e.k_pad, cap, vs, e.kv_part));
+    AttnParams p;
+    p.T = T;
+    p.t_pad = e.t_pad;
+    p.n_keys = n_keys;
+    p.k_pad = e.k_pad;
+    p.nh = nh;
+    p.hd = hd;
+    p.pos0 = pos0;
+    p.bh_total = (int)bh;
+    p.scale = 1.f / sqrtf((float)hd);
+    p.out = out;
+    return e.hdp == 64 ? launch_attn<64>(mq, mk, mv, p, B, st) : launch_attn<128>(mq, mk, mv, p, B, st);
+}
+
+bitnet_a48_status a48_read_attn_status(unsigned int words_host[4]) {
+    A48_CUDA_TRY(cudaMemcpyFromSymbol(words_host, g_attn_status, sizeof(unsigned int) * 4));
+    const unsigned int zero[4] = {0, 0, 0, 0};
+    A48_CUDA_TRY(cudaMemcpyToSymbol(g_attn_status, zero, sizeof(zero)));
+    return BITNET_A48_OK;
+}

@@ -31,10 +31,10 @@ BlockWs block_ws(const bitnet_a48_block* blk, int B, int T) {
     w.rope = take((size_t)T * (hd / 2) * 8);
     w.kc = take(M * H * 4);
     w.vc = take(M * H * 4);
-    // split-bf16 operands of the tensor-core prefill attention: queries of the call, keys/values of every position
-    // the call can reach (the cache's capacity, or the call's own tokens without a cache)
+    // operands of the tensor-core prefill attention split into bf16 parts: queries of the call, keys/values of every
+    // position the call can reach (the cache's capacity, or the call's own tokens without a cache)
     const int reach = blk->cfg.ctx_cap > T ? blk->cfg.ctx_cap : T;
-    w.mma = take(T > 8 && a48_attn_mma_supported((int)hd) ? a48_attn_mma_workspace_bytes(B, blk->cfg.n_heads, (int)hd, T, reach) : 0);
+    w.mma = take(T > 8 && a48_attn_tc_supported((int)hd) ? a48_attn_tc_workspace_bytes(B, blk->cfg.n_heads, (int)hd, T, reach) : 0);
     size_t lin = 0;
     for (int i = 0; i < 7; ++i) {
         size_t b = bitnet_a48_linear_workspace_bytes(blk->w[i], (int)M);
@@ -500,8 +500,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
                                             tile_path ? dq_k : nullptr, tile_path ? dq_v : nullptr, st));
         if (!tile_path) {
             A48_TRY(a48_launch_attn_row_lowbit(q, kcache, vcache, B, T, nh, hd, pos0, c.ctx_cap, c.kv_bits, att, st));
-        } else if (a48_attn_mma_supported(hd)) {
-            A48_TRY(a48_launch_attn_mma(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, base + o.mma, st));
+        } else if (a48_attn_tc_supported(hd)) {
+            A48_TRY(a48_launch_attn_tc(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, base + o.mma, st));
         } else if (hd <= 64) {
             A48_TRY(launch_attn_tile<64>(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, st));
         } else {
@@ -521,8 +521,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         if (hd <= 64) A48_CUDA_TRY(launch_attn_row<2>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
         else if (hd <= 128) A48_CUDA_TRY(launch_attn_row<4>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
         else A48_CUDA_TRY(launch_attn_row<8>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
-    } else if (a48_attn_mma_supported(hd)) {
-        A48_TRY(a48_launch_attn_mma(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, base + o.mma, st));
+    } else if (a48_attn_tc_supported(hd)) {
+        A48_TRY(a48_launch_attn_tc(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, base + o.mma, st));
     } else if (hd <= 64) {
         A48_TRY(launch_attn_tile<64>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     } else if (hd <= 128) {

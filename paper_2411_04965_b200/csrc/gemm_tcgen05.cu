@@ -1197,5 +1197,9 @@ bitnet_a48_status a48_read_kernel_status(unsigned int words_host[4]) {
     if (ds != BITNET_A48_OK) return ds;
     if (words_host[0] == 0 && dec[0] != 0)
         for (int i = 0; i < 4; ++i) words_host[i] = dec[i];
+    ds = a48_read_attn_status(dec);
+    if (ds != BITNET_A48_OK) return ds;
+    if (words_host[0] == 0 && dec[0] != 0)
+        for (int i = 0; i < 4; ++i) words_host[i] = dec[i];
     return BITNET_A48_OK;
 }

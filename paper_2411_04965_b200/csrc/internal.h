@@ -172,11 +172,12 @@ bool a48_decode_trit5_supported(const bitnet_a48_weight* w, int M);
 bitnet_a48_status a48_launch_decode_trit5(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M, float* Y,
                                           int32_t* acc, cudaStream_t st);
 
-// ---- attn_mma.cu (prefill attention on the tensor cores, split-bf16 operands)
-bool a48_attn_mma_supported(int hd);
-size_t a48_attn_mma_workspace_bytes(int B, int nh, int hd, int T, int n_keys);
-bitnet_a48_status a48_launch_attn_mma(const float* q, const float* kcache, const float* vcache, int B, int T, int nh, int hd,
-                                      int pos0, int cap, float* out, void* ws, cudaStream_t st);
+// ---- attn_tcgen05.cu (prefill attention on the tensor cores, operands split into bf16 parts)
+bool a48_attn_tc_supported(int hd);
+size_t a48_attn_tc_workspace_bytes(int B, int nh, int hd, int T, int n_keys);
+bitnet_a48_status a48_launch_attn_tc(const float* q, const float* kcache, const float* vcache, int B, int T, int nh, int hd,
+                                     int pos0, int cap, float* out, void* ws, cudaStream_t st);
+bitnet_a48_status a48_read_attn_status(unsigned int words_host[4]);
 
 // ---- block.cu
 size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T);
