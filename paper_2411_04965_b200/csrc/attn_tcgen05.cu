@@ -15,14 +15,17 @@
 // [0, pos0 + T) as bf16 arrays [part][B * heads][rows padded to a tile][head dim padded to 64 or 128];
 // attn_split_vt_kernel writes the parts of the values transposed, [part][B * heads][head dim][keys], so that both
 // operands of both contractions are K-major.  attn_tc_kernel: one CTA per (128 queries, head, sequence), 1 per SM.
-//   warp 8, one lane: tensor copies (TMA, 128-byte swizzle) of the query parts once and of one key tile (64 keys) and
-//     one value tile at a time, and all tcgen05.mma: S(t) = Q K(t)^T with both operands in shared memory, O(t) =
-//     P(t) V(t) with P in tensor memory.  Keys and values have one buffer each: K(t+1) is requested when S(t) has
-//     completed, V(t+1) when O(t) has, and S(t+1) is issued right behind O(t), so the copies and the softmax of
-//     the next tile overlap the MMAs of this one.
+//   warp 9, one lane: tensor copies (TMA, 128-byte swizzle) of the query parts once and of one key tile (64 keys) and
+//     one value tile at a time.  Keys and values have one buffer each: K(t+1) is requested when S(t) has completed,
+//     V(t+1) when O(t) has.
+//   warp 8, one lane: all tcgen05.mma.  S(t) = Q K(t)^T with both operands in shared memory goes to one of two score
+//     buffers in tensor memory; O(t) = P(t) V(t) takes P from tensor memory, where the softmax threads stored it over
+//     the scores.  The pipe runs S(0), S(1), O(0), S(2), O(1), ...: the scores of the next tile are ready while the
+//     softmax of this one is taken.  Measured, the MMAs themselves set the pace: a S(t) MMA (128 x 64 x 16, both
+//     operands from shared memory) takes about 60 clocks, which is the 6 KB it reads at 128 bytes per clock.
 //   warps 0-7: two threads per query row (tensor-memory lane), each with half of the tile's keys and half of the head
-//     dimension: read S, exchange the row maximum through shared memory, exponentials, split P into parts, store them
-//     to tensor memory, rescale the running output, then add O(t).
+//     dimension: read S(t), exchange the row maximum through shared memory, exponentials, split P into parts, store
+//     them to tensor memory, add O(t-1) (which ran meanwhile) to the running output and rescale it.
 // Every wait is bounded; a wait that gives up records itself (bitnet_a48_kernel_status) and lets every later wait of
 // the CTA fall through, so the kernel ends by itself; the issuer then waits for its copies in flight before it leaves.
 #include <cuda.h>
@@ -35,10 +38,11 @@ namespace {
 constexpr int TQ = 128;  // queries per CTA = MMA M = tensor-memory lanes
 constexpr int TK = 64;   // keys per tile: one 128-byte swizzle row of bf16
 constexpr int NS = 3;    // parts per operand
-constexpr int SOFTMAX_WARPS = 8, THREADS = 32 * (SOFTMAX_WARPS + 1);
+constexpr int SOFTMAX_WARPS = 8, MMA_WARP = SOFTMAX_WARPS, TMA_WARP = SOFTMAX_WARPS + 1, THREADS = 32 * (SOFTMAX_WARPS + 2);
 constexpr int TMEM_COLS = 512;
-// tensor-memory columns: S leading | S corrections | O(t) leading | O(t) corrections | P parts (two keys per column)
-constexpr int COL_S = 0, COL_SC = 64, COL_O = 128, COL_OC = 256, COL_P = 384;
+// Tensor-memory columns: two score buffers (leading products | corrections; the parts of P, two keys per column, are
+// stored over the scores once every thread has read them), then the leading and the correction accumulators of O(t).
+constexpr int COL_S = 0, S_BUF = 2 * TK, COL_O = 2 * S_BUF, COL_OC = COL_O + 128;
 constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
 constexpr unsigned long long kDrainClocks = 400000000ull;  // what the issuer grants its copies in flight when it gives up
 
@@ -229,7 +233,7 @@ struct AttnCfg {
     static constexpr int Q_BYTES = NS * KB * Q_BLOCK, K_BYTES = NS * KB * K_BLOCK, V_BYTES = NS * V_PART;
     static constexpr int SMEM_BYTES = Q_BYTES + K_BYTES + V_BYTES + 1024 /*alignment slack*/ + 4096 /*barriers, row maxima*/;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-    static_assert(COL_O + HDP <= COL_OC && COL_OC + HDP <= COL_P && COL_P + NS * TK / 2 <= TMEM_COLS, "tensor memory budget");
+    static_assert(COL_O + HDP <= COL_OC && COL_OC + HDP <= TMEM_COLS && NS * TK / 2 <= S_BUF, "tensor memory budget");
 };
 
 // barrier ids reported through the status words
@@ -248,8 +252,8 @@ __global__ void __launch_bounds__(THREADS, 1)
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 68);
     float* row_max = reinterpret_cast<float*>(ctrl + 1024);  // [tile parity][half][row]
     const uint32_t sq = smem_u32(smem), sk = sq + C::Q_BYTES, sv = sk + C::K_BYTES;
-    const uint32_t bar_q = smem_u32(ctrl), bar_k = bar_q + 8, bar_v = bar_q + 16, bar_s = bar_q + 24, bar_o = bar_q + 32,
-                   bar_p = bar_q + 40;
+    const uint32_t bar_q = smem_u32(ctrl), bar_k = bar_q + 8, bar_v = bar_q + 16, bar_s = bar_q + 24 /* two */, bar_o = bar_q + 40,
+                   bar_p = bar_q + 48;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -257,12 +261,13 @@ __global__ void __launch_bounds__(THREADS, 1)
         mbar_init(bar_k, 1);
         mbar_init(bar_v, 1);
         mbar_init(bar_s, 1);
+        mbar_init(bar_s + 8, 1);
         mbar_init(bar_o, 1);
         mbar_init(bar_p, 32 * SOFTMAX_WARPS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == SOFTMAX_WARPS) {
+    if (warp == MMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -278,9 +283,11 @@ __global__ void __launch_bounds__(THREADS, 1)
     const int keys_needed = min(p.n_keys, p.pos0 + min(q0 + TQ, p.T));  // causal: nothing beyond the last query's position
     const int n_tiles = (keys_needed + TK - 1) / TK;
 
-    if (warp == SOFTMAX_WARPS) {
+    if (warp == TMA_WARP) {
         if (lane == 0) {
-            // ------------------------------------------------------------- copies and MMAs
+            // ------------------------------------------------------------- tensor copies
+            // One buffer for keys, one for values: K(t+1) goes out when S(t) has completed, V(t+1) when O(t) has.  The
+            // tensor pipe runs S(0), S(1), O(0), S(2), O(1), S(3), ..., and the waits below follow that order.
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
@@ -308,17 +315,37 @@ __global__ void __launch_bounds__(THREADS, 1)
                     tma_load_2d(sq + (a * KB + kb) * C::Q_BLOCK, &tm_q, kb * 64, (a * p.bh_total + bh) * p.t_pad + q0, bar_q);
             load_k(0);
             load_v(0);
+            if (n_tiles > 1) {  // S(0) has read the key tile
+                mbar_wait(bar_s, 0, abort_flag, WAIT_S, 0);
+                load_k(1);
+            }
+            for (int t = 0; t + 1 < n_tiles; ++t) {
+                if (t + 2 < n_tiles) {  // S(t+1) has read the key tile
+                    mbar_wait(bar_s + 8 * ((t + 1) & 1), ((t + 1) >> 1) & 1, abort_flag, WAIT_S, t + 1);
+                    load_k(t + 2);
+                }
+                mbar_wait(bar_o, t & 1, abort_flag, WAIT_O, t);  // O(t) has read the value tile
+                load_v(t + 1);
+            }
+            if (*abort_flag) {  // a wait gave up: the copies in flight must land before the shared memory goes back
+                mbar_wait_slow(bar_q, 0, abort_flag, WAIT_DRAIN, 0, kDrainClocks);
+                mbar_wait_slow(bar_k, (k_issued - 1) & 1, abort_flag, WAIT_DRAIN, 1, kDrainClocks);
+                mbar_wait_slow(bar_v, (v_issued - 1) & 1, abort_flag, WAIT_DRAIN, 2, kDrainClocks);
+            }
+        }
+        __syncwarp();
+    } else if (warp == MMA_WARP) {
+        if (lane == 0) {
+            // ------------------------------------------------------------- MMAs
             constexpr uint32_t idesc_s = idesc_bf16(TQ, TK), idesc_o = idesc_bf16(TQ, HDP);
-            const uint32_t t_s = tmem_base + COL_S, t_sc = tmem_base + COL_SC, t_o = tmem_base + COL_O, t_oc = tmem_base + COL_OC,
-                           t_p = tmem_base + COL_P;
+            const uint32_t t_o = tmem_base + COL_O, t_oc = tmem_base + COL_OC;
             // the correction products, smallest first: (part of A, part of B)
             constexpr int CA[5] = {0, 1, 2, 0, 1}, CB[5] = {2, 1, 0, 1, 0};
-            mbar_wait(bar_q, 0, abort_flag, WAIT_Q, 0);
-            for (int t = 0; t < n_tiles; ++t) {
-                const uint32_t par = t & 1;
-                mbar_wait(bar_k, par, abort_flag, WAIT_K, t);
+            // S(t) = Q K(t)^T into score buffer t % 2: HDP / 16 steps of six MMAs
+            auto issue_s = [&](int t) {
+                mbar_wait(bar_k, t & 1, abort_flag, WAIT_K, t);
                 tc_fence_after();
-                // ---- S(t) = Q K(t)^T: HDP / 16 steps of six MMAs
+                const uint32_t t_s = tmem_base + COL_S + (t & 1) * S_BUF, t_sc = t_s + TK;
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
@@ -333,17 +360,18 @@ __global__ void __launch_bounds__(THREADS, 1)
 #pragma unroll
                         for (int c = 0; c < 5; ++c) mma_ss(t_sc, qd[CA[c]], kd[CB[c]], idesc_s, (kb | j | c) != 0);
                     }
-                tc_commit(bar_s);
-                if (t > 0) {  // O(t-1) has read the value tile: request the next one
-                    mbar_wait(bar_o, par ^ 1, abort_flag, WAIT_O, t);
-                    load_v(t);
-                }
-                mbar_wait(bar_s, par, abort_flag, WAIT_S, t);  // S(t) has read the key tile: request the next one
-                if (t + 1 < n_tiles) load_k(t + 1);
-                mbar_wait(bar_p, par, abort_flag, WAIT_P, t);
+                tc_commit(bar_s + 8 * (t & 1));
+            };
+            mbar_wait(bar_q, 0, abort_flag, WAIT_Q, 0);
+            issue_s(0);
+            if (n_tiles > 1) issue_s(1);
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t par = t & 1;
+                mbar_wait(bar_p, par, abort_flag, WAIT_P, t);  // P(t) is stored and O(t-1) has been read
                 mbar_wait(bar_v, par, abort_flag, WAIT_V, t);
                 tc_fence_after();
-                // ---- O(t) = P(t) V(t): four steps of 16 keys
+                // ---- O(t) = P(t) V(t): four steps of 16 keys; P(t) sits where S(t) was
+                const uint32_t t_p = tmem_base + COL_S + par * S_BUF;
 #pragma unroll
                 for (int j = 0; j < TK / 16; ++j) {
                     uint64_t vd[NS];
@@ -354,13 +382,9 @@ __global__ void __launch_bounds__(THREADS, 1)
                     for (int c = 0; c < 5; ++c) mma_ts(t_oc, t_p + CA[c] * (TK / 2) + 8 * j, vd[CB[c]], idesc_o, (j | c) != 0);
                 }
                 tc_commit(bar_o);
+                if (t + 2 < n_tiles) issue_s(t + 2);  // behind O(t) on the pipe, so P(t) is not overwritten early
             }
             mbar_wait(bar_o, (n_tiles - 1) & 1, abort_flag, WAIT_O, n_tiles);
-            if (*abort_flag) {  // a wait gave up: the copies in flight must land before the shared memory goes back
-                mbar_wait_slow(bar_q, 0, abort_flag, WAIT_DRAIN, 0, kDrainClocks);
-                mbar_wait_slow(bar_k, (k_issued - 1) & 1, abort_flag, WAIT_DRAIN, 1, kDrainClocks);
-                mbar_wait_slow(bar_v, (v_issued - 1) & 1, abort_flag, WAIT_DRAIN, 2, kDrainClocks);
-            }
         }
         __syncwarp();
     } else {
@@ -369,20 +393,36 @@ __global__ void __launch_bounds__(THREADS, 1)
         const int row = quad * 32 + lane, q = q0 + row;
         const uint32_t lanes = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int lim = min(p.pos0 + q, p.n_keys - 1);  // the last key this query sees
+        constexpr float kLog2e = 1.4426950408889634f;
         float o[OD];
 #pragma unroll
         for (int d = 0; d < OD; ++d) o[d] = 0.f;
         float m_run = -INFINITY, l_run = 0.f;
+        // o += O(t): the leading and the correction accumulators of this thread's head dims
+        auto add_tile = [&](int t) {
+            mbar_wait(bar_o, t & 1, abort_flag, WAIT_O, t);
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < OD; c0 += 32) {
+                uint32_t lead[32], corr2[32];
+                tmem_ld32(lanes + COL_O + half * OD + c0, lead);
+                tmem_ld32(lanes + COL_OC + half * OD + c0, corr2);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c0 + i] += __uint_as_float(lead[i]) + __uint_as_float(corr2[i]);
+            }
+        };
         for (int t = 0; t < n_tiles; ++t) {
             const uint32_t par = t & 1;
+            const uint32_t buf = lanes + COL_S + par * S_BUF;
             float s[32];
             float mx = -INFINITY;
-            mbar_wait(bar_s, par, abort_flag, WAIT_S, t);
+            mbar_wait(bar_s + 8 * par, (t >> 1) & 1, abort_flag, WAIT_S, t);
             tc_fence_after();
             {
                 uint32_t lead[32], corr[32];
-                tmem_ld32(lanes + COL_S + 32 * half, lead);
-                tmem_ld32(lanes + COL_SC + 32 * half, corr);
+                tmem_ld32(buf + 32 * half, lead);
+                tmem_ld32(buf + TK + 32 * half, corr);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int key0 = t * TK + 32 * half;
                 if (t * TK + TK - 1 <= min(p.pos0 + q0, p.n_keys - 1)) {  // every query of the CTA sees the whole tile
@@ -401,11 +441,10 @@ __global__ void __launch_bounds__(THREADS, 1)
                 }
             }
             row_max[(par * 2 + half) * TQ + row] = mx;
-            softmax_warps_sync();
+            softmax_warps_sync();  // (also: every thread has read its scores, so P may go where they were)
             mx = fmaxf(mx, row_max[(par * 2 + (half ^ 1)) * TQ + row]);
             // exp(s - m) as 2^((s - m) log2 e): the difference is formed first, so the constant's rounding only
             // touches the probability relatively.  Key 0 is visible to every query, so m_new is finite.
-            constexpr float kLog2e = 1.4426950408889634f;
             const float m_new = fmaxf(m_run, mx);
             const float corr = exp2_approx((m_run - m_new) * kLog2e);
             m_run = m_new;
@@ -421,27 +460,18 @@ __global__ void __launch_bounds__(THREADS, 1)
                 uint32_t w[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) w[i] = take_part(s[2 * i], s[2 * i + 1]);
-                tmem_st16(lanes + COL_P + a * (TK / 2) + 16 * half, w);
+                tmem_st16(buf + a * (TK / 2) + 16 * half, w);
             }
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            tc_fence_before();
-            mbar_arrive(bar_p);
+            if (t > 0) add_tile(t - 1);  // O(t-1) ran while the exponentials above were taken
             if (__any_sync(0xffffffffu, corr != 1.f)) {  // (the maximum settles after a few tiles)
 #pragma unroll
                 for (int d = 0; d < OD; ++d) o[d] *= corr;
             }
-            mbar_wait(bar_o, par, abort_flag, WAIT_O, t);
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < OD; c0 += 32) {
-                uint32_t lead[32], corr2[32];
-                tmem_ld32(lanes + COL_O + half * OD + c0, lead);
-                tmem_ld32(lanes + COL_OC + half * OD + c0, corr2);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[c0 + i] += __uint_as_float(lead[i]) + __uint_as_float(corr2[i]);
-            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(bar_p);  // P(t) is in place and the output accumulators are free for O(t)
         }
+        add_tile(n_tiles - 1);
         // ---- out = O / l (the two halves of a row add their sums)
         const int lb = n_tiles & 1;  // the buffer the last tile did not use
         row_max[(lb * 2 + half) * TQ + row] = l_run;
@@ -463,7 +493,7 @@ __global__ void __launch_bounds__(THREADS, 1)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == SOFTMAX_WARPS) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
