@@ -171,52 +171,79 @@ __device__ __forceinline__ float exp2_approx(float x) {
     return y;
 }
 
-// src rows of hd floats -> NS parts (part_stride elements apart) of rows of hdp bf16, zero past hd and for rows >=
-// rows_valid.  mode 0: queries, src = q [B*T][nh*hd], row (b, h, r) = token r of sequence b; mode 1: cache
-// [B][nh][cap][hd].
-__global__ void __launch_bounds__(256) attn_split_kernel(const float* __restrict__ src, int mode, int B, int nh, int hd, int hdp,
-                                                         int rows_valid, int rows_pad, int T, int cap,
-                                                         __nv_bfloat16* __restrict__ parts, size_t part_stride) {
-    a48_pdl_prologue();
-    const int pairs = hdp / 2;
-    const size_t total = (size_t)B * nh * rows_pad * pairs;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % pairs) * 2;
-        const size_t row = i / pairs;
-        const int r = (int)(row % rows_pad);
-        const size_t bh = row / rows_pad;
-        const int h = (int)(bh % nh), b = (int)(bh / nh);
-        float x = 0.f, y = 0.f;
-        if (r < rows_valid && c < hd) {
-            const float* p = mode == 0 ? src + ((size_t)b * T + r) * ((size_t)nh * hd) + (size_t)h * hd + c
-                                       : src + (((size_t)b * nh + h) * cap + r) * hd + c;
-            x = p[0];
-            y = c + 1 < hd ? p[1] : 0.f;
-        }
+// four floats -> the two bf16x2 words of each part
+__device__ __forceinline__ void split4(float (&v)[4], uint2 (&w)[NS]) {
 #pragma unroll
-        for (int a = 0; a < NS; ++a) reinterpret_cast<uint32_t*>(parts + a * part_stride)[i] = take_part(x, y);
+    for (int a = 0; a < NS; ++a) {
+        w[a].x = take_part(v[0], v[1]);
+        w[a].y = take_part(v[2], v[3]);
+    }
+}
+// four consecutive floats of a row of hd, zero past the row's end
+__device__ __forceinline__ void load4(const float* __restrict__ row, int c, int hd, bool vec, float (&v)[4]) {
+    if (vec && c + 3 < hd) {
+        const float4 f = *reinterpret_cast<const float4*>(row + c);
+        v[0] = f.x, v[1] = f.y, v[2] = f.z, v[3] = f.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = c + j < hd ? row[c + j] : 0.f;
     }
 }
 
-// The values of one head and 64 positions, transposed: vcache [B*nh][cap][hd] -> parts [part][B*nh][hdp][k_pad].
-// grid (k_pad / 64, B * nh); dynamic shared memory 64 * (hdp + 1) floats.
-__global__ void __launch_bounds__(256) attn_split_vt_kernel(const float* __restrict__ vcache, int hd, int hdp, int n_keys, int k_pad,
-                                                            int cap, __nv_bfloat16* __restrict__ parts, size_t part_stride) {
-    extern __shared__ float vt_tile[];  // [64 keys][hdp + 1]
+// src rows of hd floats -> NS parts (part_stride elements apart) of rows of HDP bf16, zero past hd and for rows >=
+// rows_valid.  mode 0: queries, src = q [B*T][nh*hd], row (b, h, r) = token r of sequence b; mode 1: cache
+// [B][nh][cap][hd].  grid (rows_pad / 64, nh, B): a block takes 64 rows of one head, a thread four head dims at a time.
+template <int HDP>
+__global__ void __launch_bounds__(256) attn_split_kernel(const float* __restrict__ src, int mode, int hd, int rows_valid, int rows_pad,
+                                                         int T, int cap, __nv_bfloat16* __restrict__ parts, size_t part_stride) {
     a48_pdl_prologue();
-    const int k0 = blockIdx.x * TK, ld = hdp + 1;
-    const size_t bh = blockIdx.y;
-    for (int i = threadIdx.x; i < TK * hdp; i += blockDim.x) {
-        const int key = i / hdp, d = i - key * hdp;
-        vt_tile[key * ld + d] = (k0 + key < n_keys && d < hd) ? vcache[(bh * cap + k0 + key) * hd + d] : 0.f;
+    constexpr int QUADS = HDP / 4, ROWS = 256 / QUADS;  // threads per row, rows per pass
+    const int nh = gridDim.y, h = blockIdx.y, b = blockIdx.z;
+    const size_t bh = (size_t)b * nh + h;
+    const int c = (threadIdx.x % QUADS) * 4;
+    const float* base = mode == 0 ? src + (size_t)b * T * nh * hd + (size_t)h * hd : src + bh * cap * hd;
+    const size_t pitch = mode == 0 ? (size_t)nh * hd : (size_t)hd;
+    const bool vec = (hd & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+    for (int r = blockIdx.x * 64 + threadIdx.x / QUADS; r < blockIdx.x * 64 + 64; r += ROWS) {
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (r < rows_valid && c < hd) load4(base + r * pitch, c, hd, vec, v);
+        uint2 w[NS];
+        split4(v, w);
+        const size_t o = (bh * rows_pad + r) * HDP + c;
+#pragma unroll
+        for (int a = 0; a < NS; ++a) *reinterpret_cast<uint2*>(parts + a * part_stride + o) = w[a];
+    }
+}
+
+// The values of one head and 64 positions, transposed: vcache [B*nh][cap][hd] -> parts [part][B*nh][HDP][k_pad].
+// grid (k_pad / 64, nh, B); a tile of 64 keys goes through shared memory.
+template <int HDP>
+__global__ void __launch_bounds__(256) attn_split_vt_kernel(const float* __restrict__ vcache, int hd, int n_keys, int k_pad, int cap,
+                                                            __nv_bfloat16* __restrict__ parts, size_t part_stride) {
+    constexpr int LD = HDP + 1;
+    __shared__ float vt_tile[TK * LD];  // [64 keys][HDP + 1]
+    a48_pdl_prologue();
+    const int k0 = blockIdx.x * TK;
+    const size_t bh = (size_t)blockIdx.z * gridDim.y + blockIdx.y;
+    const bool vec = (hd & 3) == 0 && (reinterpret_cast<uintptr_t>(vcache) & 15) == 0;
+    for (int i = threadIdx.x; i < TK * (HDP / 4); i += 256) {
+        const int key = i / (HDP / 4), d = (i % (HDP / 4)) * 4;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (k0 + key < n_keys && d < hd) load4(vcache + (bh * cap + k0 + key) * hd, d, hd, vec, v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) vt_tile[key * LD + d + j] = v[j];
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < hdp * (TK / 2); i += blockDim.x) {
-        const int d = i / (TK / 2), kp = i - d * (TK / 2);
-        float x = vt_tile[(2 * kp) * ld + d], y = vt_tile[(2 * kp + 1) * ld + d];
-        const size_t o = ((bh * hdp + d) * (size_t)k_pad + k0) / 2 + kp;
+    for (int i = threadIdx.x; i < HDP * (TK / 4); i += 256) {  // a thread: one head dim, four keys
+        const int d = i / (TK / 4), kq = (i % (TK / 4)) * 4;
+        float v[4];
 #pragma unroll
-        for (int a = 0; a < NS; ++a) reinterpret_cast<uint32_t*>(parts + a * part_stride)[o] = take_part(x, y);
+        for (int j = 0; j < 4; ++j) v[j] = vt_tile[(kq + j) * LD + d];
+        uint2 w[NS];
+        split4(v, w);
+        const size_t o = (bh * HDP + d) * (size_t)k_pad + k0 + kq;
+#pragma unroll
+        for (int a = 0; a < NS; ++a) *reinterpret_cast<uint2*>(parts + a * part_stride + o) = w[a];
     }
 }
 
@@ -578,14 +605,16 @@ bitnet_a48_status a48_launch_attn_tc(const float* q, const float* kcache, const 
     if (!make_map(&mq, qs, NS * bh * e.t_pad, e.hdp, TQ) || !make_map(&mk, ks, NS * bh * e.k_pad, e.hdp, TK) ||
         !make_map(&mv, vs, NS * bh * e.hdp, e.k_pad, e.hdp))
         return BITNET_A48_ERR_CUDA;
-    int dev = 0, sms = 0;
-    A48_CUDA_TRY(cudaGetDevice(&dev));
-    A48_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const dim3 grid(sms * 8), block(256);
-    A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel, grid, block, 0, st, q, 0, B, nh, hd, e.hdp, T, e.t_pad, T, cap, qs, e.q_part));
-    A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel, grid, block, 0, st, kcache, 1, B, nh, hd, e.hdp, n_keys, e.k_pad, T, cap, ks, e.kv_part));
-    A48_CUDA_TRY(a48_launch_pdl(attn_split_vt_kernel, dim3(e.k_pad / TK, (unsigned)bh), block, (size_t)TK * (e.hdp + 1) * sizeof(float), st,
-                                vcache, hd, e.hdp, n_keys, e.k_pad, cap, vs, e.kv_part));
+    const dim3 block(256), grid_q(e.t_pad / 64, nh, B), grid_k(e.k_pad / 64, nh, B), grid_v(e.k_pad / TK, nh, B);
+    if (e.hdp == 64) {
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel<64>, grid_q, block, 0, st, q, 0, hd, T, e.t_pad, T, cap, qs, e.q_part));
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel<64>, grid_k, block, 0, st, kcache, 1, hd, n_keys, e.k_pad, T, cap, ks, e.kv_part));
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_vt_kernel<64>, grid_v, block, 0, st, vcache, hd, n_keys, e.k_pad, cap, vs, e.kv_part));
+    } else {
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel<128>, grid_q, block, 0, st, q, 0, hd, T, e.t_pad, T, cap, qs, e.q_part));
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel<128>, grid_k, block, 0, st, kcache, 1, hd, n_keys, e.k_pad, T, cap, ks, e.kv_part));
+        A48_CUDA_TRY(a48_launch_pdl(attn_split_vt_kernel<128>, grid_v, block, 0, st, vcache, hd, n_keys, e.k_pad, cap, vs, e.kv_part));
+    }
     AttnParams p;
     p.T = T;
     p.t_pad = e.t_pad;

@@ -3,11 +3,13 @@
     python profile_cases.py gemm   --M 8192 --N 11008 --K 4096 --kind int4 --reps 3
     python profile_cases.py quant  --M 16384 --K 4096 --kind topk --reps 3
     python profile_cases.py decode --M 1 --N 11008 --K 4096 --kind topk --copies 32 --reps 3
+    python profile_cases.py block  --B 1 --T 2048 --hidden 4096 --ffn 11008 --heads 32 --reps 3
 
 Each case builds seeded synthetic inputs (the same recipes the benchmark uses),
 runs the kernel `reps` times after one warm-up call and prints the mean time
 from CUDA events on the launching stream.  `decode` cycles over `copies`
-distinct weight matrices so that the weight bytes come from HBM, not L2.
+distinct weight matrices so that the weight bytes come from HBM, not L2.  `block` is one transformer block on a
+prefill of B sequences of T tokens (quantisers, the seven BitLinears, RoPE, the tensor-core attention).
 (The sweep over the token count is a leg of the benchmark: `python bench.py --legs sweep`.)
 """
 from __future__ import annotations
@@ -48,7 +50,7 @@ def _acts(kind, M, K, dev, k_frac=0.5):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "quant", "decode"])
+    ap.add_argument("case", choices=["gemm", "quant", "decode", "block"])
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=11008)
     ap.add_argument("--K", type=int, default=4096)
@@ -56,6 +58,11 @@ def main():
     ap.add_argument("--algo", type=int, default=a48.ALGO_AUTO)
     ap.add_argument("--copies", type=int, default=32)
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--B", type=int, default=1)
+    ap.add_argument("--T", type=int, default=2048)
+    ap.add_argument("--hidden", type=int, default=4096)
+    ap.add_argument("--ffn", type=int, default=11008)
+    ap.add_argument("--heads", type=int, default=32)
     args = ap.parse_args()
     a48_build.build()
     dev = torch.device("cuda:0")
@@ -63,7 +70,21 @@ def main():
     stream = torch.cuda.current_stream()
     M, N, K = args.M, args.N, args.K
     out = {"case": args.case, "M": M, "N": N, "K": K, "kind": args.kind}
-    if args.case == "quant":
+    if args.case == "block":
+        Hs, Fs, B, T = args.hidden, args.ffn, args.B, args.T
+        shapes = (("q", Hs, Hs), ("k", Hs, Hs), ("v", Hs, Hs), ("o", Hs, Hs), ("gate", Fs, Hs), ("up", Fs, Hs), ("down", Hs, Fs))
+        w = {n: a48.pack_ternary(synth.ternary_latents(r, c, seed=200 + i, device=dev), EPS, a48.LAYOUT_ALL)
+             for i, (n, r, c) in enumerate(shapes)}
+        blk = a48.Block(w, synth.norm_gains(Hs, 60, device=dev), synth.norm_gains(Hs, 61, device=dev), n_heads=args.heads,
+                        k_o=Hs // 2, k_down=Fs // 2)
+        x = synth.gaussian_outlier_activations(B * T, Hs, seed=13, device=dev)
+        y = torch.empty_like(x)
+        wsp = torch.empty(blk.workspace_bytes(B, T), dtype=torch.uint8, device=dev)
+        ms = _time(lambda: blk.forward(x, B, T, Y=y, workspace=wsp), args.reps, stream)
+        hd = Hs // args.heads
+        out = {"case": "block", "B": B, "T": T, "hidden": Hs, "ffn": Fs, "heads": args.heads, "ms": ms,
+               "tokens_per_s": B * T / (ms * 1e-3), "attention_gflop": 4.0 * B * args.heads * (T * T / 2.0) * hd / 1e9}
+    elif args.case == "quant":
         x = (synth.student_t3 if args.kind == "topk" else synth.gaussian_outlier_activations)(M, K, 11, device=dev)
         codes = torch.empty(M, K, dtype=torch.int8, device=dev)
         scale = torch.empty(M, dtype=torch.float32, device=dev)
