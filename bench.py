@@ -921,7 +921,7 @@ def bench_block(a48, synth, dev, stream, layer):
     # the same steps with 4-bit queries and a 3-bit key/value cache (Section 3, low-bit attention)
     low = bench_block_decode(a48, synth, dev, stream, SHAPE_7B, (1, 8), layer=layer, q_bits=4, kv_bits=3)
     out["decode_b1_q4_kv3"], out["decode_b8_q4_kv3"] = low["b1"], low["b8"]
-    out["note"] = "one 7B-shape block (fp32 attention glue included); tokens/s per block, not per model"
+    out["note"] = "one 7B-shape block, attention included (prefill: tcgen05 on bf16-split operands; decode: fp32 or packed low-bit cache); tokens/s per block, not per model"
     return out
 
 
