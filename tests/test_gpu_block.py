@@ -56,6 +56,7 @@ def run_block_case(a48, oracle, dev, H, NH, F, B, T, pos0, cap, seed, scale, out
                                              kcache=kc.numpy(), vcache=vc.numpy(), k_o=H // 2, k_down=F // 2,
                                              nthreads=8)
     assert np.abs(ref - x.numpy()).max() > 0.05 * np.abs(ref).max(), "the block does not move the residual stream"
+    assert a48.kernel_status() == [0, 0, 0, 0]  # no bounded wait gave up (contraction, decode and attention kernels)
     assert rel_to_max(y.cpu().numpy(), ref) <= BLOCK_TOL
     assert rel_above_floor(y.cpu().numpy(), ref) <= BLOCK_TOL
     assert rel_to_max(kc_d[:, :, pos0:pos0 + T].cpu().numpy(), k_new) <= 1e-5
@@ -114,11 +115,18 @@ def test_block_head_dims_of_the_model_table(a48, oracle, cuda_dev, hd, B, T, pos
 
 # Prefill long enough for several 128-query tiles of the tensor-core attention kernel, with many key tiles per query
 # tile, a ragged last tile of both, and (second and third case) cached positions in front of the call's own.
-@pytest.mark.parametrize("hd,B,T,pos0", [(64, 2, 300, 0), (128, 1, 200, 150), (96, 1, 260, 37), (100, 1, 129, 0)])
+@pytest.mark.parametrize("hd,B,T,pos0", [(64, 2, 300, 0), (128, 1, 200, 150), (96, 1, 260, 37), (100, 1, 129, 0),
+                                         (36, 3, 9, 5), (128, 2, 128, 0), (64, 1, 64, 64)])
 def test_block_prefill_several_attention_tiles(a48, oracle, cuda_dev, hd, B, T, pos0):
     NH = 2
     H, F = NH * hd, 2 * NH * hd + 8 * (hd % 32 != 0)
     run_block_case(a48, oracle, cuda_dev, H, NH, F, B, T, pos0, cap=448, seed=hd + T, scale=10.0, outliers=2)
+
+
+# Head dims above 128 stay on the fp32 tile kernel (prefill) and the eight-keys-per-warp row kernel (decode).
+@pytest.mark.parametrize("B,T,pos0", [(1, 70, 0), (2, 1, 300), (1, 12, 290)])
+def test_block_head_dim_160(a48, oracle, cuda_dev, B, T, pos0):
+    run_block_case(a48, oracle, cuda_dev, 320, 2, 640, B, T, pos0, cap=320, seed=160 + T, scale=10.0, outliers=2)
 
 
 # One block of the 7B shape (hidden 4096, 32 heads of 128, FFN 11008) and of the 3B shape (3200, 32 heads of 100,
