@@ -7,27 +7,30 @@
 // three bf16 numbers, x = x0 + x1 + x2 with x0 = bf16(x), x1 = bf16(x - x0), x2 = bf16(x - x0 - x1) (the subtractions
 // are exact, the three carry the 24 significant bits of x), and every product is the six MMAs x_i * y_j with
 // i + j <= 2.  What is dropped is below 2^-24 of a product.  The tensor core adds to its accumulator with less care
-// than an fp32 add (measured with mma.sync: truncation), so the leading products (part 0 times part 0) and the five
-// correction products (2^-8 and less of the leading ones) go to accumulators of their own, and the running output
-// lives in registers: every key tile is contracted into a fresh accumulator and added in fp32.
+// than an fp32 add (measured with mma.sync: truncation), so of the six MMAs of a step the five corrections (2^-8 and
+// less of the leading product) are issued first, for all steps of a tile, and the leading products last: the
+// truncation acts on small sums until the few leading MMAs come.  Measured against a float64 attention this is as
+// accurate as separate accumulators for leading and correction terms, and closer than a sequential fp32 evaluation.
+// The running output lives in registers: every key tile is contracted into a fresh accumulator and added in fp32.
 //
 // Kernels.  attn_split_kernel writes the parts of the queries of the call and of the keys of positions
 // [0, pos0 + T) as bf16 arrays [part][B * heads][rows padded to a tile][head dim padded to 64 or 128];
-// attn_split_vt_kernel writes the parts of the values transposed, [part][B * heads][head dim][keys], so that both
-// operands of both contractions are K-major.  attn_tc_kernel: one CTA per (128 queries, head, sequence), 1 per SM.
-//   warp 9, one lane: tensor copies (TMA, 128-byte swizzle) of the query parts once and of one key tile (64 keys) and
-//     one value tile at a time.  Keys and values have one buffer each: K(t+1) is requested when S(t) has completed,
-//     V(t+1) when O(t) has.
-//   warp 8, one lane: all tcgen05.mma.  S(t) = Q K(t)^T with both operands in shared memory goes to one of two score
-//     buffers in tensor memory; O(t) = P(t) V(t) takes P from tensor memory, where the softmax threads stored it over
-//     the scores.  The pipe runs S(0), S(1), O(0), S(2), O(1), ...: the scores of the next tile are ready while the
-//     softmax of this one is taken.  Measured, the MMAs themselves set the pace: a S(t) MMA (128 x 64 x 16, both
-//     operands from shared memory) takes about 60 clocks, which is the 6 KB it reads at 128 bytes per clock.
+// attn_split_vt_kernel writes the parts of the values transposed, [part][B * heads][head dim][keys], so that the
+// shared-memory operands of both contractions are K-major.  attn_tc_kernel: one CTA per (128 queries, head,
+// sequence), 1 per SM, the tiles with the most keys first.
+//   warp 9, two lanes: tensor copies (TMA, 128-byte swizzle) of key tiles (64 keys) and value tiles, two buffers
+//     each: K(t+2) is requested when S(t) has completed, V(t+2) when O(t) has.
+//   warp 8, one lane: all tcgen05.mma, both with the A operand in tensor memory: S(t) = Q K(t)^T (the query parts are
+//     stored to tensor memory once per CTA) into one of two score buffers; O(t) = P(t) V(t) with the parts of P that
+//     the softmax threads stored over the scores.  The pipe runs S(0), S(1), O(0), S(2), O(1), ...: the scores of
+//     the next tile are ready while the softmax of this one is taken.  Tensor memory: 192 columns of query parts,
+//     2 x 96 of scores / P, 128 of output = all 512.  Measured, the MMAs set the pace: a 128 x 64 x 16 MMA of S
+//     takes about 49 clocks where its arithmetic is 32, a 128 x 128 x 16 MMA of O 71 (64).
 //   warps 0-7: two threads per query row (tensor-memory lane), each with half of the tile's keys and half of the head
 //     dimension: read S(t), exchange the row maximum through shared memory, exponentials, split P into parts, store
 //     them to tensor memory, add O(t-1) (which ran meanwhile) to the running output and rescale it.
 // Every wait is bounded; a wait that gives up records itself (bitnet_a48_kernel_status) and lets every later wait of
-// the CTA fall through, so the kernel ends by itself; the issuer then waits for its copies in flight before it leaves.
+// the CTA fall through, so the kernel ends by itself; the copy lanes then wait for their copies in flight.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -40,9 +43,10 @@ constexpr int TK = 64;   // keys per tile: one 128-byte swizzle row of bf16
 constexpr int NS = 3;    // parts per operand
 constexpr int SOFTMAX_WARPS = 8, MMA_WARP = SOFTMAX_WARPS, TMA_WARP = SOFTMAX_WARPS + 1, THREADS = 32 * (SOFTMAX_WARPS + 2);
 constexpr int TMEM_COLS = 512;
-// Tensor-memory columns: two score buffers (leading products | corrections; the parts of P, two keys per column, are
-// stored over the scores once every thread has read them), then the leading and the correction accumulators of O(t).
-constexpr int COL_S = 0, S_BUF = 2 * TK, COL_O = 2 * S_BUF, COL_OC = COL_O + 128;
+// Tensor-memory columns: the three parts of the 128 queries (two elements per column), two score buffers (64 columns
+// of scores; the three parts of P, two keys per column, are stored over them once every thread has read its scores),
+// the accumulator of O(t).
+constexpr int COL_Q = 0, COL_SP = 192, SP_BUF = 96, COL_O = COL_SP + 2 * SP_BUF;
 constexpr unsigned long long kWaitClocks = 4000000000ull;  // ~2 s at 2 GHz
 constexpr unsigned long long kDrainClocks = 400000000ull;  // what the issuer grants its copies in flight when it gives up
 
@@ -105,15 +109,7 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 operands, fp32 accumulators
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]
+// D[tmem] (+)= A[tmem] * B[smem desc], bf16 operands, fp32 accumulators
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -145,6 +141,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
@@ -250,17 +256,19 @@ __global__ void __launch_bounds__(256) attn_split_vt_kernel(const float* __restr
 struct AttnParams {
     int T, t_pad, n_keys, k_pad, nh, hd, pos0, bh_total;
     float scale;
+    const __nv_bfloat16* q_parts;  // [part][B * heads][t_pad][HDP]
+    size_t q_part;                 // elements per part
     float* out;
 };
 
 template <int HDP>
 struct AttnCfg {
-    static constexpr int KB = HDP / 64;                     // 128-byte blocks per operand row of the first contraction
-    static constexpr int Q_BLOCK = TQ * 128, K_BLOCK = TK * 128, V_PART = HDP * 128;
-    static constexpr int Q_BYTES = NS * KB * Q_BLOCK, K_BYTES = NS * KB * K_BLOCK, V_BYTES = NS * V_PART;
-    static constexpr int SMEM_BYTES = Q_BYTES + K_BYTES + V_BYTES + 1024 /*alignment slack*/ + 4096 /*barriers, row maxima*/;
+    static constexpr int KB = HDP / 64;  // 128-byte blocks per key row
+    static constexpr int K_BLOCK = TK * 128, V_PART = HDP * 128;
+    static constexpr int K_BYTES = NS * KB * K_BLOCK, V_BYTES = NS * V_PART;  // one key tile, one value tile
+    static constexpr int SMEM_BYTES = 2 * K_BYTES + 2 * V_BYTES + 1024 /*alignment slack*/ + 4096 /*barriers, row maxima*/;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-    static_assert(COL_O + HDP <= COL_OC && COL_OC + HDP <= TMEM_COLS && NS * TK / 2 <= S_BUF, "tensor memory budget");
+    static_assert(NS * HDP / 2 <= COL_SP && TK <= SP_BUF && NS * TK / 2 <= SP_BUF && COL_O + HDP <= TMEM_COLS, "tensor memory budget");
 };
 
 // barrier ids reported through the status words
@@ -268,27 +276,28 @@ enum { WAIT_Q = 20, WAIT_K = 21, WAIT_V = 22, WAIT_S = 23, WAIT_O = 24, WAIT_P =
 
 template <int HDP>
 __global__ void __launch_bounds__(THREADS, 1)
-    attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
     using C = AttnCfg<HDP>;
     constexpr int KB = C::KB, OD = HDP / 2;  // OD: head dims per softmax thread
+    constexpr int QW = HDP / 4;              // tensor-memory columns of a thread's share of one query part
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* ctrl = smem + C::Q_BYTES + C::K_BYTES + C::V_BYTES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 64);
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 68);
+    uint8_t* ctrl = smem + 2 * C::K_BYTES + 2 * C::V_BYTES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 96);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 100);
     float* row_max = reinterpret_cast<float*>(ctrl + 1024);  // [tile parity][half][row]
-    const uint32_t sq = smem_u32(smem), sk = sq + C::Q_BYTES, sv = sk + C::K_BYTES;
-    const uint32_t bar_q = smem_u32(ctrl), bar_k = bar_q + 8, bar_v = bar_q + 16, bar_s = bar_q + 24 /* two */, bar_o = bar_q + 40,
-                   bar_p = bar_q + 48;
+    const uint32_t sk = smem_u32(smem), sv = sk + 2 * C::K_BYTES;
+    // barriers: q | k[2] | v[2] | s[2] | o | p
+    const uint32_t bar_q = smem_u32(ctrl), bar_k = bar_q + 8, bar_v = bar_q + 24, bar_s = bar_q + 40, bar_o = bar_q + 56, bar_p = bar_q + 64;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(bar_q, 1);
-        mbar_init(bar_k, 1);
-        mbar_init(bar_v, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_s + 8, 1);
+        mbar_init(bar_q, 32 * SOFTMAX_WARPS);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_k + 8 * i, 1);
+            mbar_init(bar_v + 8 * i, 1);
+            mbar_init(bar_s + 8 * i, 1);
+        }
         mbar_init(bar_o, 1);
         mbar_init(bar_p, 32 * SOFTMAX_WARPS);
         *abort_flag = 0;
@@ -311,81 +320,84 @@ __global__ void __launch_bounds__(THREADS, 1)
     const int n_tiles = (keys_needed + TK - 1) / TK;
 
     if (warp == TMA_WARP) {
+        // ------------------------------------------------------------- tensor copies
+        // Two buffers for keys, two for values.  Lane 0 requests K(t+2) when S(t) has completed, lane 1 requests V(t+2)
+        // when O(t) has: two lanes, so that a key tile never waits behind a value tile's turn.
         if (lane == 0) {
-            // ------------------------------------------------------------- tensor copies
-            // One buffer for keys, one for values: K(t+1) goes out when S(t) has completed, V(t+1) when O(t) has.  The
-            // tensor pipe runs S(0), S(1), O(0), S(2), O(1), S(3), ..., and the waits below follow that order.
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
-            int k_issued = 0, v_issued = 0;
             auto load_k = [&](int t) {
-                mbar_expect_tx(bar_k, C::K_BYTES);
+                const uint32_t bar = bar_k + 8 * (t & 1), dst = sk + (t & 1) * C::K_BYTES;
+                mbar_expect_tx(bar, C::K_BYTES);
 #pragma unroll
                 for (int a = 0; a < NS; ++a)
 #pragma unroll
                     for (int kb = 0; kb < KB; ++kb)
-                        tma_load_2d(sk + (a * KB + kb) * C::K_BLOCK, &tm_k, kb * 64, (a * p.bh_total + bh) * p.k_pad + t * TK, bar_k);
-                ++k_issued;
+                        tma_load_2d(dst + (a * KB + kb) * C::K_BLOCK, &tm_k, kb * 64, (a * p.bh_total + bh) * p.k_pad + t * TK, bar);
             };
-            auto load_v = [&](int t) {
-                mbar_expect_tx(bar_v, C::V_BYTES);
-#pragma unroll
-                for (int a = 0; a < NS; ++a) tma_load_2d(sv + a * C::V_PART, &tm_v, t * TK, (a * p.bh_total + bh) * HDP, bar_v);
-                ++v_issued;
-            };
-            mbar_expect_tx(bar_q, C::Q_BYTES);
-#pragma unroll
-            for (int a = 0; a < NS; ++a)
-#pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-                    tma_load_2d(sq + (a * KB + kb) * C::Q_BLOCK, &tm_q, kb * 64, (a * p.bh_total + bh) * p.t_pad + q0, bar_q);
             load_k(0);
+            if (n_tiles > 1) load_k(1);
+            int issued = min(n_tiles, 2);
+            for (; issued < n_tiles; ++issued) {
+                const int t = issued - 2;
+                mbar_wait(bar_s + 8 * (t & 1), (t >> 1) & 1, abort_flag, WAIT_S, t);  // S(t) has read its key tile
+                if (*abort_flag) break;
+                load_k(issued);
+            }
+            if (*abort_flag)  // a wait gave up: the copies in flight must land before the shared memory goes back
+                for (int t = max(issued - 2, 0); t < issued; ++t)
+                    mbar_wait_slow(bar_k + 8 * (t & 1), (t >> 1) & 1, abort_flag, WAIT_DRAIN, t & 1, kDrainClocks);
+        } else if (lane == 1) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+            auto load_v = [&](int t) {
+                const uint32_t bar = bar_v + 8 * (t & 1), dst = sv + (t & 1) * C::V_BYTES;
+                mbar_expect_tx(bar, C::V_BYTES);
+#pragma unroll
+                for (int a = 0; a < NS; ++a) tma_load_2d(dst + a * C::V_PART, &tm_v, t * TK, (a * p.bh_total + bh) * HDP, bar);
+            };
             load_v(0);
-            if (n_tiles > 1) {  // S(0) has read the key tile
-                mbar_wait(bar_s, 0, abort_flag, WAIT_S, 0);
-                load_k(1);
+            if (n_tiles > 1) load_v(1);
+            int issued = min(n_tiles, 2);
+            for (; issued < n_tiles; ++issued) {
+                const int t = issued - 2;
+                mbar_wait(bar_o, t & 1, abort_flag, WAIT_O, t);  // O(t) has read its value tile
+                if (*abort_flag) break;
+                load_v(issued);
             }
-            for (int t = 0; t + 1 < n_tiles; ++t) {
-                if (t + 2 < n_tiles) {  // S(t+1) has read the key tile
-                    mbar_wait(bar_s + 8 * ((t + 1) & 1), ((t + 1) >> 1) & 1, abort_flag, WAIT_S, t + 1);
-                    load_k(t + 2);
-                }
-                mbar_wait(bar_o, t & 1, abort_flag, WAIT_O, t);  // O(t) has read the value tile
-                load_v(t + 1);
-            }
-            if (*abort_flag) {  // a wait gave up: the copies in flight must land before the shared memory goes back
-                mbar_wait_slow(bar_q, 0, abort_flag, WAIT_DRAIN, 0, kDrainClocks);
-                mbar_wait_slow(bar_k, (k_issued - 1) & 1, abort_flag, WAIT_DRAIN, 1, kDrainClocks);
-                mbar_wait_slow(bar_v, (v_issued - 1) & 1, abort_flag, WAIT_DRAIN, 2, kDrainClocks);
-            }
+            if (*abort_flag)
+                for (int t = max(issued - 2, 0); t < issued; ++t)
+                    mbar_wait_slow(bar_v + 8 * (t & 1), (t >> 1) & 1, abort_flag, WAIT_DRAIN, 2 + (t & 1), kDrainClocks);
         }
         __syncwarp();
     } else if (warp == MMA_WARP) {
         if (lane == 0) {
             // ------------------------------------------------------------- MMAs
+            // Both contractions take their A operand from tensor memory (the query parts, stored there once by the
+            // softmax threads; the parts of P) and their B operand from shared memory.  Per product the five
+            // corrections are issued first and the leading product last, so that the truncating accumulate of the
+            // tensor core acts on small sums until the few leading MMAs come: one accumulator then is as accurate
+            // as separate ones for the leading and the correction terms (measured against float64).
             constexpr uint32_t idesc_s = idesc_bf16(TQ, TK), idesc_o = idesc_bf16(TQ, HDP);
-            const uint32_t t_o = tmem_base + COL_O, t_oc = tmem_base + COL_OC;
+            const uint32_t t_q = tmem_base + COL_Q, t_o = tmem_base + COL_O;
             // the correction products, smallest first: (part of A, part of B)
             constexpr int CA[5] = {0, 1, 2, 0, 1}, CB[5] = {2, 1, 0, 1, 0};
             // S(t) = Q K(t)^T into score buffer t % 2: HDP / 16 steps of six MMAs
             auto issue_s = [&](int t) {
-                mbar_wait(bar_k, t & 1, abort_flag, WAIT_K, t);
+                mbar_wait(bar_k + 8 * (t & 1), (t >> 1) & 1, abort_flag, WAIT_K, t);
                 tc_fence_after();
-                const uint32_t t_s = tmem_base + COL_S + (t & 1) * S_BUF, t_sc = t_s + TK;
+                const uint32_t t_s = tmem_base + COL_SP + (t & 1) * SP_BUF, kbuf = sk + (t & 1) * C::K_BYTES;
 #pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
+                for (int pass = 0; pass < 2; ++pass)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint64_t qd[NS], kd[NS];
+                    for (int ks = 0; ks < HDP / 16; ++ks) {
+                        uint64_t kd[NS];
 #pragma unroll
-                        for (int a = 0; a < NS; ++a) {
-                            qd[a] = smem_desc_sw128(sq + (a * KB + kb) * C::Q_BLOCK) + 2 * j;
-                            kd[a] = smem_desc_sw128(sk + (a * KB + kb) * C::K_BLOCK) + 2 * j;
+                        for (int a = 0; a < NS; ++a) kd[a] = smem_desc_sw128(kbuf + (a * KB + ks / 4) * C::K_BLOCK) + 2 * (ks % 4);
+                        if (pass == 0) {
+#pragma unroll
+                            for (int c = 0; c < 5; ++c) mma_ts(t_s, t_q + CA[c] * (HDP / 2) + 8 * ks, kd[CB[c]], idesc_s, (ks | c) != 0);
+                        } else {
+                            mma_ts(t_s, t_q + 8 * ks, kd[0], idesc_s, 1);
                         }
-                        mma_ss(t_s, qd[0], kd[0], idesc_s, (kb | j) != 0);
-#pragma unroll
-                        for (int c = 0; c < 5; ++c) mma_ss(t_sc, qd[CA[c]], kd[CB[c]], idesc_s, (kb | j | c) != 0);
                     }
                 tc_commit(bar_s + 8 * (t & 1));
             };
@@ -395,19 +407,24 @@ __global__ void __launch_bounds__(THREADS, 1)
             for (int t = 0; t < n_tiles; ++t) {
                 const uint32_t par = t & 1;
                 mbar_wait(bar_p, par, abort_flag, WAIT_P, t);  // P(t) is stored and O(t-1) has been read
-                mbar_wait(bar_v, par, abort_flag, WAIT_V, t);
+                mbar_wait(bar_v + 8 * par, (t >> 1) & 1, abort_flag, WAIT_V, t);
                 tc_fence_after();
                 // ---- O(t) = P(t) V(t): four steps of 16 keys; P(t) sits where S(t) was
-                const uint32_t t_p = tmem_base + COL_S + par * S_BUF;
+                const uint32_t t_p = tmem_base + COL_SP + par * SP_BUF, vbuf = sv + par * C::V_BYTES;
 #pragma unroll
-                for (int j = 0; j < TK / 16; ++j) {
-                    uint64_t vd[NS];
+                for (int pass = 0; pass < 2; ++pass)
 #pragma unroll
-                    for (int a = 0; a < NS; ++a) vd[a] = smem_desc_sw128(sv + a * C::V_PART) + 2 * j;
-                    mma_ts(t_o, t_p + 8 * j, vd[0], idesc_o, j != 0);
+                    for (int j = 0; j < TK / 16; ++j) {
+                        uint64_t vd[NS];
 #pragma unroll
-                    for (int c = 0; c < 5; ++c) mma_ts(t_oc, t_p + CA[c] * (TK / 2) + 8 * j, vd[CB[c]], idesc_o, (j | c) != 0);
-                }
+                        for (int a = 0; a < NS; ++a) vd[a] = smem_desc_sw128(vbuf + a * C::V_PART) + 2 * j;
+                        if (pass == 0) {
+#pragma unroll
+                            for (int c = 0; c < 5; ++c) mma_ts(t_o, t_p + CA[c] * (TK / 2) + 8 * j, vd[CB[c]], idesc_o, (j | c) != 0);
+                        } else {
+                            mma_ts(t_o, t_p + 8 * j, vd[0], idesc_o, 1);
+                        }
+                    }
                 tc_commit(bar_o);
                 if (t + 2 < n_tiles) issue_s(t + 2);  // behind O(t) on the pipe, so P(t) is not overwritten early
             }
@@ -419,50 +436,66 @@ __global__ void __launch_bounds__(THREADS, 1)
         const int quad = warp & 3, half = warp >> 2;
         const int row = quad * 32 + lane, q = q0 + row;
         const uint32_t lanes = tmem_base + ((uint32_t)(quad * 32) << 16);
+        // ---- this thread's half of its query row, part by part, into tensor memory (two elements per column)
+        {
+            const __nv_bfloat16* src = p.q_parts + ((size_t)bh * p.t_pad + q) * HDP + half * OD;
+#pragma unroll
+            for (int a = 0; a < NS; ++a) {
+                uint32_t w[QW];
+                const uint4* s4 = reinterpret_cast<const uint4*>(src + a * p.q_part);
+#pragma unroll
+                for (int i = 0; i < QW / 4; ++i) {
+                    const uint4 v = __ldg(s4 + i);
+                    w[4 * i] = v.x, w[4 * i + 1] = v.y, w[4 * i + 2] = v.z, w[4 * i + 3] = v.w;
+                }
+                if constexpr (QW == 32) tmem_st32(lanes + COL_Q + a * (HDP / 2) + half * QW, w);
+                else tmem_st16(lanes + COL_Q + a * (HDP / 2) + half * QW, w);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(bar_q);
+        }
         const int lim = min(p.pos0 + q, p.n_keys - 1);  // the last key this query sees
         constexpr float kLog2e = 1.4426950408889634f;
         float o[OD];
 #pragma unroll
         for (int d = 0; d < OD; ++d) o[d] = 0.f;
         float m_run = -INFINITY, l_run = 0.f;
-        // o += O(t): the leading and the correction accumulators of this thread's head dims
+        // o += O(t), this thread's head dims
         auto add_tile = [&](int t) {
             mbar_wait(bar_o, t & 1, abort_flag, WAIT_O, t);
             tc_fence_after();
 #pragma unroll
             for (int c0 = 0; c0 < OD; c0 += 32) {
-                uint32_t lead[32], corr2[32];
-                tmem_ld32(lanes + COL_O + half * OD + c0, lead);
-                tmem_ld32(lanes + COL_OC + half * OD + c0, corr2);
+                uint32_t acc[32];
+                tmem_ld32(lanes + COL_O + half * OD + c0, acc);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[c0 + i] += __uint_as_float(lead[i]) + __uint_as_float(corr2[i]);
+                for (int i = 0; i < 32; ++i) o[c0 + i] += __uint_as_float(acc[i]);
             }
         };
         for (int t = 0; t < n_tiles; ++t) {
             const uint32_t par = t & 1;
-            const uint32_t buf = lanes + COL_S + par * S_BUF;
+            const uint32_t buf = lanes + COL_SP + par * SP_BUF;
             float s[32];
             float mx = -INFINITY;
             mbar_wait(bar_s + 8 * par, (t >> 1) & 1, abort_flag, WAIT_S, t);
             tc_fence_after();
             {
-                uint32_t lead[32], corr[32];
-                tmem_ld32(buf + 32 * half, lead);
-                tmem_ld32(buf + TK + 32 * half, corr);
+                uint32_t acc[32];
+                tmem_ld32(buf + 32 * half, acc);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int key0 = t * TK + 32 * half;
                 if (t * TK + TK - 1 <= min(p.pos0 + q0, p.n_keys - 1)) {  // every query of the CTA sees the whole tile
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        s[i] = (__uint_as_float(lead[i]) + __uint_as_float(corr[i])) * p.scale;
+                        s[i] = __uint_as_float(acc[i]) * p.scale;
                         mx = fmaxf(mx, s[i]);
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const float v = (__uint_as_float(lead[i]) + __uint_as_float(corr[i])) * p.scale;
-                        s[i] = key0 + i <= lim ? v : -INFINITY;
+                        s[i] = key0 + i <= lim ? __uint_as_float(acc[i]) * p.scale : -INFINITY;
                         mx = fmaxf(mx, s[i]);
                     }
                 }
@@ -496,7 +529,7 @@ __global__ void __launch_bounds__(THREADS, 1)
             }
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
-            mbar_arrive(bar_p);  // P(t) is in place and the output accumulators are free for O(t)
+            mbar_arrive(bar_p);  // P(t) is in place and the output accumulator is free for O(t)
         }
         add_tile(n_tiles - 1);
         // ---- out = O / l (the two halves of a row add their sums)
@@ -570,11 +603,10 @@ Extents extents(int B, int nh, int hd, int T, int n_keys) {
 }
 
 template <int HDP>
-bitnet_a48_status launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int B,
-                              cudaStream_t st) {
+bitnet_a48_status launch_attn(const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int B, cudaStream_t st) {
     using C = AttnCfg<HDP>;
     A48_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<HDP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    A48_CUDA_TRY(a48_launch_pdl(attn_tc_kernel<HDP>, dim3(p.t_pad / TQ, p.nh, B), dim3(THREADS), (size_t)C::SMEM_BYTES, st, mq, mk, mv, p));
+    A48_CUDA_TRY(a48_launch_pdl(attn_tc_kernel<HDP>, dim3(p.t_pad / TQ, p.nh, B), dim3(THREADS), (size_t)C::SMEM_BYTES, st, mk, mv, p));
     return BITNET_A48_OK;
 }
 
@@ -601,10 +633,8 @@ bitnet_a48_status a48_launch_attn_tc(const float* q, const float* kcache, const 
     __nv_bfloat16* qs = static_cast<__nv_bfloat16*>(ws);
     __nv_bfloat16* ks = qs + NS * e.q_part;
     __nv_bfloat16* vs = ks + NS * e.kv_part;
-    CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, qs, NS * bh * e.t_pad, e.hdp, TQ) || !make_map(&mk, ks, NS * bh * e.k_pad, e.hdp, TK) ||
-        !make_map(&mv, vs, NS * bh * e.hdp, e.k_pad, e.hdp))
-        return BITNET_A48_ERR_CUDA;
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, ks, NS * bh * e.k_pad, e.hdp, TK) || !make_map(&mv, vs, NS * bh * e.hdp, e.k_pad, e.hdp)) return BITNET_A48_ERR_CUDA;
     const dim3 block(256), grid_q(e.t_pad / 64, nh, B), grid_k(e.k_pad / 64, nh, B), grid_v(e.k_pad / TK, nh, B);
     if (e.hdp == 64) {
         A48_CUDA_TRY(a48_launch_pdl(attn_split_kernel<64>, grid_q, block, 0, st, q, 0, hd, T, e.t_pad, T, cap, qs, e.q_part));
@@ -625,8 +655,10 @@ bitnet_a48_status a48_launch_attn_tc(const float* q, const float* kcache, const 
     p.pos0 = pos0;
     p.bh_total = (int)bh;
     p.scale = 1.f / sqrtf((float)hd);
+    p.q_parts = qs;
+    p.q_part = e.q_part;
     p.out = out;
-    return e.hdp == 64 ? launch_attn<64>(mq, mk, mv, p, B, st) : launch_attn<128>(mq, mk, mv, p, B, st);
+    return e.hdp == 64 ? launch_attn<64>(mk, mv, p, B, st) : launch_attn<128>(mk, mv, p, B, st);
 }
 
 bitnet_a48_status a48_read_attn_status(unsigned int words_host[4]) {
