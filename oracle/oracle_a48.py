@@ -177,6 +177,36 @@ def ffn_gate_first(X, tg, ag, tu, au, td, ad, k_down, eps=1e-5):
     return y, active
 
 
+def attention_causal(q, kcache, vcache, *, B, T, n_heads, pos0=0):
+    """Causal softmax attention of the block (Section 2.1: the attention between the q/k/v BitLinears and the output
+    BitLinear is the ordinary one), written out as its definition in float64.
+
+    q [B*T, n_heads*head_dim] (already rotated); kcache, vcache [B, n_heads, cap, head_dim] holding positions
+    0 .. pos0+T-1.  Token t of a sequence sits at position pos0 + t and sees positions 0 .. pos0 + t:
+    out[t] = sum_j softmax_j(q[t] . k[j] / sqrt(head_dim)) v[j].  Returns float64 [B*T, n_heads*head_dim].
+    """
+    q = np.asarray(q, np.float64)
+    kcache = np.asarray(kcache, np.float64)
+    vcache = np.asarray(vcache, np.float64)
+    H = q.shape[1]
+    hd = H // n_heads
+    assert q.shape[0] == B * T and kcache.shape[:2] == (B, n_heads) and kcache.shape[3] == hd
+    out = np.empty((B * T, H), np.float64)
+    position = pos0 + np.arange(T)[:, None]      # of each query
+    key_index = np.arange(pos0 + T)[None, :]
+    for b in range(B):
+        for h in range(n_heads):
+            Q = q[b * T:(b + 1) * T, h * hd:(h + 1) * hd]
+            K = kcache[b, h, :pos0 + T]
+            V = vcache[b, h, :pos0 + T]
+            S = (Q @ K.T) / np.sqrt(float(hd))
+            S = np.where(key_index <= position, S, -np.inf)
+            P = np.exp(S - S.max(axis=1, keepdims=True))
+            P /= P.sum(axis=1, keepdims=True)
+            out[b * T:(b + 1) * T, h * hd:(h + 1) * hd] = P @ V
+    return out
+
+
 def block_forward(X, weights, g1, g2, *, n_heads, B, T, pos0=0, ctx_cap=0, kcache=None, vcache=None,
                   k_o, k_down, norm_eps=1e-5, quant_eps=1e-5, rope_base=10000.0, nthreads=1, act_fp4=False,
                   q_bits=0, kv_bits=0):
