@@ -55,7 +55,7 @@ NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part (2 x the 2.25 P
 SHAPE_3B = dict(H=3200, F=8640, NH=32, LAYERS=26)
 SHAPE_700M = dict(H=1536, F=4096, NH=16, LAYERS=24)  # 16 heads as the benchmark configuration fixes (head dim 96)
 SHAPE_7B = dict(H=H, F=F, NH=NH, LAYERS=LAYERS)
-ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "gatefirst", "formats", "cpu")
+ALL_LEGS = ("e2e", "decode7b", "decode3b", "prefill700m", "sweep", "block", "attention", "gatefirst", "formats", "cpu")
 
 
 def proj_list(Hs, Fs):
@@ -478,6 +478,10 @@ def run_ours(args):
         sweep = bench_sweep(a48, synth, dev, stream)
     if "block" in legs:
         block = bench_block(a48, synth, dev, stream, layer)
+    attention = None
+    if "attention" in legs:
+        attention = bench_attention(a48, synth, dev, stream, peaks)
+        rooflines.append(attention.pop("roofline"))
     gate_first = bench_gate_first(a48, synth, dev, stream) if "gatefirst" in legs else None
     formats = None
     if "formats" in legs:
@@ -510,7 +514,7 @@ def run_ours(args):
                             "window": f"first {n_burst} passes of the timed region"},
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "rooflines": rooflines, "e2e": e2e,
             "cpu_baseline": cpu_baseline, "decode": decode, "decode_3b": decode3b, "prefill_700m": prefill700m,
-            "sweep": sweep, "block": block, "ffn_gate_first": gate_first, "formats": formats,
+            "sweep": sweep, "block": block, "attention": attention, "ffn_gate_first": gate_first, "formats": formats,
         }
         print(json.dumps(line))
     reps.close()
@@ -769,6 +773,34 @@ def time_ms(fn, stream, reps, warm=3):
     e1.record(stream)
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / reps
+
+
+def bench_attention(a48, synth, dev, stream, peaks):
+    """Prefill attention of the 7B shape on its own: 4 sequences of 4096 tokens, 32 heads of 128 (the block leg's shape)."""
+    B, T, nh, hd = 4, 4096, NH, H // NH
+    g = torch.Generator(device=dev).manual_seed(91)
+    q = torch.randn(B * T, nh * hd, generator=g, device=dev)
+    kc = synth.kv_cache(B, nh, T, hd, seed=92, device=dev)
+    vc = synth.kv_cache(B, nh, T, hd, seed=93, device=dev)
+    out = torch.empty_like(q)
+    ws = torch.empty(a48.attention_prefill_workspace_bytes(B, nh, hd, T, T), dtype=torch.uint8, device=dev)
+    ms = time_ms(lambda: a48.attention_prefill(q, kc, vc, B, T, 0, out=out, workspace=ws), stream, 10)
+    flops = 4.0 * B * nh * (T * (T + 1) / 2.0) * hd  # q.k and p.v for every visible (query, key) pair
+    tiles = B * nh * sum(min(2 * (i + 1), T // 64) for i in range(T // 128))  # key tiles of 64 per 128-query tile
+    mma_flops = tiles * 6.0 * 2 * (2.0 * 128 * 64 * hd)  # six bf16 MMAs per product, whole tiles, both contractions
+    tf = flops / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    roof = {"kernel": "prefill attention, 4 x 4096 tokens, 32 heads of 128 (tcgen05 kind::f16 on bf16-split operands; "
+                      "three launches that split the operands included)",
+            "bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
+            "avg_launch_ms": ms, "algorithmic_flops_per_launch": flops,
+            "mma_tflops": mma_flops / (ms * 1e-3) / 1e12, "mma_frac": mma_flops / (ms * 1e-3) / 1e12 / peak,
+            "note": "achieved counts the attention's own flops; the kernel issues six bf16 MMAs per fp32 product to stay "
+                    "within fp32 rounding of the float64 oracle (mma_tflops counts those, whole tiles)",
+            "peak_source": f"bf16_tflops of {peaks['source']} peaks"}
+    del q, kc, vc, out, ws
+    torch.cuda.empty_cache()
+    return {"ms": ms, "tokens_per_s": B * T / (ms * 1e-3), "B": B, "T": T, "heads": nh, "head_dim": hd, "roofline": roof}
 
 
 def bench_formats(a48, synth, dev, stream, peaks, layer):

@@ -287,6 +287,26 @@ bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const fl
                                            size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * The attention of the block on its own, for a prefill (Section 2.1: between the q/k/v BitLinears and the output
+ * BitLinear the block keeps the ordinary causal softmax attention; bitnet_a48_block_forward runs this same kernel
+ * for more than 8 tokens per sequence).  out[t] = sum_j softmax_j(q[t] . k[j] / sqrt(head_dim)) v[j] per head, where
+ * token t of sequence b sits at position pos0 + t and sees positions 0 .. pos0 + t of that sequence's cache.
+ *   q_dev       fp32 [B*T, n_heads*head_dim], already rotated (read only)
+ *   kcache_dev, vcache_dev  fp32 [B, n_heads, ctx_cap, head_dim]; positions 0 .. pos0+T-1 are read, nothing is written
+ *   out_dev     fp32 [B*T, n_heads*head_dim]
+ *   workspace_dev  bitnet_a48_attention_prefill_workspace_bytes(B, n_heads, head_dim, T, pos0 + T) bytes, 16-byte
+ *               aligned (it receives the operands split into bf16 parts; no need to clear it)
+ * 1 <= head_dim <= 128 (BITNET_A48_ERR_UNSUPPORTED above), pos0 + T <= ctx_cap, B and n_heads at most 65535.  The
+ * contractions run on the tensor cores with every fp32 operand split into three bf16 parts, which keeps the result
+ * within fp32 rounding of the definition (about 4e-8 |score| relative to the largest output of a row).  All
+ * kernels run on `stream`; nothing synchronises; a bounded wait that gives up reports through
+ * bitnet_a48_kernel_status. */
+size_t bitnet_a48_attention_prefill_workspace_bytes(int B, int n_heads, int head_dim, int T, int n_keys);
+bitnet_a48_status bitnet_a48_attention_prefill(const float* q_dev, const float* kcache_dev, const float* vcache_dev, int B,
+                                               int T, int n_heads, int head_dim, int pos0, int ctx_cap, float* out_dev,
+                                               void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
  * Feed-forward sub-layer for M <= 8 tokens with the gate projection first (Section 2.1, paragraph after Eq. 5;
  * Section 3 "Sparsity"): INT4 input (Eq. 7) -> gate BitLinear (Eq. 6) -> up BitLinear only for the output channels n
  * with ReLU²(gate[m, n]) != 0 for some token m (the other rows of W_up are not read) -> Eq. 5 -> top-k + INT8

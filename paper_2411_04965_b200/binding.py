@@ -36,6 +36,7 @@ EXPORTS = [
     "bitnet_a48_ffn_gate_first", "bitnet_a48_ffn_gate_first_workspace_bytes",
     "bitnet_a48_ffn_dense", "bitnet_a48_kv_cache_bytes", "bitnet_a48_weight_layout_bytes",
     "bitnet_a48_quant_int4_bf16", "bitnet_a48_topk_quant_int8_bf16", "bitnet_a48_linear_bf16",
+    "bitnet_a48_attention_prefill", "bitnet_a48_attention_prefill_workspace_bytes",
 ]
 
 
@@ -101,6 +102,10 @@ def lib() -> ctypes.CDLL:
         L.bitnet_a48_topk_quant_int8_bf16.argtypes = [c_void_p, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p]
         L.bitnet_a48_linear_bf16.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t,
                                              c_void_p]
+        L.bitnet_a48_attention_prefill_workspace_bytes.restype = c_size_t
+        L.bitnet_a48_attention_prefill_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int]
+        L.bitnet_a48_attention_prefill.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_int,
+                                                   c_void_p, c_void_p, c_size_t, c_void_p]
         L.bitnet_a48_kv_cache_bytes.restype = c_size_t
         L.bitnet_a48_kv_cache_bytes.argtypes = [c_void_p, c_int]
         L.bitnet_a48_linear_multi.argtypes = [c_int, POINTER(c_void_p), c_void_p, c_void_p, c_int, c_int, POINTER(c_void_p),
@@ -425,6 +430,24 @@ class Block:
                                               _ptr(Y), _ptr(workspace), workspace.numel(), _stream(stream)),
                "block_forward")
         return Y
+
+
+def attention_prefill_workspace_bytes(B: int, n_heads: int, head_dim: int, T: int, n_keys: int) -> int:
+    return int(lib().bitnet_a48_attention_prefill_workspace_bytes(B, n_heads, head_dim, T, n_keys))
+
+
+def attention_prefill(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tensor, B: int, T: int, pos0: int = 0, out=None,
+                      workspace=None, stream=None) -> torch.Tensor:
+    """Causal softmax attention of a prefill.  q fp32 [B*T, n_heads*head_dim] (rotated), caches fp32 [B, n_heads, cap, head_dim]."""
+    _, n_heads, cap, hd = kcache.shape
+    if out is None:
+        out = torch.empty_like(q)
+    need = attention_prefill_workspace_bytes(B, n_heads, hd, T, pos0 + T)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    _check(lib().bitnet_a48_attention_prefill(_ptr(q), _ptr(kcache), _ptr(vcache), B, T, n_heads, hd, pos0, cap, _ptr(out),
+                                              _ptr(workspace), workspace.numel(), _stream(stream)), "attention_prefill")
+    return out
 
 
 def kernel_status():

@@ -449,6 +449,27 @@ bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const fl
                              (cudaStream_t)stream);
 }
 
+size_t bitnet_a48_attention_prefill_workspace_bytes(int B, int n_heads, int head_dim, int T, int n_keys) {
+    if (B <= 0 || n_heads <= 0 || T <= 0 || n_keys < T || !a48_attn_tc_supported(head_dim)) return 0;
+    return a48_attn_tc_workspace_bytes(B, n_heads, head_dim, T, n_keys);
+}
+
+bitnet_a48_status bitnet_a48_attention_prefill(const float* q_dev, const float* kcache_dev, const float* vcache_dev, int B,
+                                               int T, int n_heads, int head_dim, int pos0, int ctx_cap, float* out_dev,
+                                               void* workspace_dev, size_t workspace_bytes, void* stream) {
+    if (!q_dev || !kcache_dev || !vcache_dev || !out_dev || !workspace_dev) return BITNET_A48_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || n_heads <= 0 || head_dim <= 0 || pos0 < 0 || (long long)B * T > (1 << 24)) return BITNET_A48_ERR_SHAPE;
+    if ((long long)pos0 + T > ctx_cap || B > 65535 || n_heads > 65535) return BITNET_A48_ERR_SHAPE;
+    if (!a48_attn_tc_supported(head_dim)) return BITNET_A48_ERR_UNSUPPORTED;
+    if (!a48_aligned16(q_dev) || !a48_aligned16(kcache_dev) || !a48_aligned16(vcache_dev) || !a48_aligned16(out_dev) ||
+        !a48_aligned16(workspace_dev))
+        return BITNET_A48_ERR_ALIGNMENT;
+    if (workspace_bytes < a48_attn_tc_workspace_bytes(B, n_heads, head_dim, T, pos0 + T)) return BITNET_A48_ERR_NOMEM;
+    if (!have_device()) return BITNET_A48_ERR_CUDA;
+    return a48_launch_attn_tc(q_dev, kcache_dev, vcache_dev, B, T, n_heads, head_dim, pos0, ctx_cap, out_dev, workspace_dev,
+                              (cudaStream_t)stream);
+}
+
 bitnet_a48_status bitnet_a48_kernel_status(unsigned int words_host[4]) {
     if (!words_host) return BITNET_A48_ERR_INVALID_ARG;
     if (!have_device()) return BITNET_A48_ERR_CUDA;
