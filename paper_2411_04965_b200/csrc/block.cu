@@ -431,6 +431,19 @@ bitnet_a48_status launch_attn_tile(const float* q, const float* kc, const float*
     return BITNET_A48_OK;
 }
 
+// Prefill attention: the tensor-core kernel where it takes the shape (head dim <= 128, tensor-copy coordinates within
+// 32 bits), the fp32 tile kernel otherwise.
+bitnet_a48_status prefill_attention(const float* q, const float* kc, const float* vc, int B, int T, int nh, int hd, int pos0,
+                                    int cap, float* att, void* mma_ws, cudaStream_t st) {
+    if (a48_attn_tc_supported(hd)) {
+        const bitnet_a48_status s = a48_launch_attn_tc(q, kc, vc, B, T, nh, hd, pos0, cap, att, mma_ws, st);
+        if (s != BITNET_A48_ERR_UNSUPPORTED) return s;
+    }
+    if (hd <= 64) return launch_attn_tile<64>(q, kc, vc, B, T, nh, hd, pos0, cap, att, st);
+    if (hd <= 128) return launch_attn_tile<128>(q, kc, vc, B, T, nh, hd, pos0, cap, att, st);
+    return launch_attn_tile<256>(q, kc, vc, B, T, nh, hd, pos0, cap, att, st);
+}
+
 }  // namespace
 
 size_t a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int T) { return block_ws(blk, B, T).total; }
@@ -500,12 +513,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
                                             tile_path ? dq_k : nullptr, tile_path ? dq_v : nullptr, st));
         if (!tile_path) {
             A48_TRY(a48_launch_attn_row_lowbit(q, kcache, vcache, B, T, nh, hd, pos0, c.ctx_cap, c.kv_bits, att, st));
-        } else if (a48_attn_tc_supported(hd)) {
-            A48_TRY(a48_launch_attn_tc(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, base + o.mma, st));
-        } else if (hd <= 64) {
-            A48_TRY(launch_attn_tile<64>(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, st));
         } else {
-            A48_TRY(launch_attn_tile<128>(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, st));
+            A48_TRY(prefill_attention(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, base + o.mma, st));
         }
     } else {
     {
@@ -521,14 +530,8 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
         if (hd <= 64) A48_CUDA_TRY(launch_attn_row<2>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
         else if (hd <= 128) A48_CUDA_TRY(launch_attn_row<4>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
         else A48_CUDA_TRY(launch_attn_row<8>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
-    } else if (a48_attn_tc_supported(hd)) {
-        A48_TRY(a48_launch_attn_tc(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, base + o.mma, st));
-    } else if (hd <= 64) {
-        A48_TRY(launch_attn_tile<64>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
-    } else if (hd <= 128) {
-        A48_TRY(launch_attn_tile<128>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
     } else {
-        A48_TRY(launch_attn_tile<256>(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, st));
+        A48_TRY(prefill_attention(q, kcache, vcache, B, T, nh, hd, pos0, cap, att, base + o.mma, st));
     }
     }
     if (fp4) {  // the floating-point variant quantises the attention output densely (no top-K)
