@@ -279,8 +279,9 @@ size_t bitnet_a48_block_workspace_bytes(const bitnet_a48_block* blk, int B, int 
  * those positions and attention reads positions 0..own position.  The caches
  * may be NULL only when pos0 == 0 and T is the whole sequence (keys/values then
  * live in the workspace).  With kv_bits != 0 the caches are packed buffers of bitnet_a48_kv_cache_bytes bytes
- * (passed through the same pointers), head_dim <= 128, ctx_cap a multiple of 4, and a call is either a prefill from position 0 or a decode
- * step of T <= 8 tokens (BITNET_A48_ERR_UNSUPPORTED otherwise); q_bits != 0 needs kv_bits != 0.
+ * (passed through the same pointers), head_dim <= 128 and ctx_cap a multiple of 4; a call of more than 8 tokens
+ * per sequence reads the cached positions through fp32 copies in the workspace (whose size then grows with ctx_cap);
+ * q_bits != 0 needs kv_bits != 0.
  * All kernels run on `stream`; nothing synchronises. */
 bitnet_a48_status bitnet_a48_block_forward(const bitnet_a48_block* blk, const float* X_dev, int B, int T, int pos0,
                                            float* kcache_dev, float* vcache_dev, float* Y_dev, void* workspace_dev,

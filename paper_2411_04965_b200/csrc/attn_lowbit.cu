@@ -87,7 +87,8 @@ __device__ __forceinline__ void store_codes_warp(uint8_t* row, int nbytes, const
 // table: nullptr (a few tokens: the angles are evaluated here) or cos/sin pairs [T][hd/2].
 // q is overwritten with the rotated (and, q_bits != 0, quantise-dequantised) query.  The rotated key and the value
 // go to the packed caches at position pos0 + t; dq_k / dq_v (may be nullptr) receive their dequantised fp32 values
-// laid out [B][nh][T][hd] for the prefill attention kernel.
+// at position pos0 + t of copies laid out [B][nh][pos0 + T][hd] for the prefill attention kernel (the positions before
+// pos0 come from dequant_prefix_kernel).
 __global__ void __launch_bounds__(256) rope_quant_cache_kernel(float* __restrict__ q, const float* __restrict__ k,
                                                                const float* __restrict__ v, const float2* __restrict__ table,
                                                                double base, int B, int T, int nh,
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(256) rope_quant_cache_kernel(float* __restrict
     const int use_bits = (kv_bits == 3 && pos == 0) ? 4 : kv_bits;  // the bos heads keep 4 bits
     const int L = (1 << (use_bits - 1)) - 1;
     const size_t slot = ((size_t)b * nh + h) * cap + pos;
-    const size_t dq = (((size_t)b * nh + h) * T + t) * hd;
+    const size_t dq = (((size_t)b * nh + h) * (pos0 + T) + pos) * hd;  // copies hold positions 0 .. pos0 + T - 1
     for (int which = 0; which < 2; ++which) {
         const float(&x)[4] = which == 0 ? kr : vr;
         KvView view = kv_view(which == 0 ? kcache : vcache, B, nh, cap, hd, kv_bits);
@@ -177,6 +178,32 @@ __device__ __forceinline__ void load8(const uint8_t* row, int bits, int sub, boo
 #pragma unroll
     for (int i = 0; i < 8; ++i)
         f[i] = __uint_as_float(0x4B000000u | ((w >> (bits * i)) & mask)) - offset;  // exact: u - (L + 1)
+}
+
+// Positions 0 .. pos0-1 of the packed caches as fp32, into copies laid out [B][nh][rows][hd]: what a prefill that
+// starts behind cached positions hands to the attention kernel.  One warp per (sequence, head, position): lanes 0-15
+// take the key row, lanes 16-31 the value row, eight entries each.
+__global__ void __launch_bounds__(256) dequant_prefix_kernel(const void* kcache, const void* vcache, int B, int nh, int hd, int pos0,
+                                                             int cap, int rows, int kv_bits, float* __restrict__ dq_k,
+                                                             float* __restrict__ dq_v) {
+    a48_pdl_prologue();
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31, sub = lane & 15, which = lane >> 4;
+    if (warp >= (long long)B * nh * pos0) return;
+    const int pos = (int)(warp % pos0);
+    const size_t head = (size_t)(warp / pos0);  // b * nh + h
+    const KvView view = kv_view(const_cast<void*>(which == 0 ? kcache : vcache), B, nh, cap, hd, kv_bits);
+    const bool bos = kv_bits == 3 && pos == 0;  // position 0 keeps 4 bits in a 3-bit cache
+    const int bits = bos ? 4 : kv_bits;
+    const size_t slot = head * cap + pos;
+    const uint8_t* row = bos ? view.bos + head * view.row4 : view.codes + slot * view.row;
+    float f[8];
+    load8(row, bits, sub, 8 * sub < padded_dim(hd), f);
+    const float sc = view.scales[slot];
+    float* out = (which == 0 ? dq_k : dq_v) + (head * rows + pos) * hd;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if (8 * sub + i < hd) out[8 * sub + i] = sc * f[i];
 }
 
 constexpr int ATTN_SPLITS = 8;
@@ -379,6 +406,16 @@ bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const fl
     const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
     A48_CUDA_TRY(a48_launch_pdl(rope_quant_cache_kernel, dim3(blocks), dim3(256), 0, st, q, k, v, table, base, B, T, nh, hd, pos0,
                                 cap, q_bits, kv_bits, (double)eps, kcache, vcache, dq_k, dq_v));
+    return BITNET_A48_OK;
+}
+
+bitnet_a48_status a48_launch_dequant_prefix(const void* kcache, const void* vcache, int B, int nh, int hd, int pos0, int cap, int rows,
+                                            int kv_bits, float* dq_k, float* dq_v, cudaStream_t st) {
+    if (hd > 128 || hd % 4 != 0 || pos0 <= 0) return BITNET_A48_ERR_UNSUPPORTED;
+    const long long warps = (long long)B * nh * pos0;
+    const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
+    A48_CUDA_TRY(a48_launch_pdl(dequant_prefix_kernel, dim3(blocks), dim3(256), 0, st, kcache, vcache, B, nh, hd, pos0, cap, rows,
+                                kv_bits, dq_k, dq_v));
     return BITNET_A48_OK;
 }
 

@@ -29,11 +29,15 @@ BlockWs block_ws(const bitnet_a48_block* blk, int B, int T) {
     w.gate = take(M * F * 4);
     w.up = take(M * F * 4);
     w.rope = take((size_t)T * (hd / 2) * 8);
-    w.kc = take(M * H * 4);
-    w.vc = take(M * H * 4);
-    // operands of the tensor-core prefill attention split into bf16 parts: queries of the call, keys/values of every
-    // position the call can reach (the cache's capacity, or the call's own tokens without a cache)
+    // positions a call can reach: the cache's capacity, or the call's own tokens without a cache
     const int reach = blk->cfg.ctx_cap > T ? blk->cfg.ctx_cap : T;
+    // keys/values of a call without a cache; with a packed cache, the fp32 copies of every reachable position that a
+    // prefill hands to the attention kernel
+    const size_t kv_rows = blk->cfg.kv_bits != 0 && T > 8 ? (size_t)B * reach : M;
+    w.kc = take(kv_rows * H * 4);
+    w.vc = take(kv_rows * H * 4);
+    // operands of the tensor-core prefill attention split into bf16 parts: queries of the call, keys/values of every
+    // reachable position
     w.mma = take(T > 8 && a48_attn_tc_supported((int)hd) ? a48_attn_tc_workspace_bytes(B, blk->cfg.n_heads, (int)hd, T, reach) : 0);
     size_t lin = 0;
     for (int i = 0; i < 7; ++i) {
@@ -500,21 +504,24 @@ bitnet_a48_status a48_block_forward(const bitnet_a48_block* blk, const float* X,
     const bool lowbit = c.q_bits != 0 || c.kv_bits != 0;
     if (lowbit) {
         // Section 3, low-bit attention: post-RoPE absmax quantisation of the heads; packed key/value cache
-        if (c.kv_bits != 0 && (!caller_cache || (T > 8 && pos0 != 0))) return BITNET_A48_ERR_UNSUPPORTED;
+        if (c.kv_bits != 0 && !caller_cache) return BITNET_A48_ERR_UNSUPPORTED;
         const bool inline_angles = T <= 8;
         int n = T * (hd / 2);
         if (!inline_angles) rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(pos0, T, hd / 2, (double)c.rope_base, rope);
         float* dq_k = reinterpret_cast<float*>(base + o.kc);
         float* dq_v = reinterpret_cast<float*>(base + o.vc);
         if (c.kv_bits == 0) return BITNET_A48_ERR_UNSUPPORTED;  // quantised queries go with a quantised cache
-        const bool tile_path = T > 8;  // prefill from position 0: attention runs on the dequantised copies
+        const bool tile_path = T > 8;  // prefill: attention runs on dequantised fp32 copies
         A48_TRY(a48_launch_rope_quant_cache(q, k, v, inline_angles ? nullptr : rope, (double)c.rope_base, B, T, nh, hd, pos0,
                                             c.ctx_cap, c.q_bits, c.kv_bits, c.quant_eps, kcache, vcache,
                                             tile_path ? dq_k : nullptr, tile_path ? dq_v : nullptr, st));
         if (!tile_path) {
             A48_TRY(a48_launch_attn_row_lowbit(q, kcache, vcache, B, T, nh, hd, pos0, c.ctx_cap, c.kv_bits, att, st));
         } else {
-            A48_TRY(prefill_attention(q, dq_k, dq_v, B, T, nh, hd, 0, T, att, base + o.mma, st));
+            // a prefill behind cached positions: those come out of the packed cache into the fp32 copies first
+            if (pos0 > 0)
+                A48_TRY(a48_launch_dequant_prefix(kcache, vcache, B, nh, hd, pos0, c.ctx_cap, pos0 + T, c.kv_bits, dq_k, dq_v, st));
+            A48_TRY(prefill_attention(q, dq_k, dq_v, B, T, nh, hd, pos0, pos0 + T, att, base + o.mma, st));
         }
     } else {
     {

@@ -164,6 +164,8 @@ bitnet_a48_status a48_launch_rope_quant_cache(float* q, const float* k, const fl
                                               int B, int T, int nh, int hd, int pos0, int cap, int q_bits, int kv_bits,
                                               float eps, void* kcache, void* vcache, float* dq_k, float* dq_v,
                                               cudaStream_t st);
+bitnet_a48_status a48_launch_dequant_prefix(const void* kcache, const void* vcache, int B, int nh, int hd, int pos0, int cap,
+                                            int rows, int kv_bits, float* dq_k, float* dq_v, cudaStream_t st);
 bitnet_a48_status a48_launch_attn_row_lowbit(const float* q, const void* kcache, const void* vcache, int B, int T, int nh,
                                              int hd, int pos0, int cap, int kv_bits, float* out, cudaStream_t st);
 
