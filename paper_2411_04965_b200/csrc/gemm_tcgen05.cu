@@ -61,6 +61,7 @@ namespace {
 constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
 constexpr int TILE_M_WIDE = 192;   // tokens per tile (MMA N) of the prefill kernel
 constexpr int TILE_M_SKINNY = 64;  // ... and of the kernel for at most 64 tokens
+constexpr int TILE_M_MID = 128;    // ... and where 128-token tiles cover the call with as few tiles as 192-token ones
 constexpr int BK = 128;      // channels per 128-byte swizzle row of int8
 constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
 constexpr int ACC_BUFS = 2;
@@ -983,7 +984,9 @@ struct Plan {
 
 Plan make_plan(int count, const bitnet_a48_weight* const* ws, int M, bool ts) {
     Plan pl;
-    pl.tile_m = M <= TILE_M_SKINNY ? TILE_M_SKINNY : TILE_M_WIDE;
+    // 65..128 and 193..256 tokens: as many 128-token tiles as 192-token ones, and a unit of a narrower tile is shorter
+    const bool mid = M > TILE_M_SKINNY && (M + TILE_M_MID - 1) / TILE_M_MID == (M + TILE_M_WIDE - 1) / TILE_M_WIDE;
+    pl.tile_m = M <= TILE_M_SKINNY ? TILE_M_SKINNY : (mid ? TILE_M_MID : TILE_M_WIDE);
     pl.n_tiles = 0;
     for (int j = 0; j < count; ++j) pl.n_tiles += (ws[j]->N + TILE_N - 1) / TILE_N;
     pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
@@ -1168,6 +1171,9 @@ bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8
     if (pl.tile_m == TILE_M_SKINNY)
         return ss ? launch<false, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st)
                   : launch<true, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st);
+    if (pl.tile_m == TILE_M_MID)
+        return ss ? launch<false, TILE_M_MID>(1, &w, codes, scale, M, &Y, acc, pl, st)
+                  : launch<true, TILE_M_MID>(1, &w, codes, scale, M, &Y, acc, pl, st);
     return ss ? launch<false, TILE_M_WIDE>(1, &w, codes, scale, M, &Y, acc, pl, st)
               : launch<true, TILE_M_WIDE>(1, &w, codes, scale, M, &Y, acc, pl, st);
 }
@@ -1183,6 +1189,7 @@ bitnet_a48_status a48_launch_gemm_tcgen05_multi(int count, const bitnet_a48_weig
                                                 const float* scale, int M, float* const* Y, cudaStream_t st) {
     if (!a48_gemm_tcgen05_multi_supported(count, ws, M)) return BITNET_A48_ERR_UNSUPPORTED;
     const Plan pl = make_plan(count, ws, M, true);
+    if (pl.tile_m == TILE_M_MID) return launch<true, TILE_M_MID>(count, ws, codes, scale, M, Y, nullptr, pl, st);
     return pl.tile_m == TILE_M_SKINNY ? launch<true, TILE_M_SKINNY>(count, ws, codes, scale, M, Y, nullptr, pl, st)
                                       : launch<true, TILE_M_WIDE>(count, ws, codes, scale, M, Y, nullptr, pl, st);
 }

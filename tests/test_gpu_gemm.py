@@ -12,7 +12,9 @@ EPS = 1e-5
 # (M, N, K): one tile; several k-blocks; ragged M and N tails; K a multiple of 64 but not 128 (like 8640);
 # K a multiple of 16 only; several tiles per CTA wave
 SHAPES = [(256, 128, 128), (256, 128, 1024), (300, 200, 384), (70, 130, 320), (513, 257, 144), (1, 128, 256),
-          (1100, 1536, 1536)]
+          (1100, 1536, 1536),
+          # 65..128 and 193..256 tokens run on 128-token tiles: ragged second tile, few tiles with the cluster split
+          (100, 300, 512), (200, 384, 640), (250, 130, 2048), (100, 256, 4096), (250, 384, 4096), (128, 2048, 1024)]
 
 
 def _algos(a48):
