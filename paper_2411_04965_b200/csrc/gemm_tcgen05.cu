@@ -61,6 +61,7 @@ namespace {
 constexpr int TILE_N = 128;  // weight rows per tile  (MMA M)
 constexpr int TILE_M_WIDE = 192;   // tokens per tile (MMA N) of the prefill kernel
 constexpr int TILE_M_SKINNY = 64;  // ... and of the kernel for at most 64 tokens
+constexpr int TILE_M_TINY = 32;    // ... and of the same kernel for at most 32 tokens (half the token bytes per unit)
 constexpr int TILE_M_MID = 128;    // ... and where 128-token tiles cover the call with as few tiles as 192-token ones
 constexpr int BK = 128;      // channels per 128-byte swizzle row of int8
 constexpr int UMMA_K = 32;   // channels per kind::i8 MMA
@@ -79,17 +80,17 @@ struct Cfg {
     // Expander groups of four warps (TS).  A group spends about 740 clocks on a unit; at 64 tokens the kernel is
     // bound by the fill rate of shared memory (24 KB per unit and CTA), so two groups are enough there too.
     static constexpr int EXPAND_GROUPS = 2;
-    static constexpr int EPI_SPLIT = 2;  // epilogue warps per lane quadrant
+    static constexpr int EPI_SPLIT = TM >= 64 ? 2 : 1;  // epilogue warps per lane quadrant
     static constexpr int NUM_THREADS = 32 * (2 + 4 * EXPAND_GROUPS + 4 * EPI_SPLIT);
     static constexpr int EPI_COLS = TM / EPI_SPLIT;
     static_assert(EPI_COLS % 32 == 0, "the epilogue drains 32 columns at a time");
     static constexpr int KBU = TS ? 2 : 1;  // 128-channel blocks per pipeline stage
     // the narrow activation tile leaves room for a deeper ring: more weight bytes in flight per SM
-    static constexpr int STAGES = TM == TILE_M_SKINNY ? 8 : (TS ? 4 : 5);
+    static constexpr int STAGES = TM <= TILE_M_SKINNY ? 8 : (TS ? 4 : 5);
     // Tensor-memory slots of the expanded weight operand, 64 columns each.  A slot is busy from the expanders'
     // store until the MMAs that read it have completed, a round trip of well over a thousand clocks whatever
     // the MMA's size; two slots leave that round trip exposed, the narrow accumulators make room for more.
-    static constexpr int A_SLOTS = TM == TILE_M_SKINNY ? 6 : 2;
+    static constexpr int A_SLOTS = TM <= TILE_M_SKINNY ? 6 : 2;
     static_assert(A_SLOTS % EXPAND_GROUPS == 0, "unit it goes to group it % groups and to slot it % slots");
     static constexpr int STAGE_BYTES = KBU * (B_TILE_BYTES + (TS ? W_PACKED_BYTES : A_TILE_BYTES));
     static constexpr int A_SLOT_COLS = KBU * BK / 4;
@@ -986,7 +987,7 @@ Plan make_plan(int count, const bitnet_a48_weight* const* ws, int M, bool ts) {
     Plan pl;
     // 65..128 and 193..256 tokens: as many 128-token tiles as 192-token ones, and a unit of a narrower tile is shorter
     const bool mid = M > TILE_M_SKINNY && (M + TILE_M_MID - 1) / TILE_M_MID == (M + TILE_M_WIDE - 1) / TILE_M_WIDE;
-    pl.tile_m = M <= TILE_M_SKINNY ? TILE_M_SKINNY : (mid ? TILE_M_MID : TILE_M_WIDE);
+    pl.tile_m = M <= TILE_M_TINY ? TILE_M_TINY : (M <= TILE_M_SKINNY ? TILE_M_SKINNY : (mid ? TILE_M_MID : TILE_M_WIDE));
     pl.n_tiles = 0;
     for (int j = 0; j < count; ++j) pl.n_tiles += (ws[j]->N + TILE_N - 1) / TILE_N;
     pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
@@ -1171,6 +1172,9 @@ bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8
     if (pl.tile_m == TILE_M_SKINNY)
         return ss ? launch<false, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st)
                   : launch<true, TILE_M_SKINNY>(1, &w, codes, scale, M, &Y, acc, pl, st);
+    if (pl.tile_m == TILE_M_TINY)
+        return ss ? launch<false, TILE_M_TINY>(1, &w, codes, scale, M, &Y, acc, pl, st)
+                  : launch<true, TILE_M_TINY>(1, &w, codes, scale, M, &Y, acc, pl, st);
     if (pl.tile_m == TILE_M_MID)
         return ss ? launch<false, TILE_M_MID>(1, &w, codes, scale, M, &Y, acc, pl, st)
                   : launch<true, TILE_M_MID>(1, &w, codes, scale, M, &Y, acc, pl, st);
@@ -1189,6 +1193,7 @@ bitnet_a48_status a48_launch_gemm_tcgen05_multi(int count, const bitnet_a48_weig
                                                 const float* scale, int M, float* const* Y, cudaStream_t st) {
     if (!a48_gemm_tcgen05_multi_supported(count, ws, M)) return BITNET_A48_ERR_UNSUPPORTED;
     const Plan pl = make_plan(count, ws, M, true);
+    if (pl.tile_m == TILE_M_TINY) return launch<true, TILE_M_TINY>(count, ws, codes, scale, M, Y, nullptr, pl, st);
     if (pl.tile_m == TILE_M_MID) return launch<true, TILE_M_MID>(count, ws, codes, scale, M, Y, nullptr, pl, st);
     return pl.tile_m == TILE_M_SKINNY ? launch<true, TILE_M_SKINNY>(count, ws, codes, scale, M, Y, nullptr, pl, st)
                                       : launch<true, TILE_M_WIDE>(count, ws, codes, scale, M, Y, nullptr, pl, st);

@@ -132,7 +132,7 @@ def test_gemm_full_size_sampled(a48, oracle, cuda_dev):
 # several weight-row tiles, a ragged N tail, K = 3200 / 8640 (padded to whole pipeline units), M around the
 # 64-token boundary and a two-tile M of the wide kernel.
 SKINNY = [(9, 128, 512), (16, 384, 2048), (33, 200, 3200), (64, 1024, 8640), (65, 256, 2048), (100, 640, 4096),
-          (191, 130, 1536), (40, 3200, 3200)]
+          (191, 130, 1536), (40, 3200, 3200), (32, 1000, 4096), (17, 130, 11008), (31, 4096, 1024)]
 
 
 @pytest.mark.parametrize("M,N,K", SKINNY)
