@@ -213,8 +213,8 @@ bitnet_a48_status bitnet_a48_linear_ex(const bitnet_a48_weight* w, const int8_t*
             algo = BITNET_A48_ALGO_DECODE_SPARSE;
         else if (a48_decode_trit5_supported(w, M) && !w->gemm && !a48_y_bf16)
             algo = BITNET_A48_ALGO_DECODE_TRIT5;  // a handle packed for decode at 1.6 bits per weight only
-        else if (M >= 384 && a48_gemm_pair_supported(w, M))
-            algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // measured 3-11 % ahead of the single-CTA form from 384 tokens on
+        else if (a48_gemm_pair_preferred(1, &w, M))
+            algo = BITNET_A48_ALGO_GEMM_TCGEN05_PAIR;  // from 384 tokens on, unless 128-token tiles fill the SMs better
         else if (a48_gemm_tcgen05_supported(w, M, false))
             algo = BITNET_A48_ALGO_GEMM_TCGEN05;
         else
@@ -325,8 +325,8 @@ bitnet_a48_status bitnet_a48_linear_multi(int count, const bitnet_a48_weight* co
     {  // beyond the decode kernel's token count: one tensor-core launch over the tiles of all matrices
         bool any_decode = false;
         for (int j = 0; j < count; ++j) any_decode = any_decode || a48_decode_supported(weights[j], M);
-        // (from 384 tokens on a launch per matrix on CTA pairs is faster than the grouped single-CTA launch)
-        if (!any_decode && M < 384 && a48_gemm_tcgen05_multi_supported(count, weights, M))
+        // (where CTA pairs win, a launch per matrix on pairs is faster than the grouped single-CTA launch)
+        if (!any_decode && !a48_gemm_pair_preferred(count, weights, M) && a48_gemm_tcgen05_multi_supported(count, weights, M))
             return a48_launch_gemm_tcgen05_multi(count, weights, codes_dev, scale_dev, M, Y_dev, (cudaStream_t)stream);
     }
     for (int j = 0; j < count; ++j) {

@@ -54,6 +54,8 @@
 // the activation codes (q/k/v, gate/up).
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "internal.h"
 
 namespace {
@@ -983,13 +985,27 @@ struct Plan {
     int tile_m, n_tiles, m_tiles, ksplit;
 };
 
+// Time model of a launch above 64 tokens: rounds of tiles over the SMs times the time of a pipeline unit, which the
+// token sweep gives as about 0.43 us on 128-token tiles, 0.54 us on 192-token tiles and 0.50 us on 192-token tiles of
+// a CTA pair (4096 -> 11008 and 11008 -> 4096, 128 to 2048 tokens); the unit count and the fixed cost of a launch
+// are the same for the forms compared.
+long long single_cost(int n_tiles, int M, int tile_m) {
+    const long long tiles = (long long)n_tiles * ((M + tile_m - 1) / tile_m), sms = sm_count();
+    return (tiles + sms - 1) / sms * (tile_m == TILE_M_MID ? 43 : 54);
+}
+long long pair_cost(int n_tiles, int M) {
+    const long long items = (long long)((n_tiles + 1) / 2) * ((M + 191) / 192), slots = sm_count() / 2;
+    return (items + slots - 1) / slots * 50;
+}
+
 Plan make_plan(int count, const bitnet_a48_weight* const* ws, int M, bool ts) {
     Plan pl;
-    // 65..128 and 193..256 tokens: as many 128-token tiles as 192-token ones, and a unit of a narrower tile is shorter
-    const bool mid = M > TILE_M_SKINNY && (M + TILE_M_MID - 1) / TILE_M_MID == (M + TILE_M_WIDE - 1) / TILE_M_WIDE;
-    pl.tile_m = M <= TILE_M_TINY ? TILE_M_TINY : (M <= TILE_M_SKINNY ? TILE_M_SKINNY : (mid ? TILE_M_MID : TILE_M_WIDE));
     pl.n_tiles = 0;
     for (int j = 0; j < count; ++j) pl.n_tiles += (ws[j]->N + TILE_N - 1) / TILE_N;
+    // above 64 tokens: 128- or 192-token tiles, whichever leaves the CTAs less to do (fewer idle slots in the last
+    // round of tiles against a longer unit)
+    const bool mid = M > TILE_M_SKINNY && single_cost(pl.n_tiles, M, TILE_M_MID) < single_cost(pl.n_tiles, M, TILE_M_WIDE);
+    pl.tile_m = M <= TILE_M_TINY ? TILE_M_TINY : (M <= TILE_M_SKINNY ? TILE_M_SKINNY : (mid ? TILE_M_MID : TILE_M_WIDE));
     pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
     const int tiles = pl.n_tiles * pl.m_tiles, sms = sm_count();
     const int kunits = ws[0]->Kp / BK / (ts ? 2 : 1);
@@ -1152,6 +1168,22 @@ bitnet_a48_status launch_pair(const bitnet_a48_weight* w, const int8_t* codes, c
 }  // namespace
 
 bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M) { return a48_gemm_tcgen05_supported(w, M, false); }
+
+// Whether the library's own choice for these matrices on the same tokens is a CTA-pair launch per matrix rather than
+// one single-CTA launch over all their tiles.
+bool a48_gemm_pair_preferred(int count, const bitnet_a48_weight* const* ws, int M) {
+    if (M < 384) return false;
+    int n_all = 0;
+    long long pairs = 0;
+    for (int j = 0; j < count; ++j) {
+        if (!a48_gemm_pair_supported(ws[j], M)) return false;
+        const int n = (ws[j]->N + TILE_N - 1) / TILE_N;
+        n_all += n;
+        pairs += pair_cost(n, M);
+    }
+    const long long single = std::min(single_cost(n_all, M, TILE_M_MID), single_cost(n_all, M, TILE_M_WIDE));
+    return pairs <= single;
+}
 
 bitnet_a48_status a48_launch_gemm_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                        float* Y, int32_t* acc, cudaStream_t st) {

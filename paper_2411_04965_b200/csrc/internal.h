@@ -133,6 +133,7 @@ bitnet_a48_status a48_launch_gemm_tcgen05(const bitnet_a48_weight* w, const int8
                                           float* Y, int32_t* acc, bool ss, cudaStream_t st);
 // CTA-pair form (one tile of 256 weight rows per two SMs).
 bool a48_gemm_pair_supported(const bitnet_a48_weight* w, int M);
+bool a48_gemm_pair_preferred(int count, const bitnet_a48_weight* const* ws, int M);
 bitnet_a48_status a48_launch_gemm_pair(const bitnet_a48_weight* w, const int8_t* codes, const float* scale, int M,
                                        float* Y, int32_t* acc, cudaStream_t st);
 // Up to four weight matrices with one K on the same codes in one launch (tile-major layout, tensor-memory operand).
