@@ -49,6 +49,11 @@ STEP_OPS = sum(2 * M_PREFILL * n * k for _, n, k, _ in PROJ)
 # the output still in L2 when the kernel ends), scaled by the units processed: x (488 MB / 208.5 MB), the mean
 # algorithmic bytes M*K + N*K/4 + 4*M*N of the seven launches of a pass at M = 16384 over those of the captured case.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 150.9e6 * (488.0 / 208.5)
+# DRAM bytes per launch of the quantisers from the ncu captures under profiles/ (read + write): top-K + INT8 at
+# M = 4096, K = 11008 (180.5 + 28.1 MB) scaled x4 to 16384 tokens, traffic growing with the rows; INT4 at the
+# benchmark's own shape (268.4 + 51.1 MB).  In both the input is read once; part of the output is still in L2 at kernel end.
+NCU_TRAFFIC_TOPK_F = (180.5e6 + 28.1e6) * 4.0
+NCU_TRAFFIC_INT4_H = 268.4e6 + 51.1e6
 NOMINAL_INT8_TOPS = 4500.0  # dense int8 tensor peak of the part (2 x the 2.25 PFLOP/s dense bf16 figure)
 
 # the other shapes of the paper's model-configuration table used by the legs
@@ -438,19 +443,19 @@ def run_ours(args):
         roofline["library_int8_tops"] = lib
         roofline["library_int8_note"] = "torch._int_mm (vendor int8 GEMM) 8192^3, 20 calls, same GPU, outside the timed region"
 
-    def hbm_entry(kernel, names, K):
+    def hbm_entry(kernel, names, K, traffic=None):
         ms = sum(kms[n] for n in names) / len(names)
         bytes_ = 5.0 * M * K + 4.0 * M  # fp32 in, int8 out, one fp32 scale per token
         gbs = bytes_ / (ms * 1e-3) / 1e9
         return {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": gbs / peaks["hbm_gbs"], "traffic": None, "avg_launch_ms": ms,
+                "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "avg_launch_ms": ms,
                 "launches": len(names) * len(pass_events), "algorithmic_bytes_per_launch": bytes_,
                 "peak_source": f"hbm_gbs of {peaks['source']} peaks"}
 
     rooflines = [dict(roofline),
-                 hbm_entry("top-K + INT8 quantiser, 16384 x 11008 (Eq. 1, 3)", ("topk_f",), F),
+                 hbm_entry("top-K + INT8 quantiser, 16384 x 11008 (Eq. 1, 3)", ("topk_f",), F, NCU_TRAFFIC_TOPK_F),
                  hbm_entry("top-K + INT8 quantiser, 16384 x 4096 (Eq. 1, 3)", ("topk_h",), H),
-                 hbm_entry("INT4 quantiser, 16384 x 4096 (Eq. 7)", ("int4_h", "int4_h2"), H)]
+                 hbm_entry("INT4 quantiser, 16384 x 4096 (Eq. 7)", ("int4_h", "int4_h2"), H, NCU_TRAFFIC_INT4_H)]
 
     # ---- end to end with host buffers (pinned), copies inside the timed region
     e2e = bench_e2e(a48, dev, layer, work, reps, barrier, args) if "e2e" in legs else None
