@@ -268,7 +268,10 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <int CPL>
+// AHEAD: the loads of the next four keys are issued before the current four are taken.  With few CTAs (one sequence)
+// a warp's rounds of loads are what is left to wait for; with many CTAs their number hides them and the registers are
+// better spent on residency.
+template <int CPL, bool AHEAD>
 __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__ q, const float* __restrict__ kcache,
                                                        const float* __restrict__ vcache, int T, int nh, int hd,
                                                        int pos0, int cap, float scale, float* __restrict__ out) {
@@ -285,30 +288,55 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
     const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
     const float* kbase = kcache + ((size_t)b * nh + h) * cap * hd;
     const float* vbase = vcache + ((size_t)b * nh + h) * cap * hd;
+    // lane l owns the CPL consecutive head dims CPL*l .. CPL*l + CPL-1: one or two 128-bit loads per row (64-bit at CPL = 2)
+    const int col0 = lane * CPL;
+    const bool whole = col0 + CPL <= hd;  // (hd is a multiple of 4; at CPL = 8 a lane may straddle the end)
     float qreg[CPL], o[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) {
-        int col = lane + 32 * c;
-        qreg[c] = col < hd ? qr[col] * scale : 0.f;
+        qreg[c] = col0 + c < hd ? qr[col0 + c] * scale : 0.f;
         o[c] = 0.f;
     }
     float m = -INFINITY, l = 0.f;
     const int n_keys = pos0 + t + 1;
     const int per = (n_keys + ATTN_SPLITS - 1) / ATTN_SPLITS;
     const int j_end = min(n_keys, (split + 1) * per);
-    for (int j = split * per + warp; j < j_end; j += 32) {
-        float kk[4][CPL], vv[4][CPL], dot[4];
+    auto load_row = [&](const float* __restrict__ row, float (&x)[CPL]) {
+        if (whole) {
+            if constexpr (CPL == 2) {
+                const float2 f = __ldg(reinterpret_cast<const float2*>(row + col0));
+                x[0] = f.x, x[1] = f.y;
+            } else {
+#pragma unroll
+                for (int c = 0; c < CPL; c += 4) {
+                    const float4 f = __ldg(reinterpret_cast<const float4*>(row + col0 + c));
+                    x[c] = f.x, x[c + 1] = f.y, x[c + 2] = f.z, x[c + 3] = f.w;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) x[c] = col0 + c < hd ? __ldg(row + col0 + c) : 0.f;
+        }
+    };
+    // The kernel is bound by the instructions it issues per key, so four keys share one step of the online softmax
+    // (one rescale of the running output instead of four), and the exponentials are ex2.approx of a difference
+    // times log2 e (two units in the last place, as in the prefill kernel; 2^-inf = 0 covers keys past the end).
+    constexpr float kLog2e = 1.4426950408889634f;
+    auto exp2a = [](float x) {
+        float y;
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+        return y;
+    };
+    auto load4 = [&](int j, float (&kk)[4][CPL], float (&vv)[4][CPL]) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int jj = j + 8 * u;
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                const int col = lane + 32 * c;
-                const bool ok = jj < j_end && col < hd;
-                kk[u][c] = ok ? __ldg(kbase + (size_t)jj * hd + col) : 0.f;
-                vv[u][c] = ok ? __ldg(vbase + (size_t)jj * hd + col) : 0.f;
-            }
+            const int jj = max(min(j + 8 * u, j_end - 1), 0);  // (a row past the end is read again and given no weight)
+            load_row(kbase + (size_t)jj * hd, kk[u]);
+            load_row(vbase + (size_t)jj * hd, vv[u]);
         }
+    };
+    auto take4 = [&](int j, const float (&kk)[4][CPL], const float (&vv)[4][CPL]) {
+        float dot[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             dot[u] = 0.f;
@@ -321,16 +349,34 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
             for (int u = 0; u < 4; ++u) dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], off);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (j + 8 * u < j_end) {
-                const float m_new = fmaxf(m, dot[u]);
-                const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
-                const float pr = expf(dot[u] - m_new);
-                l = l * corr + pr;
+        for (int u = 1; u < 4; ++u)
+            if (j + 8 * u >= j_end) dot[u] = -INFINITY;
+        const float m_new = fmaxf(fmaxf(m, dot[0]), fmaxf(fmaxf(dot[1], dot[2]), dot[3]));  // finite: key j exists
+        const float corr = exp2a((m - m_new) * kLog2e);
+        float pr[4];
 #pragma unroll
-                for (int c = 0; c < CPL; ++c) o[c] = o[c] * corr + pr * vv[u][c];
-                m = m_new;
-            }
+        for (int u = 0; u < 4; ++u) pr[u] = exp2a((dot[u] - m_new) * kLog2e);
+        l = l * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3]));
+#pragma unroll
+        for (int c = 0; c < CPL; ++c)
+            o[c] = o[c] * corr + ((pr[0] * vv[0][c] + pr[1] * vv[1][c]) + (pr[2] * vv[2][c] + pr[3] * vv[3][c]));
+        m = m_new;
+    };
+    const int j0 = split * per + warp;
+    if constexpr (AHEAD) {
+        float ka[4][CPL], va[4][CPL], kb[4][CPL], vb[4][CPL];
+        if (j0 < j_end) load4(j0, ka, va);
+        for (int j = j0; j < j_end; j += 64) {
+            if (j + 32 < j_end) load4(j + 32, kb, vb);
+            take4(j, ka, va);
+            if (j + 64 < j_end) load4(j + 64, ka, va);
+            if (j + 32 < j_end) take4(j + 32, kb, vb);
+        }
+    } else {
+        for (int j = j0; j < j_end; j += 32) {
+            float kk[4][CPL], vv[4][CPL];
+            load4(j, kk, vv);
+            take4(j, kk, vv);
         }
     }
     if (lane == 0) {
@@ -338,7 +384,7 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
         sm_l[warp] = l;
     }
 #pragma unroll
-    for (int c = 0; c < CPL; ++c) sm_o[warp][lane + 32 * c] = o[c];
+    for (int c = 0; c < CPL; ++c) sm_o[warp][col0 + c] = o[c];
     __syncthreads();
     if (warp == 0) {
         float mm = -INFINITY;
@@ -352,14 +398,14 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
             float f = expf(sm_m[w] - mm);
             ll += sm_l[w] * f;
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][lane + 32 * c] * f;
+            for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][col0 + c] * f;
         }
         if (lane == 0) {
             cta_ml[0] = mm;
             cta_ml[1] = ll;
         }
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) cta_o[lane + 32 * c] = acc[c];
+        for (int c = 0; c < CPL; ++c) cta_o[col0 + c] = acc[c];
     }
     cluster_sync_all();  // every CTA's partial is in its shared memory
     constexpr int CPR = COLS / ATTN_SPLITS;  // columns finished by each rank
@@ -403,8 +449,13 @@ cudaError_t launch_attn_row(const float* q, const float* kcache, const float* vc
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, attn_row_kernel<CPL>, q, kcache, vcache, T, nh, hd, pos0, cap,
-                              1.f / sqrtf((float)hd), out);
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const float scale = 1.f / sqrtf((float)hd);
+    if ((long long)ATTN_SPLITS * nh * B * T <= 2ll * sms)
+        return cudaLaunchKernelEx(&cfg, attn_row_kernel<CPL, true>, q, kcache, vcache, T, nh, hd, pos0, cap, scale, out);
+    return cudaLaunchKernelEx(&cfg, attn_row_kernel<CPL, false>, q, kcache, vcache, T, nh, hd, pos0, cap, scale, out);
 }
 
 __global__ void add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ y, size_t n4) {
