@@ -290,16 +290,28 @@ __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __res
     const size_t head = (size_t)b * nh + h;
     const unsigned half_mask = 0xffffu << (lane & 16);
     const bool mine = 8 * sub < padded_dim(hd);
+    // The kernel is bound by the instructions it issues per key (ncu: 118 per key with one softmax step and two expf per
+    // key), so the exponentials are ex2.approx of a difference times log2 e (two units in the last place; 2^-inf = 0)
+    // and four keys share one step of the online softmax.
+    constexpr float kLog2e = 1.4426950408889634f;
+    auto exp2a = [](float x) {
+        float y;
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+        return y;
+    };
+    auto half_sum = [&](float v) {
+#pragma unroll
+        for (int off = 8; off > 0; off >>= 1) v += __shfl_xor_sync(half_mask, v, off);
+        return v;
+    };
     auto take = [&](const float (&kf)[8], const float (&vf)[8], float ks, float vs) {  // one key into the running softmax
         float dot = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) dot += qreg[i] * kf[i];
-#pragma unroll
-        for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(half_mask, dot, off);
-        dot *= ks;
+        dot = half_sum(dot) * ks;
         const float m_new = fmaxf(m, dot);
-        const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
-        const float pr = expf(dot - m_new);
+        const float corr = exp2a((m - m_new) * kLog2e);
+        const float pr = exp2a((dot - m_new) * kLog2e);
         l = l * corr + pr;
         const float pv = pr * vs;
 #pragma unroll
@@ -329,12 +341,41 @@ __global__ void __launch_bounds__(256) attn_row_lowbit_kernel(const float* __res
         }
         asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
         __syncthreads();
-        for (int j = c0 + halfw; j < c1; j += HALVES) {
-            if (bos_table && j == 0) continue;
-            float kf[8], vf[8];
-            unpack8(sk + (size_t)(j - ca) * row, kv_bits, sub, mine, kf);
-            unpack8(sv + (size_t)(j - ca) * row, kv_bits, sub, mine, vf);
-            take(kf, vf, sks[j - ca], svs[j - ca]);
+        for (int j = c0 + halfw; j < c1; j += 4 * HALVES) {  // keys j, j + 16, j + 32, j + 48 of this half-warp
+            float dot[4];
+            int at[4];
+            bool any = false;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int ju = j + HALVES * u;
+                const bool valid = ju < c1 && !(bos_table && ju == 0);
+                at[u] = (valid ? ju : j) - ca;  // (a key that does not count is read where key j is and given no weight)
+                float kf[8];
+                unpack8(sk + (size_t)at[u] * row, kv_bits, sub, mine, kf);
+                float d = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) d += qreg[i] * kf[i];
+                dot[u] = valid ? half_sum(d) * sks[at[u]] : -INFINITY;
+                any |= valid;
+            }
+            if (!any) continue;  // (position 0 alone, which the side table holds)
+            const float m_new = fmaxf(fmaxf(m, dot[0]), fmaxf(fmaxf(dot[1], dot[2]), dot[3]));
+            const float corr = exp2a((m - m_new) * kLog2e);
+            float pr[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) pr[u] = exp2a((dot[u] - m_new) * kLog2e);
+            l = l * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3]));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] *= corr;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float vf[8];
+                unpack8(sv + (size_t)at[u] * row, kv_bits, sub, mine, vf);
+                const float pv = pr[u] * svs[at[u]];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] += pv * vf[i];
+            }
+            m = m_new;
         }
     }
     if (sub == 0) {
