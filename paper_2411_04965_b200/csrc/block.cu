@@ -288,13 +288,17 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
     const float* qr = q + ((size_t)b * T + t) * H + (size_t)h * hd;
     const float* kbase = kcache + ((size_t)b * nh + h) * cap * hd;
     const float* vbase = vcache + ((size_t)b * nh + h) * cap * hd;
-    // lane l owns the CPL consecutive head dims CPL*l .. CPL*l + CPL-1: one or two 128-bit loads per row (64-bit at CPL = 2)
-    const int col0 = lane * CPL;
-    const bool whole = col0 + CPL <= hd;  // (hd is a multiple of 4; at CPL = 8 a lane may straddle the end)
+    // Rows that are a whole number of 128-byte lines (head dim a multiple of 32): lane l owns the CPL consecutive head
+    // dims CPL*l .. CPL*l + CPL-1 and reads them with one or two 128-bit loads (64-bit at CPL = 2).  Other head dims
+    // (100): lane l owns l, l + 32, ..., one 32-bit load each - measured, the wide loads lose a fifth of the bandwidth
+    // on rows that start in the middle of a line.
+    const bool vec = (hd & 31) == 0;
+    auto col_of = [&](int c) { return vec ? lane * CPL + c : lane + 32 * c; };
+    const bool whole = vec && lane * CPL + CPL <= hd;
     float qreg[CPL], o[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) {
-        qreg[c] = col0 + c < hd ? qr[col0 + c] * scale : 0.f;
+        qreg[c] = col_of(c) < hd ? qr[col_of(c)] * scale : 0.f;
         o[c] = 0.f;
     }
     float m = -INFINITY, l = 0.f;
@@ -304,18 +308,21 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
     auto load_row = [&](const float* __restrict__ row, float (&x)[CPL]) {
         if (whole) {
             if constexpr (CPL == 2) {
-                const float2 f = __ldg(reinterpret_cast<const float2*>(row + col0));
+                const float2 f = __ldg(reinterpret_cast<const float2*>(row + lane * CPL));
                 x[0] = f.x, x[1] = f.y;
             } else {
 #pragma unroll
                 for (int c = 0; c < CPL; c += 4) {
-                    const float4 f = __ldg(reinterpret_cast<const float4*>(row + col0 + c));
+                    const float4 f = __ldg(reinterpret_cast<const float4*>(row + lane * CPL + c));
                     x[c] = f.x, x[c + 1] = f.y, x[c + 2] = f.z, x[c + 3] = f.w;
                 }
             }
+        } else if (vec) {  // lanes past the head have nothing to read
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) x[c] = 0.f;
         } else {
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) x[c] = col0 + c < hd ? __ldg(row + col0 + c) : 0.f;
+            for (int c = 0; c < CPL; ++c) x[c] = lane + 32 * c < hd ? __ldg(row + lane + 32 * c) : 0.f;
         }
     };
     // The kernel is bound by the instructions it issues per key, so four keys share one step of the online softmax
@@ -384,7 +391,7 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
         sm_l[warp] = l;
     }
 #pragma unroll
-    for (int c = 0; c < CPL; ++c) sm_o[warp][col0 + c] = o[c];
+    for (int c = 0; c < CPL; ++c) sm_o[warp][col_of(c)] = o[c];
     __syncthreads();
     if (warp == 0) {
         float mm = -INFINITY;
@@ -398,14 +405,14 @@ __global__ void __launch_bounds__(256) attn_row_kernel(const float* __restrict__
             float f = expf(sm_m[w] - mm);
             ll += sm_l[w] * f;
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][col0 + c] * f;
+            for (int c = 0; c < CPL; ++c) acc[c] += sm_o[w][col_of(c)] * f;
         }
         if (lane == 0) {
             cta_ml[0] = mm;
             cta_ml[1] = ll;
         }
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) cta_o[col0 + c] = acc[c];
+        for (int c = 0; c < CPL; ++c) cta_o[col_of(c)] = acc[c];
     }
     cluster_sync_all();  // every CTA's partial is in its shared memory
     constexpr int CPR = COLS / ATTN_SPLITS;  // columns finished by each rank
