@@ -4,6 +4,7 @@
     python profile_cases.py quant  --M 16384 --K 4096 --kind topk --reps 3
     python profile_cases.py decode --M 1 --N 11008 --K 4096 --kind topk --copies 32 --reps 3
     python profile_cases.py block  --B 1 --T 2048 --hidden 4096 --ffn 11008 --heads 32 --reps 3
+    python profile_cases.py block  --B 1 --T 1 --ctx 2048 --reps 4          # one decode step against a cached context
 
 Each case builds seeded synthetic inputs (the same recipes the benchmark uses),
 runs the kernel `reps` times after one warm-up call and prints the mean time
@@ -63,6 +64,7 @@ def main():
     ap.add_argument("--hidden", type=int, default=4096)
     ap.add_argument("--ffn", type=int, default=11008)
     ap.add_argument("--heads", type=int, default=32)
+    ap.add_argument("--ctx", type=int, default=0, help="block: cached positions in front of the call (fp32 cache), e.g. a decode step")
     args = ap.parse_args()
     a48_build.build()
     dev = torch.device("cuda:0")
@@ -76,11 +78,16 @@ def main():
         w = {n: a48.pack_ternary(synth.ternary_latents(r, c, seed=200 + i, device=dev), EPS, a48.LAYOUT_ALL)
              for i, (n, r, c) in enumerate(shapes)}
         blk = a48.Block(w, synth.norm_gains(Hs, 60, device=dev), synth.norm_gains(Hs, 61, device=dev), n_heads=args.heads,
-                        k_o=Hs // 2, k_down=Fs // 2)
+                        k_o=Hs // 2, k_down=Fs // 2, ctx_cap=args.ctx + T if args.ctx > 0 else 0)
         x = synth.gaussian_outlier_activations(B * T, Hs, seed=13, device=dev)
         y = torch.empty_like(x)
         wsp = torch.empty(blk.workspace_bytes(B, T), dtype=torch.uint8, device=dev)
-        ms = _time(lambda: blk.forward(x, B, T, Y=y, workspace=wsp), args.reps, stream)
+        if args.ctx > 0:
+            kc = synth.kv_cache(B, args.heads, args.ctx + T, Hs // args.heads, seed=14, device=dev)
+            vc = synth.kv_cache(B, args.heads, args.ctx + T, Hs // args.heads, seed=15, device=dev)
+            ms = _time(lambda: blk.forward(x, B, T, args.ctx, kc, vc, Y=y, workspace=wsp), args.reps, stream)
+        else:
+            ms = _time(lambda: blk.forward(x, B, T, Y=y, workspace=wsp), args.reps, stream)
         hd = Hs // args.heads
         out = {"case": "block", "B": B, "T": T, "hidden": Hs, "ffn": Fs, "heads": args.heads, "ms": ms,
                "tokens_per_s": B * T / (ms * 1e-3), "attention_gflop": 4.0 * B * args.heads * (T * T / 2.0) * hd / 1e9}
